@@ -1,0 +1,87 @@
+"""ctypes front end of the C oracle (oracle/alcs_oracle.c).  Test infrastructure only.
+
+The convolution definition it evaluates is the paper's Section 3.2.2 formula at
+k_h = k_w = 1 over mask-applied weights, in double precision, plus bias and ReLU.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import functools
+
+import numpy as np
+
+from . import build as _build
+
+
+@functools.lru_cache(maxsize=None)
+def _lib(mutant: int = 0, build_dir: str | None = None):
+    lib = C.CDLL(_build.build(mutant, build_dir))
+    lib.oracle_conv1x1.restype = C.c_int
+    lib.oracle_conv1x1.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p,
+                                   C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_long,
+                                   C.c_void_p, C.c_void_p]
+    lib.oracle_conv1x1_points.restype = C.c_int
+    lib.oracle_conv1x1_points.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p,
+                                          C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_long,
+                                          C.c_void_p, C.c_long, C.c_void_p, C.c_void_p]
+    lib.oracle_num_threads.restype = C.c_int
+    lib.oracle_mutant.restype = C.c_int
+    assert lib.oracle_mutant() == mutant
+    return lib
+
+
+def num_threads() -> int:
+    """Threads the oracle's OpenMP loops will use."""
+    return int(_lib().oracle_num_threads())
+
+
+def _prep(W, mask, X, bias, g):
+    if W.dtype not in (np.float32, np.float16) or X.dtype != W.dtype:
+        raise TypeError("W and X must both be float32 or both float16")
+    W = np.ascontiguousarray(W)
+    X = np.ascontiguousarray(X)
+    mask = np.ascontiguousarray(mask, dtype=np.uint8)
+    cout, cin = W.shape
+    n, cin2, hw = X.shape
+    rows = (cout + g - 1) // g
+    if cin2 != cin or mask.shape != (rows, cin):
+        raise ValueError("shape mismatch")
+    if bias is not None:
+        bias = np.ascontiguousarray(bias, dtype=np.float32)
+        if bias.shape != (cout,):
+            raise ValueError("bias shape")
+    return W, mask, X, bias, n, cin, cout, hw
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def conv1x1(W, mask, X, bias=None, relu=False, g=4, want_scale=False, mutant=0, build_dir=None):
+    """Y[n,cout,hw] (float64) = relu?(Wm X + bias), Wm = W with dropped blocks set to zero.
+
+    With want_scale also returns A = |bias| + sum |Wm||X| (float64, same shape).
+    """
+    W, mask, X, bias, n, cin, cout, hw = _prep(W, mask, X, bias, g)
+    Y = np.empty((n, cout, hw), dtype=np.float64)
+    A = np.empty((n, cout, hw), dtype=np.float64) if want_scale else None
+    rc = _lib(mutant, build_dir).oracle_conv1x1(
+        _ptr(W), _ptr(mask), g, _ptr(X), _ptr(bias), int(bool(relu)),
+        int(W.dtype == np.float16), n, cin, cout, hw, _ptr(Y), _ptr(A))
+    if rc != 0:
+        raise RuntimeError(f"oracle_conv1x1 failed: {rc}")
+    return (Y, A) if want_scale else Y
+
+
+def conv1x1_points(W, mask, X, flat_idx, bias=None, relu=False, g=4):
+    """The same quantities at selected flat indices of Y[n,cout,hw]; returns (values, scale)."""
+    W, mask, X, bias, n, cin, cout, hw = _prep(W, mask, X, bias, g)
+    idx = np.ascontiguousarray(flat_idx, dtype=np.int64)
+    out = np.empty(idx.shape, dtype=np.float64)
+    mag = np.empty(idx.shape, dtype=np.float64)
+    rc = _lib().oracle_conv1x1_points(
+        _ptr(W), _ptr(mask), g, _ptr(X), _ptr(bias), int(bool(relu)),
+        int(W.dtype == np.float16), n, cin, cout, hw, _ptr(idx), idx.size, _ptr(out), _ptr(mag))
+    if rc != 0:
+        raise RuntimeError(f"oracle_conv1x1_points failed: {rc}")
+    return out, mag

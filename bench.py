@@ -1,0 +1,363 @@
+#!/usr/bin/env python
+"""Benchmark of the SIMD-structured sparse 1x1 convolution stack on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl alcs|reference] [--workload NAME]
+
+One "step" = one pass of the whole hot path (every pointwise layer of the stack, bias + ReLU
+fused) over one synthetic batch.  The default workload is the batch-64 MobileNetV1-224 pointwise
+stack (fp32, g = 4, per-layer block sparsity drawn from U[0.6, 0.9]); `--workload mbv1_b1` runs the
+batch-1 stack through a CUDA graph.  Prints ONE JSON line (rank 0).
+
+`--impl reference` times the CPU oracle, as it stands, on the host cores, on a bounded sample
+(a few images) of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from alcs_workloads import config_layers, make_bias, make_mask, make_weights, make_x, with_batch  # noqa: E402
+
+METRIC = "nonzero-GFLOP/s & % of roofline, SIMD-sparse 1x1 conv stack, 1 B200, b=1/64"
+UNIT = "GFLOP/s"
+WORKLOADS = {"mbv1_b64": 2, "mbv1_b1": 1, "c1": 0, "rn50_b32": 3}
+SM_COUNT, FP32_LANES = 148, 128
+
+
+def peaks():
+    """Roofline denominators: measured HBM copy bandwidth if the driver wrote it, else the
+    pool's fallback figure; fp32 CUDA-core peak derived from unit counts and the maximum clock."""
+    hbm, src, mhz = 6650.0, "fallback", 1965.0
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            hbm, src = float(d["hbm_gbs"]), "measured"
+            mhz = float(d.get("sm_max_mhz", mhz))
+        except Exception:
+            pass
+    fp32_tflops = SM_COUNT * FP32_LANES * 2 * mhz * 1e6 / 1e12
+    return hbm, src, fp32_tflops, mhz
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0=None, t1=None):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], None, set()
+        for ts, line in self.lines:
+            if t0 is not None and not (t0 - 0.05 <= ts <= t1 + 0.15):
+                continue
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0])); mx = float(f[1])
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def layer_stats(spec, nb):
+    """Algorithmic work of one layer: nonzero FLOPs and bytes (X, Y, packed W, bias moved once)."""
+    elt = 4 if spec.dtype == "f32" else 2
+    q = spec.n * spec.hw
+    flops = 2.0 * nb * spec.g * q
+    packed = nb * (spec.g * elt + 4) + (spec.rows + 1) * 4
+    byts = packed + q * spec.cin * elt + q * spec.cout * elt + 4 * spec.cout
+    return flops, byts
+
+
+def oracle_sample(specs, target_s=15.0):
+    """Time the oracle on the first `b` images of every layer; returns (nz GFLOP/s, cores, text)."""
+    import oracle
+    arrs = []
+    for s in specs:
+        arrs.append((make_weights(s), make_mask(s), make_bias(s)))
+
+    def run(b):
+        t = 0.0
+        nz = 0.0
+        for s, (W, M, bias) in zip(specs, arrs):
+            sb = with_batch(s, min(b, s.n))
+            X = make_x(sb)
+            t0 = time.perf_counter()
+            oracle.conv1x1(W, M, X, bias, s.relu, s.g)
+            t += time.perf_counter() - t0
+            nz += layer_stats(sb, int(M.sum()))[0]
+        return t, nz
+
+    t1, nz1 = run(1)
+    b = int(max(1, min(specs[0].n, target_s / max(t1, 1e-3))))
+    if b > 1:
+        t1, nz1 = run(b)
+    return nz1 / t1 / 1e9, oracle.num_threads(), f"first {b} of {specs[0].n} images of every layer, one pass", t1
+
+
+def run_reference(args, specs, wl):
+    """The oracle as the reference arm: each step is one pass over a bounded sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    arrs = [(make_weights(s), make_mask(s), make_bias(s)) for s in specs]
+    b = 1 if specs[0].n > 1 else 1
+    sub = [with_batch(s, min(b, s.n)) for s in specs]
+    xs = [make_x(s) for s in sub]
+    nz = sum(layer_stats(s, int(a[1].sum()))[0] for s, a in zip(sub, arrs))
+
+    def step():
+        for s, (W, M, bias), X in zip(sub, arrs, xs):
+            oracle.conv1x1(W, M, X, bias, s.relu, s.g)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / args.steps
+    val = nz / dt / 1e9
+    sample = f"{b} of {specs[0].n} images of every layer per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl, "layers": len(specs), "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="alcs", choices=["alcs", "reference"])
+    ap.add_argument("--workload", default="mbv1_b64", choices=sorted(WORKLOADS))
+    ap.add_argument("--no-tune", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--layers", default="", help="comma-separated layer indices (default: all)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "alcs" else args.warmup
+    wl = args.workload
+    specs = config_layers(WORKLOADS[wl])
+    if args.layers:
+        specs = [specs[int(i)] for i in args.layers.split(",")]
+
+    if args.impl == "reference":
+        return run_reference(args, specs, wl)
+
+    import torch
+    import torch.distributed as dist
+    import paper_2109_00170_b200 as A
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    A.lib()
+    stream = torch.cuda.Stream()
+    graph = wl in ("mbv1_b1", "c1")
+
+    # ---- set-up (untimed): inputs, packing, upload, tuning -----------------------------------
+    layers, keep, stats = [], [], []
+    host = []
+    for s in specs:
+        W, M, X, b = make_weights(s), make_mask(s), make_x(s), make_bias(s)
+        p = A.alcs_packed_upload(A.alcs_pack(W, M, s.g), local)
+        xd = torch.from_numpy(X).to(dev)
+        ydt = torch.float32 if s.dtype == "f32" else torch.float16
+        yd = torch.empty((s.n, s.cout, s.hw), dtype=ydt, device=dev)
+        bd = torch.from_numpy(b).to(dev)
+        flags = A.ALCS_RELU if s.relu else 0
+        with torch.cuda.stream(stream):
+            cfg = (A.alcs_spconv1x1_plan(p, s.n, s.h, s.w, flags) if args.no_tune
+                   else A.alcs_spconv1x1_tune(p, xd, yd, s.n, s.h, s.w, bd, flags, stream))
+        layers.append(dict(w=p, x=xd, y=yd, n=s.n, h=s.h, wd=s.w, bias=bd, flags=flags))
+        nb = int(M.sum())
+        fl, by = layer_stats(s, nb)
+        stats.append(dict(name=s.name, nb=nb, sparsity=1 - nb / M.size, flops=fl, bytes=by, cfg=cfg))
+        host.append((X, b))
+        keep.append((W, M))
+    stack = A.alcs_stack_create(layers, A.ALCS_STACK_GRAPH if graph else 0)
+    total_flops = sum(st["flops"] for st in stats)
+    total_bytes = sum(st["bytes"] for st in stats)
+    hbm_gbs, peak_src, fp32_tf, sm_max = peaks()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- region A: K whole-stack steps, nothing between the launches ------------------------
+    for _ in range(args.warmup):
+        A.alcs_stack_run(stack, stream)
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    tw0 = time.time()
+    e0.record(stream)
+    for _ in range(args.steps):
+        A.alcs_stack_run(stack, stream)
+    e1.record(stream)
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+
+    # ---- region B: the same steps with an event between layers (per-layer durations) --------
+    nl = len(layers)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(nl + 1)] for _ in range(args.steps)]
+    for k in range(args.steps):
+        evs[k][0].record(stream)
+        for i, L in enumerate(layers):
+            A.alcs_spconv1x1(L["w"], L["x"], L["y"], L["n"], L["h"], L["wd"], L["bias"], L["flags"], stream)
+            evs[k][i + 1].record(stream)
+    barrier()
+    tw1 = time.time()
+    clocks = sampler.stop(tw0, tw1) if rank == 0 else None
+    per_layer_ms = [statistics.mean(evs[k][i].elapsed_time(evs[k][i + 1]) for k in range(args.steps)) for i in range(nl)]
+    per_layer_min = [min(evs[k][i].elapsed_time(evs[k][i + 1]) for k in range(args.steps)) for i in range(nl)]
+
+    if world > 1:
+        t = torch.tensor([ms_total], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    value = world * total_flops / (ms_step * 1e-3) / 1e9
+
+    # ---- end to end: host buffers through alcs_spconv1x1_host, copies inside the timed region --
+    e2e = None
+    if args.e2e_steps > 0:
+        ws_bytes = max(A.alcs_spconv1x1_host_workspace(L["w"], L["n"], L["h"], L["wd"], L["flags"]) for L in layers)
+        ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+        xh = [torch.from_numpy(X).pin_memory() for X, _ in host]
+        bh = [torch.from_numpy(b).pin_memory() for _, b in host]
+        yh = [torch.empty(tuple(L["y"].shape), dtype=L["y"].dtype).pin_memory() for L in layers]
+        h2d = sum(x.numel() * x.element_size() for x in xh) + sum(b.numel() * 4 for b in bh)
+        d2h = sum(y.numel() * y.element_size() for y in yh)
+
+        def e2e_step():
+            for L, x, y, b in zip(layers, xh, yh, bh):
+                A.alcs_spconv1x1_host(L["w"], x, y, L["n"], L["h"], L["wd"], b, L["flags"], ws, ws_bytes, stream)
+
+        e2e_step()
+        barrier()
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record(stream)
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        f1.record(stream)
+        barrier()
+        ms_e2e = f0.elapsed_time(f1)
+        if world > 1:
+            t = torch.tensor([ms_e2e], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_e2e = float(t.item())
+        ms_e2e /= args.e2e_steps
+        e2e = {"value": world * total_flops / (ms_e2e * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms_e2e,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": args.e2e_steps}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- per-layer roofline ------------------------------------------------------------------
+    rows = []
+    for st, ms, mn in zip(stats, per_layer_ms, per_layer_min):
+        t_hbm = st["bytes"] / (hbm_gbs * 1e9)
+        t_alu = st["flops"] / (fp32_tf * 1e12)
+        t_roof = max(t_hbm, t_alu)
+        rows.append(dict(layer=st["name"], sparsity=round(st["sparsity"], 4), kept_blocks=st["nb"],
+                         nz_mflop=round(st["flops"] / 1e6, 1), mbytes=round(st["bytes"] / 1e6, 2),
+                         t_roof_us=round(t_roof * 1e6, 2), bound="hbm" if t_hbm >= t_alu else "alu",
+                         us=round(ms * 1e3, 2), us_min=round(mn * 1e3, 2),
+                         nz_gflops=round(st["flops"] / (ms * 1e-3) / 1e9, 1),
+                         frac=round(t_roof / (ms * 1e-3), 4), cfg=st["cfg"]))
+    dom = max(range(nl), key=lambda i: per_layer_ms[i])
+    d = rows[dom]
+    if d["bound"] == "hbm":
+        ach = stats[dom]["bytes"] / (per_layer_ms[dom] * 1e-3) / 1e9
+        roof = {"bound": "hbm", "achieved": ach, "peak": hbm_gbs, "unit": "GB/s", "frac": ach / hbm_gbs}
+    else:
+        ach = stats[dom]["flops"] / (per_layer_ms[dom] * 1e-3) / 1e12
+        roof = {"bound": "alu", "achieved": ach, "peak": fp32_tf, "unit": "TFLOP/s", "frac": ach / fp32_tf}
+    roof.update({"traffic": None, "kernel": "spconv1x1_kernel", "layer": d["layer"],
+                 "peak_source": f"HBM {peak_src}; fp32 = {SM_COUNT} SMs x {FP32_LANES} lanes x 2 x {sm_max:.0f} MHz"})
+    sum_roof = sum(r["t_roof_us"] for r in rows)
+    sum_us = sum(r["us"] for r in rows)
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        v, cores, sample, secs = oracle_sample(specs)
+        cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample, "seconds": round(secs, 2)}
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32" if specs[0].dtype == "f32" else "f16", "data": "synthetic",
+        "config": {"workload": wl, "layers": nl, "batch": specs[0].n, "g": specs[0].g,
+                   "cache": "inputs larger than L2: one step touches %.0f MB of distinct X and Y" % (total_bytes / 1e6),
+                   "cuda_graph": graph, "tuned": not args.no_tune},
+        "roofline": roof,
+        "stack_roofline": {"sum_t_roof_us": round(sum_roof, 1), "sum_layer_us": round(sum_us, 1),
+                           "frac": round(sum_roof / sum_us, 4), "min_layer_frac": min(r["frac"] for r in rows),
+                           "us_per_layer": round(ms_step * 1e3 / nl, 2)},
+        "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": nl * args.steps, "clocks": clocks,
+        "layers": rows,
+    }
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,240 @@
+/*
+ * alcs.h -- C ABI of the SIMD-structured sparse pointwise (1x1) convolution for NVIDIA B200.
+ *
+ *   Y[n, cout, h*w] = W_sparse[cout, cin] x X[n, cin, h*w] + bias   (optionally ReLU)
+ *
+ * W is pruned in blocks of g consecutive output channels that share one input-channel index
+ * (paper, Section 3.2.1 "SIMD-structured pruning": the parameters at the same location of g
+ * adjacent filters form one group and are kept or removed together; different groups of filters
+ * may have different zero locations).  Block row r = output channels r*g .. r*g+g-1.
+ *
+ * General conventions
+ *   - Every function returns an int status: ALCS_OK (0) or a negative alcs_status.  Nothing
+ *     throws, aborts or prints.  alcs_strerror() names a status; alcs_last_cuda_error() gives
+ *     the CUDA runtime's text for the calling thread's last ALCS_ERR_CUDA.
+ *   - "host" pointers are ordinary CPU memory; "device" pointers are CUDA global memory of the
+ *     device the packed weights were uploaded to.  The caller owns every buffer it passes in;
+ *     the library owns alcs_packed and alcs_stack objects until the matching free/destroy.
+ *   - cuda_stream arguments are cudaStream_t values passed as void* (NULL = the default stream).
+ *     Device work is enqueued asynchronously; no call synchronises unless stated.
+ *   - Index type is int32.  Supported group sizes for packing: 1..64; for the GPU kernels:
+ *     1, 2, 4, 8, 16 (others: ALCS_ERR_UNSUPPORTED).
+ *   - There is no CPU implementation of the convolution in this library.  On a machine without a
+ *     usable CUDA device every device entry point fails with ALCS_ERR_CUDA.
+ */
+#ifndef ALCS_H_
+#define ALCS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define ALCS_API __attribute__((visibility("default")))
+#else
+#define ALCS_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ALCS_VERSION 1
+
+typedef enum {
+    ALCS_OK = 0,
+    ALCS_ERR_INVALID_ARG = -1,  /* null pointer, negative size, misaligned or aliased buffer        */
+    ALCS_ERR_SHAPE = -2,        /* sizes that do not fit together or overflow int32 indexing        */
+    ALCS_ERR_UNSUPPORTED = -3,  /* valid request the kernels do not implement (g, dtype, ...)       */
+    ALCS_ERR_ALLOC = -4,        /* host or device allocation failed                                 */
+    ALCS_ERR_CUDA = -5,         /* a CUDA runtime call failed; see alcs_last_cuda_error()           */
+    ALCS_ERR_CORRUPT = -6,      /* a serialized blob failed validation                              */
+    ALCS_ERR_STATE = -7         /* object not in the required state (e.g. weights not uploaded)     */
+} alcs_status;
+
+typedef enum {
+    ALCS_F32 = 0,               /* fp32 weights, activations and outputs, fp32 accumulation         */
+    ALCS_F16 = 1                /* IEEE binary16 weights and activations, fp32 accumulation         */
+} alcs_dtype;
+
+/* Bits of the `flags` argument of the convolution entry points. */
+#define ALCS_RELU 1u            /* y = max(acc + bias, 0)                                           */
+#define ALCS_Y_F32 2u           /* ALCS_F16 weights only: write Y as fp32 instead of fp16           */
+
+typedef struct alcs_packed alcs_packed;   /* opaque packed weight matrix, library-owned */
+typedef struct alcs_stack alcs_stack;     /* opaque layer stack, library-owned          */
+
+ALCS_API const char* alcs_strerror(int status);
+ALCS_API const char* alcs_last_cuda_error(void);
+ALCS_API int alcs_version(void);
+
+/* ---------------------------------------------------------------------------------------------
+ * Packing (host only).
+ *
+ * Storage format: paper, Section 3.2.2, paragraph "Storage format of SIMD-structured sparse
+ * tensor" -- a grouped CSR that keeps, for each group of g filters, the number of non-zero
+ * columns, one column offset per non-zero column (the number of columns before it in the
+ * flattened kernel matrix, i.e. its absolute 0-based index) and the non-zero values, g per
+ * column.  Here the three parts of all R = ceil(cout/g) groups are concatenated:
+ *     row_ptr[R+1]   row_ptr[r+1]-row_ptr[r] = number of kept columns of group r
+ *     col_idx[nb]    ascending inside a group
+ *     vals[nb*g]     value j of kept block k at vals[k*g + j], j = channel inside the group
+ * The mask decides what is kept, not the values: a kept block is stored even if all-zero and a
+ * dropped block is dropped even if non-zero.  Values are copied bit for bit.  If cout is not a
+ * multiple of g the last group is padded with +0 rows.
+ * ------------------------------------------------------------------------------------------- */
+
+/*
+ * alcs_pack: w is row-major [cout][cin] of dtype dt (host); block_mask is [ceil(cout/g)][cin]
+ * bytes (host), non-zero = keep.  On success *out receives a new packed matrix (free it with
+ * alcs_packed_free).  Errors: INVALID_ARG (null, g outside 1..64), SHAPE (cout/cin <= 0 or
+ * too many blocks for int32), ALLOC.
+ */
+ALCS_API int alcs_pack(const void* w, const uint8_t* block_mask, int cout, int cin, int g, alcs_dtype dt,
+              alcs_packed** out);
+
+/*
+ * alcs_unpack: inverse of alcs_pack.  w_out [cout][cin] of the packed dtype receives the kept
+ * values and +0 for dropped blocks; mask_out [ceil(cout/g)][cin] receives 0/1.  Either may be
+ * NULL.  Host pointers.
+ */
+ALCS_API int alcs_unpack(const alcs_packed* p, void* w_out, uint8_t* mask_out);
+
+/*
+ * alcs_packed_view: borrow the packed arrays (host memory owned by p, valid until p is freed).
+ * Any output pointer may be NULL.  *nb receives the number of kept blocks.
+ */
+ALCS_API int alcs_packed_view(const alcs_packed* p, int* cout, int* cin, int* g, alcs_dtype* dt, int* nb,
+                     const int32_t** row_ptr, const int32_t** col_idx, const void** vals);
+
+/*
+ * Serialisation to a flat, position-independent little-endian byte blob
+ * (header | row_ptr | col_idx | vals).  Call alcs_packed_serialize with buf == NULL to get the
+ * size in *nbytes; with a buffer, *nbytes is its capacity on entry and the bytes written on
+ * return.  alcs_packed_deserialize validates everything (magic, version, sizes, monotone row_ptr,
+ * ascending in-range columns) and returns ALCS_ERR_CORRUPT otherwise.  Host pointers.
+ */
+ALCS_API int alcs_packed_serialize(const alcs_packed* p, void* buf, size_t* nbytes);
+ALCS_API int alcs_packed_deserialize(const void* buf, size_t nbytes, alcs_packed** out);
+
+/*
+ * alcs_packed_upload: copy the packed matrix (and the launch schedule derived from it) to CUDA
+ * device `device`.  Allocates device memory owned by p, enqueues the copies on cuda_stream and
+ * waits for them, so p is usable on any stream when the call returns.  Uploading twice is an
+ * ALCS_ERR_STATE.  This is the "done in advance" re-organisation of the paper's storage-format
+ * paragraph: it is not part of the timed path.
+ */
+ALCS_API int alcs_packed_upload(alcs_packed* p, int device, void* cuda_stream);
+
+/* Free host and device memory of p (NULL is allowed). */
+ALCS_API void alcs_packed_free(alcs_packed* p);
+
+/* ---------------------------------------------------------------------------------------------
+ * The convolution (device).
+ *
+ * Operation: paper, Section 3.2.2, the convolution formula
+ *     O(n,h,w) = sum_c sum_r sum_s W(n,c,r,s) I(c,h+r,w+s)
+ * at k_h = k_w = 1, stride 1, evaluated as in the paragraph "Efficient multiplication
+ * computation": for every group, loop over its kept columns, multiply the column's g weights
+ * with the input values addressed by the column offset and accumulate.  Bias and ReLU are a
+ * fused epilogue.
+ * ------------------------------------------------------------------------------------------- */
+
+/*
+ * Launch configuration override, for tuning and tests.  Zero in a field means "choose".
+ *   pixels_per_lane   4 or 8: each warp covers 32*pixels_per_lane consecutive pixels
+ *   rows_per_warp     block rows whose accumulators one warp holds at a time
+ *   warps             warps per thread block (8 or 16)
+ *   chunk_channels    input channels staged in shared memory per pipeline stage
+ *   stages            pipeline depth (2..4)
+ *   row_groups        how many thread blocks share one pixel tile, each taking a slice of rows
+ *   min_blocks        thread blocks per SM the kernel is compiled for (1 or 2)
+ */
+typedef struct {
+    int pixels_per_lane, rows_per_warp, warps, chunk_channels, stages, row_groups, min_blocks;
+} alcs_launch_cfg;
+
+/*
+ * Introspection of the compiled kernel variants (host only): alcs_variant_count() entries, each a
+ * (dtype, g, pixels_per_lane, rows_per_warp, warps, min_blocks) combination that
+ * alcs_spconv1x1_cfg accepts; the other fields of *cfg are set to 0.
+ */
+ALCS_API int alcs_variant_count(void);
+ALCS_API int alcs_variant_get(int index, alcs_dtype* dt, int* g, alcs_launch_cfg* cfg);
+
+/*
+ * alcs_spconv1x1: x device [n][cin][h*wd], y device [n][cout][h*wd], both contiguous NCHW of the
+ * packed dtype (y fp32 if ALCS_Y_F32); bias device fp32 [cout] or NULL; flags = ALCS_RELU |
+ * ALCS_Y_F32.  x and y must not overlap and must be aligned to their element size; 16-byte
+ * aligned buffers with h*wd a multiple of 4 (fp32) or 8 (fp16) take the vectorised path, anything
+ * else a slower element-wise path with identical results.  Enqueues one kernel on cuda_stream;
+ * no allocation, no synchronisation.  n == 0 or h*wd == 0 is a successful no-op.
+ * Errors: INVALID_ARG, SHAPE (n*channels*pixels beyond int32 tiles), UNSUPPORTED (g), STATE (not
+ * uploaded / wrong current device), CUDA.
+ */
+ALCS_API int alcs_spconv1x1(const alcs_packed* w, const void* x, void* y, int n, int h, int wd,
+                   const float* bias, unsigned flags, void* cuda_stream);
+
+/* Same, with an explicit launch configuration (cfg == NULL behaves like alcs_spconv1x1). */
+ALCS_API int alcs_spconv1x1_cfg(const alcs_packed* w, const void* x, void* y, int n, int h, int wd,
+                       const float* bias, unsigned flags, const alcs_launch_cfg* cfg,
+                       void* cuda_stream);
+
+/*
+ * alcs_spconv1x1_plan: report the launch configuration alcs_spconv1x1 would use for this shape
+ * (host only, no device work).
+ */
+ALCS_API int alcs_spconv1x1_plan(const alcs_packed* w, int n, int h, int wd, unsigned flags,
+                        alcs_launch_cfg* out);
+
+/*
+ * alcs_spconv1x1_tune: time the candidate launch configurations for this shape on the given
+ * buffers (y is overwritten with the correct result each time), remember the fastest in w for
+ * later alcs_spconv1x1 calls with the same (n, h, wd, flags), and write it to *best (may be
+ * NULL).  Synchronises the stream; meant for set-up time, never for the timed path.
+ */
+ALCS_API int alcs_spconv1x1_tune(alcs_packed* w, const void* x, void* y, int n, int h, int wd,
+                        const float* bias, unsigned flags, void* cuda_stream,
+                        alcs_launch_cfg* best);
+
+/*
+ * alcs_spconv1x1_host: the same operation on HOST buffers x_host / y_host / bias_host, staged
+ * through a caller-provided device workspace of at least alcs_spconv1x1_host_workspace() bytes
+ * (256-byte aligned).  Enqueues H2D copies, the kernel and the D2H copy on cuda_stream and
+ * returns without synchronising; use pinned host memory for truly asynchronous copies.
+ */
+ALCS_API size_t alcs_spconv1x1_host_workspace(const alcs_packed* w, int n, int h, int wd, unsigned flags);
+ALCS_API int alcs_spconv1x1_host(const alcs_packed* w, const void* x_host, void* y_host, int n, int h,
+                        int wd, const float* bias_host, unsigned flags, void* workspace,
+                        size_t workspace_bytes, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Layer stack: a network's pointwise layers run back to back on one stream (paper, Section 3.3,
+ * T(W) = tau + sum_l T_l(W_l): the network's run time is the sum over its layers).
+ * ------------------------------------------------------------------------------------------- */
+
+typedef struct {
+    const alcs_packed* w;       /* uploaded packed weights                     */
+    const void* x;              /* device [n][cin][h*wd]                       */
+    void* y;                    /* device [n][cout][h*wd]                      */
+    int n, h, wd;
+    const float* bias;          /* device fp32 [cout] or NULL                  */
+    unsigned flags;             /* ALCS_RELU | ALCS_Y_F32                      */
+} alcs_layer;
+
+#define ALCS_STACK_GRAPH 1u     /* replay the launches as one CUDA graph       */
+
+/*
+ * alcs_stack_create copies the layer descriptions (the buffers stay the caller's and must outlive
+ * the stack) and fixes each layer's launch configuration.  With ALCS_STACK_GRAPH the first
+ * alcs_stack_run captures the launches into a CUDA graph on that stream and later runs replay it.
+ * alcs_stack_run enqueues all layers in order on cuda_stream without synchronising.
+ */
+ALCS_API int alcs_stack_create(const alcs_layer* layers, int n_layers, unsigned stack_flags,
+                      alcs_stack** out);
+ALCS_API int alcs_stack_run(alcs_stack* s, void* cuda_stream);
+ALCS_API int alcs_stack_destroy(alcs_stack* s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ALCS_H_ */

@@ -1,0 +1,315 @@
+"""Thin ctypes binding of libalcs.so: argument marshalling only, same names as the C ABI
+(include/alcs.h).  Every step of the convolution runs in the library's CUDA kernels; there is no
+Python or CPU fallback, and loading fails loudly if the shared object has not been built.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libalcs.so")
+
+ALCS_OK = 0
+ALCS_ERR_INVALID_ARG, ALCS_ERR_SHAPE, ALCS_ERR_UNSUPPORTED, ALCS_ERR_ALLOC = -1, -2, -3, -4
+ALCS_ERR_CUDA, ALCS_ERR_CORRUPT, ALCS_ERR_STATE = -5, -6, -7
+ALCS_F32, ALCS_F16 = 0, 1
+ALCS_RELU, ALCS_Y_F32 = 1, 2
+ALCS_STACK_GRAPH = 1
+
+# every symbol include/alcs.h declares
+EXPORTS = ["alcs_strerror", "alcs_last_cuda_error", "alcs_version", "alcs_pack", "alcs_unpack",
+           "alcs_packed_view", "alcs_packed_serialize", "alcs_packed_deserialize",
+           "alcs_packed_upload", "alcs_packed_free", "alcs_variant_count", "alcs_variant_get",
+           "alcs_spconv1x1", "alcs_spconv1x1_cfg",
+           "alcs_spconv1x1_plan", "alcs_spconv1x1_tune", "alcs_spconv1x1_host_workspace",
+           "alcs_spconv1x1_host", "alcs_stack_create", "alcs_stack_run", "alcs_stack_destroy"]
+
+
+class AlcsError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().alcs_strerror(status).decode()
+        if status == ALCS_ERR_CUDA:
+            msg += " [" + lib().alcs_last_cuda_error().decode() + "]"
+        super().__init__(f"{where}: {msg}")
+
+
+class LaunchCfg(C.Structure):
+    _fields_ = [(k, C.c_int) for k in ("pixels_per_lane", "rows_per_warp", "warps",
+                                       "chunk_channels", "stages", "row_groups", "min_blocks")]
+
+    def as_dict(self):
+        return {k: getattr(self, k) for k, _ in self._fields_}
+
+
+class Layer(C.Structure):
+    _fields_ = [("w", C.c_void_p), ("x", C.c_void_p), ("y", C.c_void_p), ("n", C.c_int),
+                ("h", C.c_int), ("wd", C.c_int), ("bias", C.c_void_p), ("flags", C.c_uint)]
+
+
+_lib = None
+
+
+def lib():
+    """Load libalcs.so once.  Raises if it is missing: there is nothing to fall back to."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} not found: build it with `python -m paper_2109_00170_b200.build`")
+    L = C.CDLL(LIB_PATH)
+    vp, ip, u, i, sz = C.c_void_p, C.POINTER(C.c_int), C.c_uint, C.c_int, C.c_size_t
+    L.alcs_strerror.restype = C.c_char_p
+    L.alcs_strerror.argtypes = [i]
+    L.alcs_last_cuda_error.restype = C.c_char_p
+    L.alcs_version.restype = i
+    L.alcs_pack.argtypes = [vp, vp, i, i, i, i, C.POINTER(vp)]
+    L.alcs_unpack.argtypes = [vp, vp, vp]
+    L.alcs_packed_view.argtypes = [vp, ip, ip, ip, ip, ip, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp)]
+    L.alcs_packed_serialize.argtypes = [vp, vp, C.POINTER(sz)]
+    L.alcs_packed_deserialize.argtypes = [vp, sz, C.POINTER(vp)]
+    L.alcs_packed_upload.argtypes = [vp, i, vp]
+    L.alcs_packed_free.argtypes = [vp]
+    L.alcs_packed_free.restype = None
+    L.alcs_variant_count.restype = i
+    L.alcs_variant_get.argtypes = [i, ip, ip, C.POINTER(LaunchCfg)]
+    L.alcs_spconv1x1.argtypes = [vp, vp, vp, i, i, i, vp, u, vp]
+    L.alcs_spconv1x1_cfg.argtypes = [vp, vp, vp, i, i, i, vp, u, C.POINTER(LaunchCfg), vp]
+    L.alcs_spconv1x1_plan.argtypes = [vp, i, i, i, u, C.POINTER(LaunchCfg)]
+    L.alcs_spconv1x1_tune.argtypes = [vp, vp, vp, i, i, i, vp, u, vp, C.POINTER(LaunchCfg)]
+    L.alcs_spconv1x1_host_workspace.argtypes = [vp, i, i, i, u]
+    L.alcs_spconv1x1_host_workspace.restype = sz
+    L.alcs_spconv1x1_host.argtypes = [vp, vp, vp, i, i, i, vp, u, vp, sz, vp]
+    L.alcs_stack_create.argtypes = [C.POINTER(Layer), i, u, C.POINTER(vp)]
+    L.alcs_stack_run.argtypes = [vp, vp]
+    L.alcs_stack_destroy.argtypes = [vp]
+    for name in EXPORTS:
+        f = getattr(L, name)
+        if f.restype is C.c_int and name not in ("alcs_version",):
+            f.restype = i
+    _lib = L
+    return L
+
+
+def _check(status: int, where: str):
+    if status != ALCS_OK:
+        raise AlcsError(status, where)
+
+
+def _addr(t) -> Optional[int]:
+    """Address of a torch tensor, a numpy array, an int, or None."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    if hasattr(t, "data_ptr"):
+        return t.data_ptr()
+    if isinstance(t, np.ndarray):
+        return t.ctypes.data
+    raise TypeError(type(t))
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        return None
+    if isinstance(stream, int):
+        return stream or None
+    return stream.cuda_stream or None     # torch.cuda.Stream
+
+
+def _cfg(cfg) -> Optional[LaunchCfg]:
+    if cfg is None or isinstance(cfg, LaunchCfg):
+        return cfg
+    return LaunchCfg(**cfg)
+
+
+class Packed:
+    """Owner of one alcs_packed object."""
+
+    def __init__(self, handle: int):
+        self._h = C.c_void_p(handle)
+
+    @property
+    def handle(self):
+        if not self._h:
+            raise AlcsError(ALCS_ERR_STATE, "Packed (freed)")
+        return self._h
+
+    def free(self):
+        if self._h:
+            lib().alcs_packed_free(self._h)
+            self._h = C.c_void_p(None)
+
+    def __del__(self):
+        try:
+            self.free()
+        except Exception:
+            pass
+
+
+def alcs_pack(w: np.ndarray, block_mask: np.ndarray, g: int) -> Packed:
+    """w: [cout, cin] float32 or float16 (host); block_mask: [ceil(cout/g), cin] uint8."""
+    if w.dtype == np.float32:
+        dt = ALCS_F32
+    elif w.dtype == np.float16:
+        dt = ALCS_F16
+    else:
+        raise TypeError("weights must be float32 or float16")
+    w = np.ascontiguousarray(w)
+    block_mask = np.ascontiguousarray(block_mask, dtype=np.uint8)
+    cout, cin = w.shape
+    if block_mask.shape != ((cout + max(g, 1) - 1) // max(g, 1), cin):
+        raise ValueError("block_mask shape")
+    out = C.c_void_p()
+    _check(lib().alcs_pack(w.ctypes.data, block_mask.ctypes.data, cout, cin, g, dt, C.byref(out)), "alcs_pack")
+    return Packed(out.value)
+
+
+def alcs_packed_view(p: Packed):
+    """Copies of the packed arrays: dict(cout, cin, g, dtype, nb, row_ptr, col_idx, vals)."""
+    cout, cin, g, dt, nb = (C.c_int() for _ in range(5))
+    rp, ci, va = C.c_void_p(), C.c_void_p(), C.c_void_p()
+    _check(lib().alcs_packed_view(p.handle, cout, cin, g, dt, nb, C.byref(rp), C.byref(ci), C.byref(va)),
+           "alcs_packed_view")
+    rows = (cout.value + g.value - 1) // g.value
+    npdt = np.float32 if dt.value == ALCS_F32 else np.float16
+
+    def arr(ptr, n, t):
+        if n == 0:
+            return np.zeros(0, dtype=t)
+        return np.ctypeslib.as_array(C.cast(ptr, C.POINTER(C.c_uint8)), shape=(n * np.dtype(t).itemsize,)).view(t).copy()
+
+    return dict(cout=cout.value, cin=cin.value, g=g.value, dtype=dt.value, nb=nb.value,
+                row_ptr=arr(rp, rows + 1, np.int32), col_idx=arr(ci, nb.value, np.int32),
+                vals=arr(va, nb.value * g.value, npdt))
+
+
+def alcs_unpack(p: Packed):
+    v = alcs_packed_view(p)
+    npdt = np.float32 if v["dtype"] == ALCS_F32 else np.float16
+    rows = (v["cout"] + v["g"] - 1) // v["g"]
+    w = np.empty((v["cout"], v["cin"]), dtype=npdt)
+    m = np.empty((rows, v["cin"]), dtype=np.uint8)
+    _check(lib().alcs_unpack(p.handle, w.ctypes.data, m.ctypes.data), "alcs_unpack")
+    return w, m
+
+
+def alcs_packed_serialize(p: Packed) -> bytes:
+    n = C.c_size_t(0)
+    _check(lib().alcs_packed_serialize(p.handle, None, C.byref(n)), "alcs_packed_serialize")
+    buf = (C.c_uint8 * n.value)()
+    _check(lib().alcs_packed_serialize(p.handle, buf, C.byref(n)), "alcs_packed_serialize")
+    return bytes(buf)
+
+
+def alcs_packed_deserialize(blob: bytes) -> Packed:
+    out = C.c_void_p()
+    buf = (C.c_uint8 * len(blob)).from_buffer_copy(blob) if len(blob) else (C.c_uint8 * 1)()
+    _check(lib().alcs_packed_deserialize(buf, len(blob), C.byref(out)), "alcs_packed_deserialize")
+    return Packed(out.value)
+
+
+def alcs_packed_upload(p: Packed, device: int = 0, stream=None) -> Packed:
+    _check(lib().alcs_packed_upload(p.handle, device, _stream(stream)), "alcs_packed_upload")
+    return p
+
+
+def alcs_packed_free(p: Packed):
+    p.free()
+
+
+def alcs_variant_count() -> int:
+    return int(lib().alcs_variant_count())
+
+
+def alcs_variant_get(index: int) -> dict:
+    """dict(dtype, g, pixels_per_lane, rows_per_warp, warps, min_blocks, ...) of one variant."""
+    dt, g, c = C.c_int(), C.c_int(), LaunchCfg()
+    _check(lib().alcs_variant_get(index, dt, g, C.byref(c)), "alcs_variant_get")
+    return dict(dtype=dt.value, g=g.value, **c.as_dict())
+
+
+def alcs_spconv1x1(w: Packed, x, y, n: int, h: int, wd: int, bias=None, flags: int = 0, stream=None,
+                   cfg=None):
+    """x, y, bias: device tensors (anything with data_ptr()) or raw device addresses."""
+    c = _cfg(cfg)
+    if c is None:
+        st = lib().alcs_spconv1x1(w.handle, _addr(x), _addr(y), n, h, wd, _addr(bias), flags, _stream(stream))
+    else:
+        st = lib().alcs_spconv1x1_cfg(w.handle, _addr(x), _addr(y), n, h, wd, _addr(bias), flags,
+                                      C.byref(c), _stream(stream))
+    _check(st, "alcs_spconv1x1")
+
+
+def alcs_spconv1x1_plan(w: Packed, n: int, h: int, wd: int, flags: int = 0) -> dict:
+    c = LaunchCfg()
+    _check(lib().alcs_spconv1x1_plan(w.handle, n, h, wd, flags, C.byref(c)), "alcs_spconv1x1_plan")
+    return c.as_dict()
+
+
+def alcs_spconv1x1_tune(w: Packed, x, y, n: int, h: int, wd: int, bias=None, flags: int = 0,
+                        stream=None) -> dict:
+    c = LaunchCfg()
+    _check(lib().alcs_spconv1x1_tune(w.handle, _addr(x), _addr(y), n, h, wd, _addr(bias), flags,
+                                     _stream(stream), C.byref(c)), "alcs_spconv1x1_tune")
+    return c.as_dict()
+
+
+def alcs_spconv1x1_host_workspace(w: Packed, n: int, h: int, wd: int, flags: int = 0) -> int:
+    return int(lib().alcs_spconv1x1_host_workspace(w.handle, n, h, wd, flags))
+
+
+def alcs_spconv1x1_host(w: Packed, x_host, y_host, n: int, h: int, wd: int, bias_host=None,
+                        flags: int = 0, workspace=None, workspace_bytes: int = 0, stream=None):
+    """x_host / y_host / bias_host: host arrays (numpy, or pinned torch CPU tensors)."""
+    _check(lib().alcs_spconv1x1_host(w.handle, _addr(x_host), _addr(y_host), n, h, wd, _addr(bias_host),
+                                     flags, _addr(workspace), workspace_bytes, _stream(stream)),
+           "alcs_spconv1x1_host")
+
+
+class Stack:
+    """Owner of one alcs_stack object."""
+
+    def __init__(self, handle, keep):
+        self._h = C.c_void_p(handle)
+        self._keep = keep      # keeps the Packed objects and tensors alive
+
+    @property
+    def handle(self):
+        if not self._h:
+            raise AlcsError(ALCS_ERR_STATE, "Stack (destroyed)")
+        return self._h
+
+    def destroy(self):
+        if self._h:
+            lib().alcs_stack_destroy(self._h)
+            self._h = C.c_void_p(None)
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def alcs_stack_create(layers: Sequence[dict], stack_flags: int = 0) -> Stack:
+    """layers: dicts with keys w (Packed), x, y, n, h, wd, bias (optional), flags (optional)."""
+    arr = (Layer * max(1, len(layers)))()
+    for k, L in enumerate(layers):
+        arr[k] = Layer(L["w"].handle, _addr(L["x"]), _addr(L["y"]), L["n"], L["h"], L["wd"],
+                       _addr(L.get("bias")), L.get("flags", 0))
+    out = C.c_void_p()
+    _check(lib().alcs_stack_create(arr, len(layers), stack_flags, C.byref(out)), "alcs_stack_create")
+    return Stack(out.value, list(layers))
+
+
+def alcs_stack_run(s: Stack, stream=None):
+    _check(lib().alcs_stack_run(s.handle, _stream(stream)), "alcs_stack_run")
+
+
+def alcs_stack_destroy(s: Stack):
+    s.destroy()

@@ -1,0 +1,282 @@
+// Host side of libalcs: the grouped-CSR packer (paper, Section 3.2.2, storage-format paragraph),
+// its inverse, the serialised blob, and the launch schedules derived from a packed matrix.
+// No CUDA in this file.
+#include <algorithm>
+#include <cstring>
+#include <limits>
+#include <new>
+#include <numeric>
+
+#include "alcs_internal.h"
+
+namespace {
+
+constexpr uint32_t kMagic = 0x53434C41u;  // "ALCS" little-endian
+constexpr uint32_t kBlobVersion = 1;
+
+struct BlobHeader {
+    uint32_t magic, version;
+    int32_t cout, cin, g, dtype, rows, nb;
+};
+
+thread_local const char* g_cuda_err = "";
+
+}  // namespace
+
+namespace alcs {
+
+void set_cuda_error_text(const char* s) { g_cuda_err = s ? s : ""; }
+
+float half_bits_to_float(uint16_t h)
+{
+    // binary16 -> binary32, exact.  Handles zeros, subnormals, infinities and NaNs.
+    const uint32_t sign = (uint32_t)(h & 0x8000u) << 16;
+    uint32_t ex = (h >> 10) & 0x1fu;
+    uint32_t man = h & 0x3ffu;
+    uint32_t bits;
+    if (ex == 0) {
+        if (man == 0) {
+            bits = sign;
+        } else {
+            int shift = 0;
+            while (!(man & 0x400u)) { man <<= 1; ++shift; }
+            man &= 0x3ffu;
+            bits = sign | ((uint32_t)(127 - 15 - shift + 1) << 23) | (man << 13);
+        }
+    } else if (ex == 31) {
+        bits = sign | 0x7f800000u | (man << 13);
+    } else {
+        bits = sign | ((ex + 127 - 15) << 23) | (man << 13);
+    }
+    float f;
+    std::memcpy(&f, &bits, 4);
+    return f;
+}
+
+void build_row_order(const alcs_packed& p, std::vector<int>& order)
+{
+    order.resize(p.rows);
+    std::iota(order.begin(), order.end(), 0);
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+        return p.row_ptr[a + 1] - p.row_ptr[a] > p.row_ptr[b + 1] - p.row_ptr[b];
+    });
+}
+
+void build_schedule(const alcs_packed& p, int kc, HostSchedule& out)
+{
+    if (kc <= 0 || kc > p.cin) kc = p.cin;
+    const int nch = (p.cin + kc - 1) / kc;
+    out.kc = kc;
+    out.nch = nch;
+    out.seg_ptr.assign((size_t)p.rows * (nch + 1), 0);
+    out.cols.clear();
+    out.vals.clear();
+    out.cols.reserve(p.nb + (size_t)p.rows * nch);
+    out.vals.reserve(((size_t)p.nb + (size_t)p.rows * nch) * p.g);
+    const int g = p.g;
+    for (int r = 0; r < p.rows; ++r) {
+        int k = p.row_ptr[r];
+        const int kend = p.row_ptr[r + 1];
+        for (int c = 0; c < nch; ++c) {
+            out.seg_ptr[(size_t)r * (nch + 1) + c] = (int)out.cols.size();
+            const int lim = (c + 1) * kc;
+            int cnt = 0;
+            while (k < kend && p.col_idx[k] < lim) {
+                out.cols.push_back(p.col_idx[k] - c * kc);
+                for (int j = 0; j < g; ++j) {
+                    const size_t vi = (size_t)k * g + j;
+                    float v;
+                    if (p.dt == ALCS_F32) {
+                        std::memcpy(&v, &p.vals[vi * 4], 4);
+                    } else {
+                        uint16_t hb;
+                        std::memcpy(&hb, &p.vals[vi * 2], 2);
+                        v = half_bits_to_float(hb);
+                    }
+                    out.vals.push_back(v);
+                }
+                ++k;
+                ++cnt;
+            }
+            if (cnt & 1) {  // pad to an even count: same column again, zero weights
+                out.cols.push_back(out.cols.back());
+                for (int j = 0; j < g; ++j) out.vals.push_back(0.0f);
+            }
+        }
+        out.seg_ptr[(size_t)r * (nch + 1) + nch] = (int)out.cols.size();
+    }
+    out.nbp = (int)out.cols.size();
+}
+
+}  // namespace alcs
+
+extern "C" {
+
+ALCS_API const char* alcs_strerror(int status)
+{
+    switch (status) {
+        case ALCS_OK: return "ALCS_OK";
+        case ALCS_ERR_INVALID_ARG: return "ALCS_ERR_INVALID_ARG: null, negative, misaligned or overlapping argument";
+        case ALCS_ERR_SHAPE: return "ALCS_ERR_SHAPE: sizes do not fit together or exceed int32 indexing";
+        case ALCS_ERR_UNSUPPORTED: return "ALCS_ERR_UNSUPPORTED: group size, dtype or option not implemented";
+        case ALCS_ERR_ALLOC: return "ALCS_ERR_ALLOC: allocation failed";
+        case ALCS_ERR_CUDA: return "ALCS_ERR_CUDA: CUDA runtime call failed";
+        case ALCS_ERR_CORRUPT: return "ALCS_ERR_CORRUPT: serialized blob failed validation";
+        case ALCS_ERR_STATE: return "ALCS_ERR_STATE: object not in the required state";
+        default: return "unknown ALCS status";
+    }
+}
+
+ALCS_API const char* alcs_last_cuda_error(void) { return g_cuda_err; }
+
+ALCS_API int alcs_version(void) { return ALCS_VERSION; }
+
+ALCS_API int alcs_pack(const void* w, const uint8_t* block_mask, int cout, int cin, int g, alcs_dtype dt,
+              alcs_packed** out)
+{
+    if (!w || !block_mask || !out) return ALCS_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (g < 1 || g > 64) return ALCS_ERR_INVALID_ARG;
+    if (dt != ALCS_F32 && dt != ALCS_F16) return ALCS_ERR_UNSUPPORTED;
+    if (cout <= 0 || cin <= 0) return ALCS_ERR_SHAPE;
+    const int rows = (cout + g - 1) / g;
+    // count kept blocks first so that overflow is detected before anything is allocated
+    uint64_t nb64 = 0;
+    for (size_t i = 0, e = (size_t)rows * cin; i < e; ++i) nb64 += block_mask[i] != 0;
+    // the device schedules pad every (row, 32-channel chunk) segment by at most one block and
+    // index values as block * g with int32
+    const uint64_t worst = (nb64 + (uint64_t)rows * (uint64_t)((cin + 31) / 32)) * (uint64_t)g;
+    if (worst >= (uint64_t)std::numeric_limits<int32_t>::max()) return ALCS_ERR_SHAPE;
+    alcs_packed* p = new (std::nothrow) alcs_packed();
+    if (!p) return ALCS_ERR_ALLOC;
+    try {
+        p->cout = cout; p->cin = cin; p->g = g; p->rows = rows; p->dt = dt; p->nb = (int)nb64;
+        const size_t es = p->elt();
+        p->row_ptr.assign(rows + 1, 0);
+        p->col_idx.resize(nb64);
+        p->vals.assign((size_t)nb64 * g * es, 0);
+        const uint8_t* wb = static_cast<const uint8_t*>(w);
+        int k = 0;
+        for (int r = 0; r < rows; ++r) {
+            p->row_ptr[r] = k;
+            for (int c = 0; c < cin; ++c) {
+                if (!block_mask[(size_t)r * cin + c]) continue;
+                p->col_idx[k] = c;
+                for (int j = 0; j < g; ++j) {
+                    const int co = r * g + j;
+                    if (co < cout)
+                        std::memcpy(&p->vals[((size_t)k * g + j) * es], wb + ((size_t)co * cin + c) * es, es);
+                }
+                ++k;
+            }
+        }
+        p->row_ptr[rows] = k;
+    } catch (const std::bad_alloc&) {
+        delete p;
+        return ALCS_ERR_ALLOC;
+    }
+    *out = p;
+    return ALCS_OK;
+}
+
+ALCS_API int alcs_unpack(const alcs_packed* p, void* w_out, uint8_t* mask_out)
+{
+    if (!p) return ALCS_ERR_INVALID_ARG;
+    const size_t es = p->elt();
+    if (w_out) std::memset(w_out, 0, (size_t)p->cout * p->cin * es);
+    if (mask_out) std::memset(mask_out, 0, (size_t)p->rows * p->cin);
+    uint8_t* wb = static_cast<uint8_t*>(w_out);
+    for (int r = 0; r < p->rows; ++r) {
+        for (int k = p->row_ptr[r]; k < p->row_ptr[r + 1]; ++k) {
+            const int c = p->col_idx[k];
+            if (mask_out) mask_out[(size_t)r * p->cin + c] = 1;
+            if (!wb) continue;
+            for (int j = 0; j < p->g; ++j) {
+                const int co = r * p->g + j;
+                if (co < p->cout)
+                    std::memcpy(wb + ((size_t)co * p->cin + c) * es, &p->vals[((size_t)k * p->g + j) * es], es);
+            }
+        }
+    }
+    return ALCS_OK;
+}
+
+ALCS_API int alcs_packed_view(const alcs_packed* p, int* cout, int* cin, int* g, alcs_dtype* dt, int* nb,
+                     const int32_t** row_ptr, const int32_t** col_idx, const void** vals)
+{
+    if (!p) return ALCS_ERR_INVALID_ARG;
+    if (cout) *cout = p->cout;
+    if (cin) *cin = p->cin;
+    if (g) *g = p->g;
+    if (dt) *dt = p->dt;
+    if (nb) *nb = p->nb;
+    if (row_ptr) *row_ptr = p->row_ptr.data();
+    if (col_idx) *col_idx = p->col_idx.data();
+    if (vals) *vals = p->vals.data();
+    return ALCS_OK;
+}
+
+ALCS_API int alcs_packed_serialize(const alcs_packed* p, void* buf, size_t* nbytes)
+{
+    if (!p || !nbytes) return ALCS_ERR_INVALID_ARG;
+    const size_t need = sizeof(BlobHeader) + p->row_ptr.size() * 4 + p->col_idx.size() * 4 + p->vals.size();
+    if (!buf) { *nbytes = need; return ALCS_OK; }
+    if (*nbytes < need) { *nbytes = need; return ALCS_ERR_SHAPE; }
+    BlobHeader h{kMagic, kBlobVersion, p->cout, p->cin, p->g, (int32_t)p->dt, p->rows, p->nb};
+    uint8_t* o = static_cast<uint8_t*>(buf);
+    std::memcpy(o, &h, sizeof h); o += sizeof h;
+    std::memcpy(o, p->row_ptr.data(), p->row_ptr.size() * 4); o += p->row_ptr.size() * 4;
+    if (!p->col_idx.empty()) std::memcpy(o, p->col_idx.data(), p->col_idx.size() * 4);
+    o += p->col_idx.size() * 4;
+    if (!p->vals.empty()) std::memcpy(o, p->vals.data(), p->vals.size());
+    *nbytes = need;
+    return ALCS_OK;
+}
+
+ALCS_API int alcs_packed_deserialize(const void* buf, size_t nbytes, alcs_packed** out)
+{
+    if (!buf || !out) return ALCS_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (nbytes < sizeof(BlobHeader)) return ALCS_ERR_CORRUPT;
+    BlobHeader h;
+    std::memcpy(&h, buf, sizeof h);
+    if (h.magic != kMagic || h.version != kBlobVersion) return ALCS_ERR_CORRUPT;
+    if (h.cout <= 0 || h.cin <= 0 || h.g < 1 || h.g > 64 || h.nb < 0) return ALCS_ERR_CORRUPT;
+    if (h.dtype != ALCS_F32 && h.dtype != ALCS_F16) return ALCS_ERR_CORRUPT;
+    if (h.rows != (h.cout + h.g - 1) / h.g) return ALCS_ERR_CORRUPT;
+    if ((uint64_t)h.nb > (uint64_t)h.rows * (uint64_t)h.cin) return ALCS_ERR_CORRUPT;
+    const size_t es = h.dtype == ALCS_F32 ? 4 : 2;
+    const size_t need = sizeof h + ((size_t)h.rows + 1) * 4 + (size_t)h.nb * 4 + (size_t)h.nb * h.g * es;
+    if (nbytes != need) return ALCS_ERR_CORRUPT;
+    alcs_packed* p = new (std::nothrow) alcs_packed();
+    if (!p) return ALCS_ERR_ALLOC;
+    try {
+        p->cout = h.cout; p->cin = h.cin; p->g = h.g; p->rows = h.rows; p->nb = h.nb;
+        p->dt = (alcs_dtype)h.dtype;
+        const uint8_t* in = static_cast<const uint8_t*>(buf) + sizeof h;
+        p->row_ptr.resize((size_t)h.rows + 1);
+        std::memcpy(p->row_ptr.data(), in, p->row_ptr.size() * 4); in += p->row_ptr.size() * 4;
+        p->col_idx.resize(h.nb);
+        if (h.nb) std::memcpy(p->col_idx.data(), in, (size_t)h.nb * 4);
+        in += (size_t)h.nb * 4;
+        p->vals.resize((size_t)h.nb * h.g * es);
+        if (!p->vals.empty()) std::memcpy(p->vals.data(), in, p->vals.size());
+    } catch (const std::bad_alloc&) {
+        delete p;
+        return ALCS_ERR_ALLOC;
+    }
+    bool ok = p->row_ptr[0] == 0 && p->row_ptr[h.rows] == h.nb;
+    for (int r = 0; ok && r < h.rows; ++r) {
+        const int a = p->row_ptr[r], b = p->row_ptr[r + 1];
+        if (a > b || b > h.nb || a < 0) { ok = false; break; }
+        for (int k = a; k < b; ++k) {
+            const int c = p->col_idx[k];
+            if (c < 0 || c >= h.cin || (k > a && c <= p->col_idx[k - 1])) { ok = false; break; }
+        }
+    }
+    if (!ok) { delete p; return ALCS_ERR_CORRUPT; }
+    *out = p;
+    return ALCS_OK;
+}
+
+}  // extern "C"

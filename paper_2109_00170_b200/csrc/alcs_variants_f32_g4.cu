@@ -1,0 +1,31 @@
+// Compiled variants of the fp32, g = 4 kernel (the paper's group size for 32-bit weights on
+// 128-bit SIMD registers, Section 4.1).
+#include "alcs_kernels.cuh"
+
+namespace alcs {
+
+static const KernelVariant kTable[] = {
+    //            XT   f16 G  P RW  NW MINB
+    ALCS_VARIANT(float, 0, 4, 8, 1, 8, 2),
+    ALCS_VARIANT(float, 0, 4, 8, 2, 8, 2),
+    ALCS_VARIANT(float, 0, 4, 8, 3, 8, 1),
+    ALCS_VARIANT(float, 0, 4, 8, 4, 8, 1),
+    ALCS_VARIANT(float, 0, 4, 8, 1, 16, 1),
+    ALCS_VARIANT(float, 0, 4, 8, 2, 16, 1),
+    ALCS_VARIANT(float, 0, 4, 8, 3, 16, 1),
+    ALCS_VARIANT(float, 0, 4, 4, 1, 8, 4),
+    ALCS_VARIANT(float, 0, 4, 4, 2, 8, 4),
+    ALCS_VARIANT(float, 0, 4, 4, 2, 8, 2),
+    ALCS_VARIANT(float, 0, 4, 4, 4, 8, 2),
+    ALCS_VARIANT(float, 0, 4, 4, 8, 8, 1),
+    ALCS_VARIANT(float, 0, 4, 4, 4, 16, 1),
+    ALCS_VARIANT(float, 0, 4, 4, 6, 16, 1),
+};
+
+const KernelVariant* variants_f32_g4(int* n)
+{
+    *n = (int)(sizeof(kTable) / sizeof(kTable[0]));
+    return kTable;
+}
+
+}  // namespace alcs

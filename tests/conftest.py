@@ -25,3 +25,13 @@ def pytest_collection_modifyitems(config, items):
     for it in items:
         if "gpu" in it.keywords:
             it.add_marker(skip)
+
+
+@pytest.fixture(scope="session")
+def alcs():
+    """The Python binding, with libalcs.so built if it is stale (nvcc cross-compiles on CPU)."""
+    from paper_2109_00170_b200 import build as _b
+    _b.build()
+    import paper_2109_00170_b200 as A
+    A.lib()
+    return A

@@ -117,13 +117,22 @@ ALCS_API int alcs_packed_serialize(const alcs_packed* p, void* buf, size_t* nbyt
 ALCS_API int alcs_packed_deserialize(const void* buf, size_t nbytes, alcs_packed** out);
 
 /*
- * alcs_packed_upload: copy the packed matrix (and the launch schedule derived from it) to CUDA
- * device `device`.  Allocates device memory owned by p, enqueues the copies on cuda_stream and
- * waits for them, so p is usable on any stream when the call returns.  Uploading twice is an
- * ALCS_ERR_STATE.  This is the "done in advance" re-organisation of the paper's storage-format
- * paragraph: it is not part of the timed path.
+ * alcs_packed_upload: bind the packed matrix to CUDA device `device`.  The launch schedule (the
+ * packed blocks re-ordered for one launch configuration) is built and copied to the device the
+ * first time a convolution, alcs_spconv1x1_tune or alcs_stack_create needs it for a new shape; that
+ * first call allocates device memory owned by p and waits for the copy, later calls do neither.
+ * Uploading twice is an ALCS_ERR_STATE.  This is the "done in advance" re-organisation of the
+ * paper's storage-format paragraph: it is not part of the timed path.
  */
 ALCS_API int alcs_packed_upload(alcs_packed* p, int device, void* cuda_stream);
+
+/*
+ * alcs_packed_status: read the device error word of p (synchronises with the device).  *code is 0
+ * unless a kernel gave up one of its bounded waits: 1 = a consumer warp waited too long for data,
+ * 2 = the producer warp waited too long for a free pipeline stage.  A non-zero code means the
+ * outputs of that launch are incomplete.
+ */
+ALCS_API int alcs_packed_status(const alcs_packed* p, int* code);
 
 /* Free host and device memory of p (NULL is allowed). */
 ALCS_API void alcs_packed_free(alcs_packed* p);
@@ -143,10 +152,10 @@ ALCS_API void alcs_packed_free(alcs_packed* p);
  * Launch configuration override, for tuning and tests.  Zero in a field means "choose".
  *   pixels_per_lane   4 or 8: each warp covers 32*pixels_per_lane consecutive pixels
  *   rows_per_warp     block rows whose accumulators one warp holds at a time
- *   warps             warps per thread block (8 or 16)
+ *   warps             consumer warps per thread block (one more warp only moves data)
  *   chunk_channels    input channels staged in shared memory per pipeline stage
- *   stages            pipeline depth (2..4)
- *   row_groups        how many thread blocks share one pixel tile, each taking a slice of rows
+ *   stages            pipeline depth (2..8)
+ *   row_groups        how many work items share one pixel tile, each taking a subset of rows
  *   min_blocks        thread blocks per SM the kernel is compiled for (1 or 2)
  */
 typedef struct {
@@ -167,7 +176,7 @@ ALCS_API int alcs_variant_get(int index, alcs_dtype* dt, int* g, alcs_launch_cfg
  * ALCS_Y_F32.  x and y must not overlap and must be aligned to their element size; 16-byte
  * aligned buffers with h*wd a multiple of 4 (fp32) or 8 (fp16) take the vectorised path, anything
  * else a slower element-wise path with identical results.  Enqueues one kernel on cuda_stream;
- * no allocation, no synchronisation.  n == 0 or h*wd == 0 is a successful no-op.
+ * no allocation and no synchronisation once this shape has been seen (see alcs_packed_upload).  n == 0 or h*wd == 0 is a successful no-op.
  * Errors: INVALID_ARG, SHAPE (n*channels*pixels beyond int32 tiles), UNSUPPORTED (g), STATE (not
  * uploaded / wrong current device), CUDA.
  */

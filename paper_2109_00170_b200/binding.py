@@ -23,7 +23,7 @@ ALCS_STACK_GRAPH = 1
 # every symbol include/alcs.h declares
 EXPORTS = ["alcs_strerror", "alcs_last_cuda_error", "alcs_version", "alcs_pack", "alcs_unpack",
            "alcs_packed_view", "alcs_packed_serialize", "alcs_packed_deserialize",
-           "alcs_packed_upload", "alcs_packed_free", "alcs_variant_count", "alcs_variant_get",
+           "alcs_packed_upload", "alcs_packed_status", "alcs_packed_free", "alcs_variant_count", "alcs_variant_get",
            "alcs_spconv1x1", "alcs_spconv1x1_cfg",
            "alcs_spconv1x1_plan", "alcs_spconv1x1_tune", "alcs_spconv1x1_host_workspace",
            "alcs_spconv1x1_host", "alcs_stack_create", "alcs_stack_run", "alcs_stack_destroy"]
@@ -73,6 +73,7 @@ def lib():
     L.alcs_packed_serialize.argtypes = [vp, vp, C.POINTER(sz)]
     L.alcs_packed_deserialize.argtypes = [vp, sz, C.POINTER(vp)]
     L.alcs_packed_upload.argtypes = [vp, i, vp]
+    L.alcs_packed_status.argtypes = [vp, ip]
     L.alcs_packed_free.argtypes = [vp]
     L.alcs_packed_free.restype = None
     L.alcs_variant_count.restype = i
@@ -216,6 +217,13 @@ def alcs_packed_deserialize(blob: bytes) -> Packed:
 def alcs_packed_upload(p: Packed, device: int = 0, stream=None) -> Packed:
     _check(lib().alcs_packed_upload(p.handle, device, _stream(stream)), "alcs_packed_upload")
     return p
+
+
+def alcs_packed_status(p: Packed) -> int:
+    """Device error word of p: 0 unless a kernel gave up a bounded wait."""
+    code = C.c_int(0)
+    _check(lib().alcs_packed_status(p.handle, code), "alcs_packed_status")
+    return code.value
 
 
 def alcs_packed_free(p: Packed):

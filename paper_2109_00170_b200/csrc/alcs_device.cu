@@ -88,55 +88,108 @@ int prepare_variant(VariantInfo& vi)
     return ALCS_OK;
 }
 
-int schedule_index_for_kc(const alcs_packed* w, int kc)
+using alcs::Plan;
+using alcs::Schedule;
+
+struct StageLayout {
+    int off_rec, off_rowoff, stage_bytes;
+};
+
+StageLayout stage_layout(const KernelVariant& v, const Schedule& sc, int elt)
 {
-    for (int i = 0; i < alcs::kNumChunkings; ++i)
-        if (w->sched[i].seg_ptr && w->sched[i].kc == kc) return i;
-    return -1;
+    StageLayout L;
+    L.off_rec = sc.kc * 32 * v.p * elt;                              // X tile first
+    L.off_rowoff = L.off_rec + sc.wcap * alcs::record_bytes(v.g);
+    L.stage_bytes = L.off_rowoff + ((sc.rpg + 1) * 4 + 15) / 16 * 16;
+    return L;
 }
 
-using alcs::Plan;
+size_t plan_smem(const StageLayout& L, int stages) { return 16 * alcs::kMaxStages + (size_t)stages * L.stage_bytes; }
 
-size_t plan_smem(const KernelVariant& v, int kc, int nch, int stages, int elt)
+// The schedule for (kc, n_rg): sizes only (with_records = false) or complete.  Cached in w.
+Schedule* get_schedule(const alcs_packed* w, int kc, int n_rg, bool with_records)
 {
-    return (size_t)std::min(stages, nch) * kc * 32 * v.p * elt;
+    if (kc <= 0 || kc > w->cin) kc = w->cin;
+    std::lock_guard<std::mutex> lk(w->mu);
+    Schedule& sc = w->sched[std::make_pair(kc, n_rg)];
+    try {
+        if (sc.n_rg == 0 || (with_records && !sc.uploaded && sc.h_rec.empty() && sc.n_rec > 0))
+            alcs::build_schedule(*w, kc, n_rg, with_records, sc);
+    } catch (const std::bad_alloc&) {
+        return nullptr;
+    }
+    return &sc;
+}
+
+int upload_schedule(const alcs_packed* w, Schedule* sc, cudaStream_t st)
+{
+    std::lock_guard<std::mutex> lk(w->mu);
+    if (sc->uploaded) return ALCS_OK;
+    auto fail = [&](cudaError_t e) {
+        alcs::set_cuda_error_text(cudaGetErrorString(e));
+        cudaFree(sc->rec); cudaFree(sc->slice); cudaFree(sc->rowoff); cudaFree(sc->rowmap);
+        sc->rec = nullptr; sc->slice = sc->rowoff = sc->rowmap = nullptr;
+        (void)cudaGetLastError();
+        return e == cudaErrorMemoryAllocation ? ALCS_ERR_ALLOC : ALCS_ERR_CUDA;
+    };
+    cudaError_t e;
+    if ((e = cudaMalloc(&sc->rec, sc->h_rec.size() + 64)) != cudaSuccess) return fail(e);
+    if ((e = cudaMalloc(&sc->slice, sc->h_slice.size() * 4)) != cudaSuccess) return fail(e);
+    if ((e = cudaMalloc(&sc->rowoff, sc->h_rowoff.size() * 4)) != cudaSuccess) return fail(e);
+    if ((e = cudaMalloc(&sc->rowmap, sc->h_rowmap.size() * 4)) != cudaSuccess) return fail(e);
+    // the sources are pageable host vectors: these copies return once the data has been staged
+    if (!sc->h_rec.empty() &&
+        (e = cudaMemcpyAsync(sc->rec, sc->h_rec.data(), sc->h_rec.size(), cudaMemcpyHostToDevice, st)) != cudaSuccess)
+        return fail(e);
+    if ((e = cudaMemcpyAsync(sc->slice, sc->h_slice.data(), sc->h_slice.size() * 4, cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail(e);
+    if ((e = cudaMemcpyAsync(sc->rowoff, sc->h_rowoff.data(), sc->h_rowoff.size() * 4, cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail(e);
+    if ((e = cudaMemcpyAsync(sc->rowmap, sc->h_rowmap.data(), sc->h_rowmap.size() * 4, cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail(e);
+    if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return fail(e);
+    sc->uploaded = true;
+    std::vector<unsigned char>().swap(sc->h_rec);
+    std::vector<int>().swap(sc->h_rowoff);
+    return ALCS_OK;
+}
+
+void free_schedule_device(Schedule& sc)
+{
+    cudaFree(sc.rec); cudaFree(sc.slice); cudaFree(sc.rowoff); cudaFree(sc.rowmap);
+    sc.rec = nullptr; sc.slice = sc.rowoff = sc.rowmap = nullptr;
+    sc.uploaded = false;
 }
 
 // A rough per-layer time model (seconds) used to rank launch configurations.  Three resources
-// are modelled per SM: FMA issue slots, shared-memory/L1 wavefronts and bytes from L2; plus the
-// HBM floor and the quantisation of thread blocks into waves.
-double model_cost(const alcs_packed* w, const KernelVariant& v, const alcs::DeviceSchedule& sc,
-                  int stages, int n_rg, int rows_per_rg, long long q, int sms, int occ)
+// are modelled per SM: FMA issue slots, shared-memory wavefronts and bytes arriving from L2;
+// plus the HBM floor and the quantisation of work items over the persistent thread blocks.
+double model_cost(const alcs_packed* w, const KernelVariant& v, const Schedule& sc, long long q,
+                  int sms, int occ)
 {
     const int elt = (int)w->elt();
     const int T = 32 * v.p;
     const long long n_tiles = (q + T - 1) / T;
-    const long long ctas = n_tiles * n_rg;
+    const long long items = n_tiles * sc.n_rg;
     const long long slots = (long long)sms * occ;
-    const long long waves = (ctas + slots - 1) / slots;
+    const long long rounds = (items + slots - 1) / slots;
     const int vg = (v.p * elt >= 16) ? 16 / elt : v.p;
     const int ng = v.p / vg;
-    const double blocks_cta = (double)sc.nbp * rows_per_rg / std::max(1, w->rows);
-    const double seg_cta = (double)rows_per_rg * sc.nch;
-    const double fma_issue = blocks_cta * (v.g * v.p + ng + 2.5 + (elt == 2 ? v.p / 2 : 0)) / 4.0 + seg_cta * 12.0 / 4.0;
-    const double lsu = blocks_cta * (ng * (vg * elt * 32 / 128.0) + 1.5) + (double)sc.nch * sc.kc * T * elt / 128.0;
-    const double l2_bytes_cta = (double)std::min(w->cin, sc.nch * sc.kc) * T * elt;
-    const double l2 = l2_bytes_cta / 48.0;   // ~48 B/clk/SM sustained from L2
-    // latency hiding: with few resident warps the pipes are not kept busy
+    const double pairs_item = (double)sc.n_rec / sc.n_rg;
+    const double seg_item = (double)sc.rpg * sc.nch;
+    const double fma_issue = pairs_item * (2.0 * v.g * v.p + 2 * ng + 6 + (elt == 2 ? v.p : 0)) / 4.0 + seg_item * 14.0 / 4.0;
+    const double lsu = pairs_item * (2.0 * ng * (vg * elt * 32 / 128.0) + 1 + v.g / 2.0) +
+                       (double)sc.nch * sc.kc * T * elt / 128.0;
+    const double l2 = ((double)w->cin * T * elt + pairs_item * alcs::record_bytes(v.g)) / 48.0;
     const double warps = (double)v.nw * occ;
-    const double hide = std::min(1.0, 0.45 + warps / 28.0);
-    const double cta_cycles = std::max(std::max(fma_issue, lsu), l2) / hide + 2500.0 / occ;
-    const double clock = 1.9e9;
-    const double t_sm = (double)waves * occ * cta_cycles / clock;
+    const double hide = std::min(1.0, 0.5 + warps / 30.0);
+    const double item_cycles = std::max(std::max(fma_issue, lsu), l2) / hide + 1500.0;
+    const double t_sm = (double)rounds * occ * item_cycles / 1.9e9;
     const double bytes = (double)q * (w->cin + w->cout) * elt;
-    const double t_hbm = bytes / 6.0e12;
-    return std::max(t_sm, t_hbm);
+    return std::max(t_sm, bytes / 6.0e12);
 }
 
 int occupancy_of(const VariantInfo& vi, size_t smem)
 {
     int occ = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, vi.v.fn, vi.v.nw * 32, smem) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, vi.v.fn, (vi.v.nw + 1) * 32, smem) != cudaSuccess) {
         (void)cudaGetLastError();
         return 0;
     }
@@ -154,6 +207,7 @@ int enumerate_plans(const alcs_packed* w, long long q, std::vector<Plan>& out)
         init_variants_locked();
     }
     const int elt = (int)w->elt();
+    const int smem_max = std::min(kMaxSmem, di.smem_optin);
     out.clear();
     for (size_t vi = 0; vi < g_variants.size(); ++vi) {
         const KernelVariant& v = g_variants[vi].v;
@@ -162,25 +216,32 @@ int enumerate_plans(const alcs_packed* w, long long q, std::vector<Plan>& out)
         if (rc) return rc;
         const int cap = v.nw * v.rw;
         const int rg_min = (w->rows + cap - 1) / cap;
-        for (int si = 0; si < alcs::kNumChunkings; ++si) {
-            const alcs::DeviceSchedule& sc = w->sched[si];
-            if (!sc.seg_ptr) continue;
-            for (int stages = 2; stages <= 4; ++stages) {
-                if (stages > 2 && sc.nch < stages) continue;
-                const size_t smem = plan_smem(v, sc.kc, sc.nch, stages, elt);
-                if (smem > (size_t)std::min(kMaxSmem, di.smem_optin)) continue;
-                const int occ = occupancy_of(g_variants[vi], smem);
-                if (occ < 1) continue;
-                int last_rpg = -1;
-                for (int n_rg = rg_min; n_rg <= std::min(w->rows, rg_min * 4 + 2); ++n_rg) {
-                    const int rpg = (w->rows + n_rg - 1) / n_rg;
-                    if (rpg == last_rpg) continue;
-                    last_rpg = rpg;
-                    const int n_rg_eff = (w->rows + rpg - 1) / rpg;
+        int last_kc = -1;
+        for (int ci = 0; ci < alcs::kNumChunkings; ++ci) {
+            int kc = alcs::kChunkings[ci];
+            if (kc == 0 || kc > w->cin) kc = w->cin;
+            if (kc == last_kc) continue;
+            last_kc = kc;
+            if ((size_t)kc * 32 * v.p * elt * 2 > (size_t)smem_max) continue;
+            int last_rpg = -1;
+            for (int n_rg = rg_min; n_rg <= std::min(w->rows, rg_min * 4 + 2); ++n_rg) {
+                const int rpg = (w->rows + n_rg - 1) / n_rg;
+                if (rpg == last_rpg || rpg > cap) continue;
+                last_rpg = rpg;
+                const Schedule* sc = get_schedule(w, kc, n_rg, false);
+                if (!sc) return ALCS_ERR_ALLOC;
+                const StageLayout L = stage_layout(v, *sc, elt);
+                for (int stages = 2; stages <= alcs::kMaxStages; ++stages) {
+                    const size_t smem = plan_smem(L, stages);
+                    if (smem > (size_t)smem_max) break;
+                    const int occ = occupancy_of(g_variants[vi], smem);
+                    if (occ < 1) continue;
                     Plan p;
-                    p.variant = (int)vi; p.sched = si; p.stages = stages;
-                    p.n_rg = n_rg_eff; p.rows_per_rg = rpg; p.smem = smem;
-                    p.cost = model_cost(w, v, sc, stages, n_rg_eff, rpg, q, di.sms, occ);
+                    p.variant = (int)vi; p.kc = sc->kc; p.n_rg = sc->n_rg; p.stages = stages;
+                    p.occ = occ; p.smem = smem;
+                    p.cost = model_cost(w, v, *sc, q, di.sms, occ);
+                    // deeper rings only help while there are chunks to prefetch; prefer the shallowest
+                    p.cost *= 1.0 + 0.01 * stages;
                     out.push_back(p);
                 }
             }
@@ -190,13 +251,13 @@ int enumerate_plans(const alcs_packed* w, long long q, std::vector<Plan>& out)
     return out.empty() ? ALCS_ERR_UNSUPPORTED : ALCS_OK;
 }
 
-void plan_to_cfg(const alcs_packed* w, const Plan& p, alcs_launch_cfg* c)
+void plan_to_cfg(const Plan& p, alcs_launch_cfg* c)
 {
     const KernelVariant& v = g_variants[p.variant].v;
     c->pixels_per_lane = v.p;
     c->rows_per_warp = v.rw;
     c->warps = v.nw;
-    c->chunk_channels = w->sched[p.sched].kc;
+    c->chunk_channels = p.kc;
     c->stages = p.stages;
     c->row_groups = p.n_rg;
     c->min_blocks = v.minb;
@@ -209,33 +270,36 @@ int cfg_to_plan(const alcs_packed* w, long long q, const alcs_launch_cfg* c, Pla
     int rc = enumerate_plans(w, q, all);
     if (rc) return rc;
     if (!c) { *out = all[0]; return ALCS_OK; }
-    for (const Plan& p : all) {
+    auto variant_ok = [&](const Plan& p) {
         const KernelVariant& v = g_variants[p.variant].v;
-        if (c->pixels_per_lane && c->pixels_per_lane != v.p) continue;
-        if (c->rows_per_warp && c->rows_per_warp != v.rw) continue;
-        if (c->warps && c->warps != v.nw) continue;
-        if (c->min_blocks && c->min_blocks != v.minb) continue;
-        if (c->chunk_channels && c->chunk_channels != w->sched[p.sched].kc) continue;
-        if (c->stages && c->stages != p.stages) continue;
-        if (c->row_groups && c->row_groups != p.n_rg) continue;
-        *out = p;
-        return ALCS_OK;
-    }
-    // row_groups outside the enumerated range: accept any feasible count for a matching variant
-    if (c->row_groups > 0) {
+        if (c->pixels_per_lane && c->pixels_per_lane != v.p) return false;
+        if (c->rows_per_warp && c->rows_per_warp != v.rw) return false;
+        if (c->warps && c->warps != v.nw) return false;
+        if (c->min_blocks && c->min_blocks != v.minb) return false;
+        if (c->chunk_channels && std::min(c->chunk_channels, w->cin) != p.kc) return false;
+        if (c->stages && c->stages != p.stages) return false;
+        return true;
+    };
+    for (const Plan& p : all)
+        if (variant_ok(p) && (!c->row_groups || c->row_groups == p.n_rg)) { *out = p; return ALCS_OK; }
+    // a row-group count outside the enumerated range: accept it for a matching variant if it fits
+    if (c->row_groups > 0 && c->row_groups <= w->rows) {
+        DeviceInfo di;
+        rc = device_info(w->device, &di);
+        if (rc) return rc;
         for (const Plan& p0 : all) {
+            if (!variant_ok(p0)) continue;
             const KernelVariant& v = g_variants[p0.variant].v;
-            if (c->pixels_per_lane && c->pixels_per_lane != v.p) continue;
-            if (c->rows_per_warp && c->rows_per_warp != v.rw) continue;
-            if (c->warps && c->warps != v.nw) continue;
-            if (c->min_blocks && c->min_blocks != v.minb) continue;
-            if (c->chunk_channels && c->chunk_channels != w->sched[p0.sched].kc) continue;
-            if (c->stages && c->stages != p0.stages) continue;
             const int rpg = (w->rows + c->row_groups - 1) / c->row_groups;
             if (rpg > v.nw * v.rw) continue;
+            const Schedule* sc = get_schedule(w, p0.kc, c->row_groups, false);
+            if (!sc) return ALCS_ERR_ALLOC;
             Plan p = p0;
-            p.rows_per_rg = rpg;
-            p.n_rg = (w->rows + rpg - 1) / rpg;
+            p.n_rg = sc->n_rg;
+            p.smem = plan_smem(stage_layout(v, *sc, (int)w->elt()), p.stages);
+            if (p.smem > (size_t)std::min(kMaxSmem, di.smem_optin)) continue;
+            p.occ = occupancy_of(g_variants[p.variant], p.smem);
+            if (p.occ < 1) continue;
             *out = p;
             return ALCS_OK;
         }
@@ -269,30 +333,43 @@ int launch_plan(const alcs_packed* w, const Plan& p, const void* x, void* y, int
                 const float* bias, unsigned flags, cudaStream_t st)
 {
     const KernelVariant& v = g_variants[p.variant].v;
-    const alcs::DeviceSchedule& sc = w->sched[p.sched];
+    Schedule* sc = get_schedule(w, p.kc, p.n_rg, true);
+    if (!sc) return ALCS_ERR_ALLOC;
+    if (!sc->uploaded) {
+        const int rc = upload_schedule(w, sc, st);
+        if (rc) return rc;
+    }
+    DeviceInfo di;
+    int rc = device_info(w->device, &di);
+    if (rc) return rc;
     const int elt = (int)w->elt();
     const int hw = h * wd;
     ConvArgs a;
     a.x = x; a.y = y; a.bias = bias;
-    a.seg_ptr = sc.seg_ptr; a.cols = sc.cols; a.vals = sc.vals; a.row_order = w->d_row_order;
+    a.rec = sc->rec; a.slice = sc->slice; a.rowoff = sc->rowoff; a.rowmap = sc->rowmap;
+    a.err = w->d_err;
     a.rows = w->rows; a.cin = w->cin; a.cout = w->cout; a.hw = hw;
     a.q_total = n * hw;
-    a.n_rg = p.n_rg; a.rows_per_rg = p.rows_per_rg;
-    a.kc = sc.kc; a.nch = sc.nch; a.stages = p.stages;
+    const int T = 32 * v.p;
+    a.n_tiles = (a.q_total + T - 1) / T;
+    a.n_rg = sc->n_rg; a.rpg = sc->rpg;
+    a.kc = sc->kc; a.nch = sc->nch; a.stages = p.stages;
     a.relu = (flags & ALCS_RELU) ? 1 : 0;
     a.y_f32 = (flags & ALCS_Y_F32) ? 1 : 0;
+    const StageLayout L = stage_layout(v, *sc, elt);
+    a.off_rec = L.off_rec; a.off_rowoff = L.off_rowoff; a.stage_bytes = L.stage_bytes;
     // widest staging copy that every (image, channel) row start and length allows
     int ld = 16;
     while (ld > elt && (((size_t)hw * elt) % ld || (uintptr_t)x % ld)) ld >>= 1;
     a.ld_bytes = ld;
     const int vg = (v.p * elt >= 16) ? 16 / elt : v.p;
     a.st_vec = (hw % vg == 0 && (uintptr_t)y % 16 == 0) ? 1 : 0;
-    const int T = 32 * v.p;
-    const long long n_tiles = ((long long)a.q_total + T - 1) / T;
-    const long long grid = n_tiles * p.n_rg;
-    if (grid > 0x7fffffffll) return ALCS_ERR_SHAPE;
+    const long long items = (long long)a.n_tiles * a.n_rg;
+    if (items > 0x7fffffffll) return ALCS_ERR_SHAPE;
+    // persistent thread blocks: as many as can be resident, each walks items with that stride
+    const long long grid = std::min<long long>(items, (long long)di.sms * std::max(1, p.occ));
     void* args[] = {&a};
-    ALCS_CUDA(cudaLaunchKernel(v.fn, dim3((unsigned)grid), dim3(v.nw * 32), args, p.smem, st));
+    ALCS_CUDA(cudaLaunchKernel(v.fn, dim3((unsigned)grid), dim3((v.nw + 1) * 32), args, p.smem, st));
     return ALCS_OK;
 }
 
@@ -348,61 +425,29 @@ ALCS_API int alcs_packed_upload(alcs_packed* p, int device, void* cuda_stream)
     ALCS_CUDA(cudaGetDevice(&prev));
     ALCS_CUDA(cudaSetDevice(device));
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    int rc = ALCS_OK;
-    std::vector<alcs::HostSchedule> hs(alcs::kNumChunkings);
-    std::vector<int> order;
-    auto fail = [&](int code) {
-        for (auto& s : p->sched) {
-            cudaFree(s.seg_ptr); cudaFree(s.cols); cudaFree(s.vals);
-            s = alcs::DeviceSchedule();
-        }
-        cudaFree(p->d_row_order);
-        p->d_row_order = nullptr;
+    cudaError_t e = cudaMalloc(&p->d_err, 256);
+    if (e == cudaSuccess) e = cudaMemsetAsync(p->d_err, 0, 256, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) {
+        alcs::set_cuda_error_text(cudaGetErrorString(e));
+        cudaFree(p->d_err);
+        p->d_err = nullptr;
         (void)cudaGetLastError();
         cudaSetDevice(prev);
-        return code;
-    };
-    try {
-        alcs::build_row_order(*p, order);
-        for (int i = 0; i < alcs::kNumChunkings; ++i) {
-            int kc = alcs::kChunkings[i];
-            if (kc == 0 || kc > p->cin) kc = p->cin;
-            bool dup = false;
-            for (int j = 0; j < i; ++j) dup |= (hs[j].kc == kc);
-            if (dup) { hs[i].kc = -1; continue; }
-            alcs::build_schedule(*p, kc, hs[i]);
-        }
-    } catch (const std::bad_alloc&) {
-        return fail(ALCS_ERR_ALLOC);
+        return e == cudaErrorMemoryAllocation ? ALCS_ERR_ALLOC : ALCS_ERR_CUDA;
     }
-#define UP_CUDA(call)                                              \
-    do {                                                           \
-        cudaError_t e_ = (call);                                   \
-        if (e_ != cudaSuccess) {                                   \
-            alcs::set_cuda_error_text(cudaGetErrorString(e_));     \
-            return fail(e_ == cudaErrorMemoryAllocation ? ALCS_ERR_ALLOC : ALCS_ERR_CUDA); \
-        }                                                          \
-    } while (0)
-    UP_CUDA(cudaMalloc(&p->d_row_order, std::max<size_t>(4, order.size() * 4)));
-    UP_CUDA(cudaMemcpyAsync(p->d_row_order, order.data(), order.size() * 4, cudaMemcpyHostToDevice, st));
-    for (int i = 0; i < alcs::kNumChunkings; ++i) {
-        if (hs[i].kc < 0) continue;
-        alcs::DeviceSchedule& d = p->sched[i];
-        d.kc = hs[i].kc; d.nch = hs[i].nch; d.nbp = hs[i].nbp;
-        UP_CUDA(cudaMalloc(&d.seg_ptr, hs[i].seg_ptr.size() * 4));
-        UP_CUDA(cudaMalloc(&d.cols, std::max<size_t>(16, hs[i].cols.size() * 4)));
-        UP_CUDA(cudaMalloc(&d.vals, std::max<size_t>(16, hs[i].vals.size() * 4)));
-        UP_CUDA(cudaMemcpyAsync(d.seg_ptr, hs[i].seg_ptr.data(), hs[i].seg_ptr.size() * 4, cudaMemcpyHostToDevice, st));
-        if (!hs[i].cols.empty()) {
-            UP_CUDA(cudaMemcpyAsync(d.cols, hs[i].cols.data(), hs[i].cols.size() * 4, cudaMemcpyHostToDevice, st));
-            UP_CUDA(cudaMemcpyAsync(d.vals, hs[i].vals.data(), hs[i].vals.size() * 4, cudaMemcpyHostToDevice, st));
-        }
-    }
-    UP_CUDA(cudaStreamSynchronize(st));
-#undef UP_CUDA
     p->device = device;
     cudaSetDevice(prev);
-    return rc;
+    return ALCS_OK;
+}
+
+ALCS_API int alcs_packed_status(const alcs_packed* p, int* code)
+{
+    if (!p || !code) return ALCS_ERR_INVALID_ARG;
+    *code = 0;
+    if (p->device < 0) return ALCS_ERR_STATE;
+    ALCS_CUDA(cudaMemcpy(code, p->d_err, sizeof(int), cudaMemcpyDeviceToHost));
+    return ALCS_OK;
 }
 
 ALCS_API void alcs_packed_free(alcs_packed* p)
@@ -411,8 +456,8 @@ ALCS_API void alcs_packed_free(alcs_packed* p)
     if (p->device >= 0) {
         int prev = -1;
         if (cudaGetDevice(&prev) == cudaSuccess && cudaSetDevice(p->device) == cudaSuccess) {
-            for (auto& s : p->sched) { cudaFree(s.seg_ptr); cudaFree(s.cols); cudaFree(s.vals); }
-            cudaFree(p->d_row_order);
+            for (auto& kv : p->sched) free_schedule_device(kv.second);
+            cudaFree(p->d_err);
             cudaSetDevice(prev);
         }
         (void)cudaGetLastError();
@@ -480,7 +525,7 @@ ALCS_API int alcs_spconv1x1_plan(const alcs_packed* w, int n, int h, int wd, uns
     Plan plan;
     const int rc = resolve_plan(w, n, h, wd, flags, std::max(1ll, q), nullptr, &plan);
     if (rc) return rc;
-    plan_to_cfg(w, plan, out);
+    plan_to_cfg(plan, out);
     return ALCS_OK;
 }
 
@@ -498,7 +543,7 @@ ALCS_API int alcs_spconv1x1_tune(alcs_packed* w, const void* x, void* y, int n, 
     std::vector<Plan> all;
     rc = enumerate_plans(w, q, all);
     if (rc) return rc;
-    const size_t max_try = 48;
+    const size_t max_try = 160;
     if (all.size() > max_try) all.resize(max_try);
     // a buffer larger than L2, rewritten before every timed launch so that each candidate is
     // timed with cold caches, as it will run inside a network
@@ -518,7 +563,7 @@ ALCS_API int alcs_spconv1x1_tune(alcs_packed* w, const void* x, void* y, int n, 
     }
     int best_i = -1;
     float best_ms = 1e30f;
-    const int reps = 3;
+    const int reps = 2;
     for (size_t i = 0; i < all.size(); ++i) {
         float tmin = 1e30f;
         bool ok = true;
@@ -539,11 +584,20 @@ ALCS_API int alcs_spconv1x1_tune(alcs_packed* w, const void* x, void* y, int n, 
     if (e != cudaSuccess) { alcs::set_cuda_error_text(cudaGetErrorString(e)); return ALCS_ERR_CUDA; }
     if (best_i < 0) return ALCS_ERR_CUDA;
     alcs_launch_cfg c;
-    plan_to_cfg(w, all[best_i], &c);
+    plan_to_cfg(all[best_i], &c);
     {
         std::lock_guard<std::mutex> lk(w->mu);
         w->tuned[alcs::ShapeKey{n, h, wd, flags}] = c;
         w->plan_cache[alcs::ShapeKey{n, h, wd, flags}] = all[best_i];
+    }
+    {   // release the device copies of the schedules that did not win
+        std::lock_guard<std::mutex> lk(w->mu);
+        for (auto& kv : w->sched)
+            if (kv.second.uploaded && !(kv.first.first == all[best_i].kc && kv.first.second == all[best_i].n_rg)) {
+                bool used = false;
+                for (auto& pc : w->plan_cache) used |= (pc.second.kc == kv.first.first && pc.second.n_rg == kv.first.second);
+                if (!used) { free_schedule_device(kv.second); kv.second.n_rg = 0; }
+            }
     }
     // leave y holding the result of the chosen configuration
     rc = launch_plan(w, all[best_i], x, y, n, h, wd, bias, flags, st);
@@ -603,6 +657,10 @@ ALCS_API int alcs_stack_create(const alcs_layer* layers, int n_layers, unsigned 
         int rc = check_conv_args(L.w, L.x, L.y, L.n, L.h, L.wd, L.flags, &it.q);
         if (!rc) rc = check_device(L.w);
         if (!rc && it.q > 0) rc = resolve_plan(L.w, L.n, L.h, L.wd, L.flags, it.q, nullptr, &it.plan);
+        if (!rc && it.q > 0) {   // the schedule must be resident before any launch is captured
+            Schedule* sc = get_schedule(L.w, it.plan.kc, it.plan.n_rg, true);
+            rc = sc ? upload_schedule(L.w, sc, nullptr) : ALCS_ERR_ALLOC;
+        }
         if (rc) { delete s; return rc; }
         s->items.push_back(it);
     }

@@ -14,38 +14,47 @@
 
 namespace alcs {
 
-// Chunk sizes (input channels per pipeline stage) for which a device schedule is prepared at
-// upload time.  0 stands for "the whole Cin in one chunk" (used when Cin is small).
-constexpr int kNumChunkings = 4;
-constexpr int kChunkings[kNumChunkings] = {32, 64, 128, 0};
+// Chunk sizes (input channels per pipeline stage) the planner considers.  0 stands for "the
+// whole Cin in one chunk" (used when Cin is small).
+constexpr int kNumChunkings = 5;
+constexpr int kChunkings[kNumChunkings] = {16, 32, 64, 128, 0};
 
-// Device-resident schedule for one chunk size KC.  Every (block row, chunk) segment of the
-// column list is padded to an even number of blocks so that the kernel can fetch column indices
-// two at a time with aligned 8-byte loads; a padding block repeats the previous column with
-// zero weights.
-struct DeviceSchedule {
-    int kc = 0;                // channels per chunk (>= 1)
-    int nch = 0;               // number of chunks = ceil(cin / kc)
-    int nbp = 0;               // padded number of blocks
-    int* seg_ptr = nullptr;    // device [R][nch+1], offsets into cols / vals
-    int* cols = nullptr;       // device [nbp], chunk-local column index
-    float* vals = nullptr;     // device [nbp][g], always fp32 (fp16 weights widened exactly)
-};
-
-struct HostSchedule {
-    int kc = 0, nch = 0, nbp = 0;
-    std::vector<int> seg_ptr, cols;
-    std::vector<float> vals;
+// Launch schedule for one (chunk size KC, number of row groups) pair.
+//
+// Block rows are sorted by descending kept-block count and dealt to the row groups in
+// serpentine order, so every row group gets the same number of rows (+-1) and nearly the same
+// number of blocks whatever the distribution of row lengths.  rowmap[rg][t] is the block row that
+// is local row t of row group rg (-1 = none).
+//
+// The kept blocks are stored as "pair records" ordered [row group][chunk][local row][pair]: two
+// chunk-local column indices followed by their two g-wide value vectors (fp32; fp16 weights are
+// widened exactly).  A local row with an odd number of blocks in a chunk gets a padding block
+// that repeats its last column with zero weights.  slice[rg*nch + k] is the first record of the
+// (row group, chunk) slice, so the producer warp copies one contiguous range per stage;
+// rowoff[rg][k][t] is where local row t starts inside that slice (rowoff[..][rpg] = its length).
+struct Schedule {
+    int kc = 0, nch = 0, n_rg = 0, rpg = 0;
+    int wcap = 0;                  // longest slice, in records
+    int n_rec = 0;                 // total records
+    // host copies (kept until uploaded)
+    std::vector<unsigned char> h_rec;
+    std::vector<int> h_slice, h_rowoff, h_rowmap;
+    // device copies (valid once uploaded)
+    unsigned char* rec = nullptr;
+    int* slice = nullptr;
+    int* rowoff = nullptr;
+    int* rowmap = nullptr;
+    bool uploaded = false;
 };
 
 // A resolved launch configuration: which compiled kernel variant, which schedule, how many
-// pipeline stages and row groups.
+// pipeline stages.
 struct Plan {
     int variant = -1;      // index into the table of compiled kernel variants
-    int sched = -1;        // index into alcs_packed::sched
+    int kc = 0;            // schedule key: channels per chunk ...
+    int n_rg = 0;          // ... and number of row groups
     int stages = 0;
-    int n_rg = 0;
-    int rows_per_rg = 0;
+    int occ = 1;           // resident thread blocks per SM
     size_t smem = 0;
     double cost = 0;       // model estimate, seconds
 };
@@ -68,11 +77,11 @@ struct alcs_packed {
     std::vector<uint8_t> vals;        // [nb*g] elements of dt, raw bytes
     // device side (valid once uploaded)
     int device = -1;
-    int* d_row_order = nullptr;       // [rows] block rows by descending kept-block count
-    alcs::DeviceSchedule sched[alcs::kNumChunkings];
+    int* d_err = nullptr;             // device error word written by a kernel whose bounded wait ran out
+    mutable std::map<std::pair<int, int>, alcs::Schedule> sched;   // by (kc, n_rg), built on demand
     std::map<alcs::ShapeKey, alcs_launch_cfg> tuned;   // filled by alcs_spconv1x1_tune
     mutable std::map<alcs::ShapeKey, alcs::Plan> plan_cache;   // resolved plans, by shape
-    mutable std::mutex mu;                                      // guards plan_cache
+    mutable std::mutex mu;                                      // guards plan_cache and sched
     size_t elt() const { return dt == ALCS_F32 ? 4 : 2; }
 };
 
@@ -80,8 +89,7 @@ namespace alcs {
 
 // Host-side helpers implemented in alcs_pack.cpp (no CUDA).
 float half_bits_to_float(uint16_t h);
-void build_row_order(const alcs_packed& p, std::vector<int>& order);
-void build_schedule(const alcs_packed& p, int kc, HostSchedule& out);
+void build_schedule(const alcs_packed& p, int kc, int n_rg, bool with_records, Schedule& out);
 
 }  // namespace alcs
 

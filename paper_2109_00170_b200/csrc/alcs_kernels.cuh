@@ -4,17 +4,26 @@
 // the loop this re-creates: zero the accumulators, loop over a group's kept columns, multiply the
 // column's g weights with the input vector addressed by the column offset, accumulate):
 //
-//   thread block = one tile of T = 32*P consecutive pixels (pixels of all images flattened,
-//                  q = n*HW + p) x one slice of block rows ("row group")
-//   warp         = RW block rows at a time, all T pixels of the tile
+//   work item    = one tile of T = 32*P consecutive pixels (pixels of all images flattened,
+//                  q = n*HW + p) x one "row group" (a balanced subset of the block rows)
+//   thread block = persistent: walks items blockIdx.x, blockIdx.x + gridDim.x, ...
+//   consumer warp= RW block rows at a time, all T pixels of the tile
 //   lane         = P pixels of each of those rows: G*P fp32 accumulators per row in registers
+//   producer warp= one extra warp that only moves data
 //
-// The input channels are walked in chunks of KC channels.  Each chunk of the X tile
-// ([KC][T] elements) is staged in shared memory by cp.async through a multi-stage ring, so the
-// copy of chunk k+stages-1 overlaps the arithmetic of chunk k.  Inside a chunk a warp walks the
-// (row, chunk) segment of the column list: column indices and weights are warp-uniform global
-// loads (one broadcast transaction each), X values are 128-bit conflict-free shared-memory
-// loads, and every X word feeds G FMAs.
+// The input channels are walked in chunks of KC channels.  For each (item, chunk) the producer
+// warp copies, with cp.async, the X tile ([KC][T] elements) and the row group's slice of the
+// packed weights for that chunk (one contiguous range of "pair records": two column indices and
+// their two g-wide value vectors) into one stage of a shared-memory ring that runs on across
+// items, so the loads of the next tile overlap the arithmetic and the stores of the current
+// one.  Stages are handed over through mbarriers: "full" is completed by the producer lanes'
+// cp.async completion, "empty" by one arrival per consumer warp, so consumer warps never wait
+// for each other, only for data.  In the hot loop everything is a shared-memory load: records
+// are warp-uniform broadcasts, X values are 128-bit conflict-free loads, and every X word feeds
+// G FMAs.
+//
+// Every mbarrier wait is bounded: after kWaitLimit polls the warp records an error code in
+// ConvArgs::err and leaves the kernel (the producer first waits for its own copies).
 #ifndef ALCS_KERNELS_CUH_
 #define ALCS_KERNELS_CUH_
 
@@ -26,24 +35,37 @@
 
 namespace alcs {
 
+constexpr int kMaxStages = 8;
+constexpr int kWaitLimit = 1 << 22;     // polls of mbarrier.try_wait before giving up
+constexpr int kErrFullWait = 1;         // a consumer gave up waiting for data
+constexpr int kErrEmptyWait = 2;        // the producer gave up waiting for a free stage
+
+// bytes of one pair record: header (2 column indices, padded to 16 bytes unless G == 1, where
+// the two values share the header's 16 bytes) followed by 2*G fp32 values
+__host__ __device__ constexpr int record_bytes(int g) { return g == 1 ? 16 : 16 + 8 * g; }
+
 struct ConvArgs {
     const void* x;            // [n][cin][hw] of XT
     void* y;                  // [n][cout][hw] of XT, or float if y_f32
     const float* bias;        // [cout] or nullptr
-    const int* seg_ptr;       // [rows][nch+1]
-    const int* cols;          // [nbp] chunk-local column
-    const float* vals;        // [nbp][G]
-    const int* row_order;     // [rows]
+    const unsigned char* rec; // pair records, ordered [row group][chunk][local row][pair]
+    const int* slice;         // [n_rg*nch + 1] first record of each (row group, chunk) slice
+    const int* rowoff;        // [n_rg][nch][rpg+1] record offsets of the local rows inside a slice
+    const int* rowmap;        // [n_rg][rpg] block row of each local row, -1 = none
+    int* err;                 // device error word (0 = ok)
     int rows, cin, cout, hw;
     int q_total;              // n * hw
-    int n_rg, rows_per_rg;    // row groups per pixel tile, block rows per row group
+    int n_tiles, n_rg, rpg;   // pixel tiles, row groups, local rows per row group (padded)
     int kc, nch, stages;
     int relu;
     int y_f32;                // only meaningful for XT = __half
-    int ld_bytes;             // bytes per staging copy: 16, 8, 4 or 2
+    int ld_bytes;             // bytes per X staging copy: 16, 8, 4 or 2
     int st_vec;               // 1 if vector stores are allowed
+    // shared-memory layout (bytes): [mbarriers | stage 0 | stage 1 | ...]
+    int off_rec, off_rowoff, stage_bytes;
 };
 
+// ---- small PTX wrappers ------------------------------------------------------------------------
 __device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src)
 {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dst), "l"(src) : "memory");
@@ -56,14 +78,37 @@ __device__ __forceinline__ void cp_async_4(uint32_t dst, const void* src)
 {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" ::"r"(dst), "l"(src) : "memory");
 }
-__device__ __forceinline__ void cp_async_commit()
+__device__ __forceinline__ void cp_async_wait_all()
 {
-    asm volatile("cp.async.commit_group;\n" ::: "memory");
+    asm volatile("cp.async.wait_all;\n" ::: "memory");
 }
-template <int N>
-__device__ __forceinline__ void cp_async_wait()
+__device__ __forceinline__ void mbar_init(uint32_t bar, int count)
 {
-    asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("{\n .reg .b64 t;\n mbarrier.arrive.shared::cta.b64 t, [%0];\n}\n" ::"r"(bar) : "memory");
+}
+// Arrive on `bar` once all cp.async copies this thread has issued so far have landed.
+__device__ __forceinline__ void mbar_arrive_on_copies(uint32_t bar)
+{
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];\n" ::"r"(bar) : "memory");
+}
+// Bounded wait for the phase with the given parity to complete.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+{
+    for (int it = 0; it < kWaitLimit; ++it) {
+        uint32_t done;
+        asm volatile(
+            "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+            " selp.u32 %0, 1, 0, p;\n}\n"
+            : "=r"(done)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (done) return true;
+    }
+    return false;
 }
 
 // Load VG consecutive X elements from shared memory and widen them to fp32.
@@ -106,32 +151,35 @@ struct XVec<__half, 4> {
     }
 };
 
-// Weights of two consecutive blocks (2*G floats, 8- or 16-byte aligned), warp-uniform address.
+// One pair record from shared memory (same address in every lane: broadcasts).
 template <int G>
-__device__ __forceinline__ void load_w2(const float* __restrict__ p, float (&w0)[G], float (&w1)[G])
+__device__ __forceinline__ void load_record(const unsigned char* p, int& c0, int& c1, float (&w0)[G],
+                                            float (&w1)[G])
 {
+    const int4 h = *reinterpret_cast<const int4*>(p);
+    c0 = h.x;
+    c1 = h.y;
     if constexpr (G == 1) {
-        const float2 v = __ldg(reinterpret_cast<const float2*>(p));
-        w0[0] = v.x;
-        w1[0] = v.y;
+        w0[0] = __int_as_float(h.z);
+        w1[0] = __int_as_float(h.w);
     } else if constexpr (G == 2) {
-        const float4 v = __ldg(reinterpret_cast<const float4*>(p));
+        const float4 v = *reinterpret_cast<const float4*>(p + 16);
         w0[0] = v.x; w0[1] = v.y; w1[0] = v.z; w1[1] = v.w;
     } else {
 #pragma unroll
         for (int i = 0; i < G / 4; ++i) {
-            const float4 v = __ldg(reinterpret_cast<const float4*>(p) + i);
+            const float4 v = *reinterpret_cast<const float4*>(p + 16 + 16 * i);
             w0[4 * i] = v.x; w0[4 * i + 1] = v.y; w0[4 * i + 2] = v.z; w0[4 * i + 3] = v.w;
         }
 #pragma unroll
         for (int i = 0; i < G / 4; ++i) {
-            const float4 v = __ldg(reinterpret_cast<const float4*>(p) + G / 4 + i);
+            const float4 v = *reinterpret_cast<const float4*>(p + 16 + 4 * G + 16 * i);
             w1[4 * i] = v.x; w1[4 * i + 1] = v.y; w1[4 * i + 2] = v.z; w1[4 * i + 3] = v.w;
         }
     }
 }
 
-template <typename XT, typename YT, int VG>
+template <typename YT, int VG>
 __device__ __forceinline__ void store_vec(YT* p, const float (&v)[VG])
 {
     if constexpr (sizeof(YT) == 4) {
@@ -158,191 +206,253 @@ __device__ __forceinline__ void store_one(YT* p, float v)
         *p = __float2half_rn(v);
 }
 
+// ---- producer: one warp copies (item, chunk) after (item, chunk) into the ring ---------------
+// LDB = bytes per X copy.  Each lane owns NCOL fixed pixel vectors of the tile and walks the
+// channels of the chunk, so its source pointers are computed once per item.
+template <typename XT, int G, int P, int LDB>
+__device__ __forceinline__ void produce(const ConvArgs& a, unsigned char* smem, int lane)
+{
+    constexpr int T = 32 * P;
+    constexpr int SZ = (int)sizeof(XT);
+    constexpr int ROWB = T * SZ;
+    constexpr int EV = LDB / SZ;            // elements per copy
+    constexpr int VPR = T / EV;             // copies per channel row
+    constexpr int NCOL = VPR >= 32 ? VPR / 32 : 1;   // copies per channel row per lane
+    constexpr int RP = VPR >= 32 ? 1 : 32 / VPR;     // channel rows the warp covers per pass
+    constexpr int REC = record_bytes(G);
+    const int vlane = lane % VPR;           // (== lane when VPR >= 32)
+    const int rlane = lane / VPR;           // first channel row of this lane (0 when VPR >= 32)
+
+    const size_t ch_bytes = (size_t)a.hw * SZ;
+    const uint32_t smem_u32 = (uint32_t)__cvta_generic_to_shared(smem);
+    const uint32_t ring = smem_u32 + 16 * kMaxStages;
+    const int S = a.stages;
+    const int items = a.n_tiles * a.n_rg;
+    int kk = 0;                             // running (item, chunk) counter = ring position
+
+    for (int item = blockIdx.x; item < items; item += gridDim.x) {
+        const int tile = item / a.n_rg;
+        const int rg = item - tile * a.n_rg;
+        const int q0 = tile * T;
+        const unsigned char* src[NCOL];
+        bool ok[NCOL];
+#pragma unroll
+        for (int i = 0; i < NCOL; ++i) {
+            const int q = q0 + (vlane + 32 * i) * EV;
+            ok[i] = q < a.q_total;
+            const int n = ok[i] ? q / a.hw : 0;
+            const int p = ok[i] ? q - n * a.hw : 0;
+            src[i] = static_cast<const unsigned char*>(a.x) + ((size_t)n * a.cin * a.hw + p) * SZ;
+        }
+        const int* slice = a.slice + rg * a.nch;
+        const int* rowoff = a.rowoff + (size_t)rg * a.nch * (a.rpg + 1);
+
+        for (int k = 0; k < a.nch; ++k, ++kk) {
+            const int s = kk % S;
+            if (kk >= S) {                  // wait until the consumers have released this stage
+                if (!mbar_wait(smem_u32 + 8 * kMaxStages + 8 * s, ((kk / S) - 1) & 1)) {
+                    if (lane == 0) atomicExch(a.err, kErrEmptyWait);
+                    cp_async_wait_all();
+                    return;
+                }
+            }
+            const uint32_t st = ring + s * a.stage_bytes;
+            // X tile of this chunk
+            const int cbase = k * a.kc;
+            const int nrows = min(a.kc, a.cin - cbase);
+#pragma unroll
+            for (int i = 0; i < NCOL; ++i) {
+                if (!ok[i]) continue;
+                const unsigned char* sp = src[i] + (size_t)cbase * ch_bytes;
+                const uint32_t dp = st + (vlane + 32 * i) * LDB;
+                if constexpr (LDB == 16) {
+                    for (int c = rlane; c < nrows; c += RP) cp_async_16(dp + c * ROWB, sp + c * ch_bytes);
+                } else if constexpr (LDB == 8) {
+                    for (int c = rlane; c < nrows; c += RP) cp_async_8(dp + c * ROWB, sp + c * ch_bytes);
+                } else if constexpr (LDB == 4) {
+                    for (int c = rlane; c < nrows; c += RP) cp_async_4(dp + c * ROWB, sp + c * ch_bytes);
+                } else {   // 2-byte elements at odd alignment: plain loads and shared-memory stores
+                    unsigned char* d = smem + 16 * kMaxStages + s * a.stage_bytes + (vlane + 32 * i) * LDB;
+                    for (int c = rlane; c < nrows; c += RP)
+                        *reinterpret_cast<unsigned short*>(d + c * ROWB) =
+                            __ldg(reinterpret_cast<const unsigned short*>(sp + c * ch_bytes));
+                }
+            }
+            // the row group's pair records of this chunk and their per-row offsets
+            const int r0 = __ldg(slice + k);
+            const int n16 = (__ldg(slice + k + 1) - r0) * (REC / 16);
+            const unsigned char* rsrc = a.rec + (size_t)r0 * REC;
+            for (int i = lane; i < n16; i += 32) cp_async_16(st + a.off_rec + i * 16, rsrc + (size_t)i * 16);
+            const int* osrc = rowoff + (size_t)k * (a.rpg + 1);
+            for (int i = lane; i <= a.rpg; i += 32) cp_async_4(st + a.off_rowoff + i * 4, osrc + i);
+            if constexpr (LDB == 2) __threadfence_block();
+            mbar_arrive_on_copies(smem_u32 + 8 * s);      // "full" completes when all 32 lanes' copies land
+        }
+    }
+    cp_async_wait_all();
+}
+
 template <typename XT, int G, int P, int RW, int NW, int MINB>
-__global__ void __launch_bounds__(NW * 32, MINB) spconv1x1_kernel(const ConvArgs a)
+__global__ void __launch_bounds__((NW + 1) * 32, MINB) spconv1x1_kernel(const ConvArgs a)
 {
     constexpr int T = 32 * P;                         // pixels per tile
     constexpr int SZ = (int)sizeof(XT);
     constexpr int VG = (P * SZ >= 16) ? 16 / SZ : P;  // elements per shared-memory vector load
     constexpr int NG = P / VG;                        // vector groups per lane
-    constexpr int NT = NW * 32;
     constexpr int ROWB = T * SZ;                      // bytes of one staged channel row
+    constexpr int REC = record_bytes(G);
 
-    extern __shared__ __align__(16) unsigned char smem[];
+    extern __shared__ __align__(16) unsigned char smem[];   // [full[8] | empty[8] | ring]
 
     const int tid = threadIdx.x;
     const int lane = tid & 31;
     const int warp = tid >> 5;
-    const int tile = blockIdx.x / a.n_rg;
-    const int rg = blockIdx.x - tile * a.n_rg;
-    const int q0 = tile * T;
-    const int stage_bytes = a.kc * ROWB;
+    const int S = a.stages;
+    const uint32_t smem_u32 = (uint32_t)__cvta_generic_to_shared(smem);
 
-    // ---- block rows owned by this warp ------------------------------------------------------
-    int row[RW], pos[RW], endv[RW];
-    {
-        const int base = rg * a.rows_per_rg;
-        const int lim = min(a.rows, base + a.rows_per_rg);
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(smem_u32 + 8 * s, 32);                        // full: the 32 producer lanes
+            mbar_init(smem_u32 + 8 * kMaxStages + 8 * s, NW);       // empty: one arrival per consumer warp
+        }
+    }
+    __syncthreads();
+
+    if (warp == NW) {   // ---- producer warp -------------------------------------------------
+        switch (a.ld_bytes) {
+            case 16: produce<XT, G, P, 16>(a, smem, lane); break;
+            case 8: produce<XT, G, P, 8>(a, smem, lane); break;
+            case 4: produce<XT, G, P, 4>(a, smem, lane); break;
+            default:
+                if constexpr (SZ == 2) produce<XT, G, P, 2>(a, smem, lane);
+                break;
+        }
+        return;
+    }
+
+    // ---- consumer warps ---------------------------------------------------------------------
+    const unsigned char* ring = smem + 16 * kMaxStages;
+    const int items = a.n_tiles * a.n_rg;
+    int kk = 0;
+
+    for (int item = blockIdx.x; item < items; item += gridDim.x) {
+        const int tile = item / a.n_rg;
+        const int rg = item - tile * a.n_rg;
+        const int q0 = tile * T;
+
+        // local rows of this warp: tier s, dealt in serpentine order so that the warps' totals match
+        int lrow[RW], rowid[RW];
 #pragma unroll
         for (int s = 0; s < RW; ++s) {
-            const int ps = base + s * NW + warp;
-            row[s] = ps < lim ? __ldg(a.row_order + ps) : -1;
-            pos[s] = row[s] >= 0 ? __ldg(a.seg_ptr + (size_t)row[s] * (a.nch + 1)) : 0;
-            endv[s] = pos[s];
+            lrow[s] = s * NW + ((s & 1) ? NW - 1 - warp : warp);
+            rowid[s] = lrow[s] < a.rpg ? __ldg(a.rowmap + rg * a.rpg + lrow[s]) : -1;
         }
-    }
 
-    float acc[RW][G][P];
-#pragma unroll
-    for (int s = 0; s < RW; ++s)
-#pragma unroll
-        for (int j = 0; j < G; ++j)
-#pragma unroll
-            for (int e = 0; e < P; ++e) acc[s][j][e] = 0.0f;
-
-    // ---- staging set-up: this thread always copies the same pixel vector of every channel ---
-    const int ev = a.ld_bytes / SZ;                   // elements per staging copy
-    const int vpr = T / ev;                           // copies per channel row
-    const int sv = tid % vpr;
-    const int sc0 = tid / vpr;
-    const int scstep = NT / vpr;
-    const int sq = q0 + sv * ev;
-    const bool svalid = sq < a.q_total;
-    const unsigned char* ssrc = nullptr;
-    if (svalid) {
-        const int n = sq / a.hw;
-        const int p = sq - n * a.hw;
-        ssrc = static_cast<const unsigned char*>(a.x) + ((size_t)n * a.cin * a.hw + p) * SZ;
-    }
-    const size_t ch_bytes = (size_t)a.hw * SZ;
-    const uint32_t smem_u32 = (uint32_t)__cvta_generic_to_shared(smem);
-    const uint32_t sdst0 = smem_u32 + sv * a.ld_bytes;
-
-    auto stage_chunk = [&](int k) {
-        if (k < a.nch && svalid) {
-            const int cbase = k * a.kc;
-            const int nrows = min(a.kc, a.cin - cbase);
-            const uint32_t dst = sdst0 + (k % a.stages) * stage_bytes;
-            const unsigned char* src = ssrc + (size_t)cbase * ch_bytes;
-            if (a.ld_bytes == 16) {
-                for (int c = sc0; c < nrows; c += scstep) cp_async_16(dst + c * ROWB, src + c * ch_bytes);
-            } else if (a.ld_bytes == 8) {
-                for (int c = sc0; c < nrows; c += scstep) cp_async_8(dst + c * ROWB, src + c * ch_bytes);
-            } else if (a.ld_bytes == 4) {
-                for (int c = sc0; c < nrows; c += scstep) cp_async_4(dst + c * ROWB, src + c * ch_bytes);
-            } else {  // 2-byte elements at odd alignment: plain loads and shared-memory stores
-                unsigned char* d = smem + (k % a.stages) * stage_bytes + sv * a.ld_bytes;
-                for (int c = sc0; c < nrows; c += scstep)
-                    *reinterpret_cast<unsigned short*>(d + c * ROWB) =
-                        __ldg(reinterpret_cast<const unsigned short*>(src + c * ch_bytes));
-            }
-        }
-        cp_async_commit();
-    };
-
-    for (int k = 0; k < a.stages - 1; ++k) stage_chunk(k);
-
-    const unsigned char* xlane = smem + lane * (VG * SZ);
-
-    // ---- main loop over channel chunks ------------------------------------------------------
-    for (int k = 0; k < a.nch; ++k) {
+        float acc[RW][G][P];
 #pragma unroll
         for (int s = 0; s < RW; ++s)
-            if (row[s] >= 0) endv[s] = __ldg(a.seg_ptr + (size_t)row[s] * (a.nch + 1) + k + 1);
+#pragma unroll
+            for (int j = 0; j < G; ++j)
+#pragma unroll
+                for (int e = 0; e < P; ++e) acc[s][j][e] = 0.0f;
 
-        if (a.stages == 2) cp_async_wait<0>();
-        else if (a.stages == 3) cp_async_wait<1>();
-        else cp_async_wait<2>();
-        __syncthreads();          // chunk k visible to all; everyone is done with chunk k-1
-        stage_chunk(k + a.stages - 1);
-
-        const unsigned char* xs = xlane + (k % a.stages) * stage_bytes;
+        for (int k = 0; k < a.nch; ++k, ++kk) {
+            const int st = kk % S;
+            if (!mbar_wait(smem_u32 + 8 * st, (kk / S) & 1)) {      // chunk has landed in stage st
+                if (lane == 0) atomicExch(a.err, kErrFullWait);
+                return;
+            }
+            const unsigned char* stage = ring + st * a.stage_bytes;
+            const unsigned char* xs = stage + lane * (VG * SZ);
+            const unsigned char* recs = stage + a.off_rec;
+            const int* roff = reinterpret_cast<const int*>(stage + a.off_rowoff);
 #pragma unroll
-        for (int s = 0; s < RW; ++s) {
-            if (row[s] < 0) continue;
-            const int e = endv[s];
-#pragma unroll 2
-            for (int b = pos[s]; b < e; b += 2) {
-                const int2 cc = __ldg(reinterpret_cast<const int2*>(a.cols + b));
-                float w0[G], w1[G];
-                load_w2<G>(a.vals + (size_t)b * G, w0, w1);
-                const unsigned char* x0p = xs + cc.x * ROWB;
-                const unsigned char* x1p = xs + cc.y * ROWB;
+            for (int s = 0; s < RW; ++s) {
+                if (lrow[s] >= a.rpg) continue;
+                const unsigned char* rp = recs + roff[lrow[s]] * REC;
+                const unsigned char* re = recs + roff[lrow[s] + 1] * REC;
+                for (; rp < re; rp += REC) {
+                    int c0, c1;
+                    float w0[G], w1[G];
+                    load_record<G>(rp, c0, c1, w0, w1);
+                    const unsigned char* x0p = xs + c0 * ROWB;
+                    const unsigned char* x1p = xs + c1 * ROWB;
 #pragma unroll
-                for (int gi = 0; gi < NG; ++gi) {
-                    float xv[VG];
-                    XVec<XT, VG>::load(x0p + gi * (32 * VG * SZ), xv);
+                    for (int gi = 0; gi < NG; ++gi) {
+                        float xv[VG];
+                        XVec<XT, VG>::load(x0p + gi * (32 * VG * SZ), xv);
 #pragma unroll
-                    for (int j = 0; j < G; ++j)
+                        for (int j = 0; j < G; ++j)
 #pragma unroll
-                        for (int t = 0; t < VG; ++t)
-                            acc[s][j][gi * VG + t] = fmaf(w0[j], xv[t], acc[s][j][gi * VG + t]);
-                }
+                            for (int t = 0; t < VG; ++t)
+                                acc[s][j][gi * VG + t] = fmaf(w0[j], xv[t], acc[s][j][gi * VG + t]);
+                    }
 #pragma unroll
-                for (int gi = 0; gi < NG; ++gi) {
-                    float xv[VG];
-                    XVec<XT, VG>::load(x1p + gi * (32 * VG * SZ), xv);
+                    for (int gi = 0; gi < NG; ++gi) {
+                        float xv[VG];
+                        XVec<XT, VG>::load(x1p + gi * (32 * VG * SZ), xv);
 #pragma unroll
-                    for (int j = 0; j < G; ++j)
+                        for (int j = 0; j < G; ++j)
 #pragma unroll
-                        for (int t = 0; t < VG; ++t)
-                            acc[s][j][gi * VG + t] = fmaf(w1[j], xv[t], acc[s][j][gi * VG + t]);
+                            for (int t = 0; t < VG; ++t)
+                                acc[s][j][gi * VG + t] = fmaf(w1[j], xv[t], acc[s][j][gi * VG + t]);
+                    }
                 }
             }
-            pos[s] = e;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32 + 8 * kMaxStages + 8 * st);   // stage st may be refilled
         }
-    }
-    cp_async_wait<0>();
 
-    // ---- epilogue: bias, ReLU, store --------------------------------------------------------
-    auto epilogue = [&](auto* ybase) {
-        using YT = std::remove_pointer_t<decltype(ybase)>;
-        size_t yoff[NG];
-        bool yok[NG];
+        // ---- epilogue: bias, ReLU, store ----------------------------------------------------
+        auto epilogue = [&](auto* ybase) {
+            using YT = std::remove_pointer_t<decltype(ybase)>;
+            size_t yoff[NG];
+            bool yok[NG];
 #pragma unroll
-        for (int gi = 0; gi < NG; ++gi) {
-            const int q = q0 + gi * (32 * VG) + lane * VG;
-            yok[gi] = q < a.q_total;
-            const int n = q / a.hw;
-            yoff[gi] = (size_t)n * a.cout * a.hw + (q - n * a.hw);
-        }
+            for (int gi = 0; gi < NG; ++gi) {
+                const int q = q0 + gi * (32 * VG) + lane * VG;
+                yok[gi] = q < a.q_total;
+                const int n = q / a.hw;
+                yoff[gi] = (size_t)n * a.cout * a.hw + (q - n * a.hw);
+            }
 #pragma unroll
-        for (int s = 0; s < RW; ++s) {
-            if (row[s] < 0) continue;
+            for (int s = 0; s < RW; ++s) {
+                if (rowid[s] < 0) continue;
 #pragma unroll
-            for (int j = 0; j < G; ++j) {
-                const int co = row[s] * G + j;
-                if (co >= a.cout) continue;
-                const float bv = a.bias ? __ldg(a.bias + co) : 0.0f;
+                for (int j = 0; j < G; ++j) {
+                    const int co = rowid[s] * G + j;
+                    if (co >= a.cout) continue;
+                    const float bv = a.bias ? __ldg(a.bias + co) : 0.0f;
 #pragma unroll
-                for (int gi = 0; gi < NG; ++gi) {
-                    float v[VG];
-#pragma unroll
-                    for (int t = 0; t < VG; ++t) {
-                        v[t] = acc[s][j][gi * VG + t] + bv;
-                        if (a.relu) v[t] = fmaxf(v[t], 0.0f);
-                    }
-                    if (a.st_vec) {
-                        if (yok[gi]) store_vec<XT, YT, VG>(ybase + yoff[gi] + (size_t)co * a.hw, v);
-                    } else {
+                    for (int gi = 0; gi < NG; ++gi) {
+                        float v[VG];
 #pragma unroll
                         for (int t = 0; t < VG; ++t) {
-                            const int q = q0 + gi * (32 * VG) + lane * VG + t;
-                            if (q < a.q_total) {
-                                const int n = q / a.hw;
-                                store_one<YT>(ybase + ((size_t)n * a.cout + co) * a.hw + (q - n * a.hw), v[t]);
+                            v[t] = acc[s][j][gi * VG + t] + bv;
+                            if (a.relu) v[t] = fmaxf(v[t], 0.0f);
+                        }
+                        if (a.st_vec) {
+                            if (yok[gi]) store_vec<YT, VG>(ybase + yoff[gi] + (size_t)co * a.hw, v);
+                        } else {
+#pragma unroll
+                            for (int t = 0; t < VG; ++t) {
+                                const int q = q0 + gi * (32 * VG) + lane * VG + t;
+                                if (q < a.q_total) {
+                                    const int n = q / a.hw;
+                                    store_one<YT>(ybase + ((size_t)n * a.cout + co) * a.hw + (q - n * a.hw), v[t]);
+                                }
                             }
                         }
                     }
                 }
             }
+        };
+        if constexpr (sizeof(XT) == 4) {
+            epilogue(static_cast<float*>(a.y));
+        } else {
+            if (a.y_f32) epilogue(static_cast<float*>(a.y));
+            else epilogue(static_cast<__half*>(a.y));
         }
-    };
-    if constexpr (sizeof(XT) == 4) {
-        epilogue(static_cast<float*>(a.y));
-    } else {
-        if (a.y_f32) epilogue(static_cast<float*>(a.y));
-        else epilogue(static_cast<__half*>(a.y));
     }
 }
 

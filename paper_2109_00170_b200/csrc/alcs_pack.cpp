@@ -53,59 +53,95 @@ float half_bits_to_float(uint16_t h)
     return f;
 }
 
-void build_row_order(const alcs_packed& p, std::vector<int>& order)
+static int rec_bytes(int g) { return g == 1 ? 16 : 16 + 8 * g; }
+
+void build_schedule(const alcs_packed& p, int kc, int n_rg, bool with_records, Schedule& out)
 {
-    order.resize(p.rows);
+    if (kc <= 0 || kc > p.cin) kc = p.cin;
+    const int R = p.rows, g = p.g;
+    n_rg = std::max(1, std::min(n_rg, R));
+    const int nch = (p.cin + kc - 1) / kc;
+    const int rpg = (R + n_rg - 1) / n_rg;
+    const int REC = rec_bytes(g);
+    out.kc = kc; out.nch = nch; out.n_rg = n_rg; out.rpg = rpg;
+
+    // rows by descending kept-block count, dealt to the row groups in serpentine order
+    std::vector<int> order(R);
     std::iota(order.begin(), order.end(), 0);
     std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
         return p.row_ptr[a + 1] - p.row_ptr[a] > p.row_ptr[b + 1] - p.row_ptr[b];
     });
-}
-
-void build_schedule(const alcs_packed& p, int kc, HostSchedule& out)
-{
-    if (kc <= 0 || kc > p.cin) kc = p.cin;
-    const int nch = (p.cin + kc - 1) / kc;
-    out.kc = kc;
-    out.nch = nch;
-    out.seg_ptr.assign((size_t)p.rows * (nch + 1), 0);
-    out.cols.clear();
-    out.vals.clear();
-    out.cols.reserve(p.nb + (size_t)p.rows * nch);
-    out.vals.reserve(((size_t)p.nb + (size_t)p.rows * nch) * p.g);
-    const int g = p.g;
-    for (int r = 0; r < p.rows; ++r) {
-        int k = p.row_ptr[r];
-        const int kend = p.row_ptr[r + 1];
-        for (int c = 0; c < nch; ++c) {
-            out.seg_ptr[(size_t)r * (nch + 1) + c] = (int)out.cols.size();
-            const int lim = (c + 1) * kc;
-            int cnt = 0;
-            while (k < kend && p.col_idx[k] < lim) {
-                out.cols.push_back(p.col_idx[k] - c * kc);
-                for (int j = 0; j < g; ++j) {
-                    const size_t vi = (size_t)k * g + j;
-                    float v;
-                    if (p.dt == ALCS_F32) {
-                        std::memcpy(&v, &p.vals[vi * 4], 4);
-                    } else {
-                        uint16_t hb;
-                        std::memcpy(&hb, &p.vals[vi * 2], 2);
-                        v = half_bits_to_float(hb);
-                    }
-                    out.vals.push_back(v);
-                }
-                ++k;
-                ++cnt;
-            }
-            if (cnt & 1) {  // pad to an even count: same column again, zero weights
-                out.cols.push_back(out.cols.back());
-                for (int j = 0; j < g; ++j) out.vals.push_back(0.0f);
-            }
-        }
-        out.seg_ptr[(size_t)r * (nch + 1) + nch] = (int)out.cols.size();
+    out.h_rowmap.assign((size_t)n_rg * rpg, -1);
+    for (int i = 0; i < R; ++i) {
+        const int t = i / n_rg, j = i % n_rg;
+        const int rg = (t & 1) ? n_rg - 1 - j : j;
+        out.h_rowmap[(size_t)rg * rpg + t] = order[i];
     }
-    out.nbp = (int)out.cols.size();
+
+    out.h_slice.assign((size_t)n_rg * nch + 1, 0);
+    out.h_rowoff.assign((size_t)n_rg * nch * (rpg + 1), 0);
+    out.h_rec.clear();
+    std::vector<int> cursor(R);
+    int rec_count = 0, wcap = 0;
+    auto value = [&](int k, int j) -> float {
+        const size_t vi = (size_t)k * g + j;
+        float v;
+        if (p.dt == ALCS_F32) {
+            std::memcpy(&v, &p.vals[vi * 4], 4);
+        } else {
+            uint16_t hb;
+            std::memcpy(&hb, &p.vals[vi * 2], 2);
+            v = half_bits_to_float(hb);
+        }
+        return v;
+    };
+    for (int rg = 0; rg < n_rg; ++rg) {
+        for (int t = 0; t < rpg; ++t) {
+            const int r = out.h_rowmap[(size_t)rg * rpg + t];
+            if (r >= 0) cursor[r] = p.row_ptr[r];
+        }
+        for (int c = 0; c < nch; ++c) {
+            out.h_slice[(size_t)rg * nch + c] = rec_count;
+            int* roff = &out.h_rowoff[((size_t)rg * nch + c) * (rpg + 1)];
+            const int lim = (c + 1) * kc;
+            int local = 0;
+            for (int t = 0; t < rpg; ++t) {
+                roff[t] = local;
+                const int r = out.h_rowmap[(size_t)rg * rpg + t];
+                if (r < 0) continue;
+                int k = cursor[r];
+                const int kend = p.row_ptr[r + 1];
+                int k1 = k;
+                while (k1 < kend && p.col_idx[k1] < lim) ++k1;
+                const int npair = (k1 - k + 1) / 2;
+                if (with_records) {
+                    const size_t base = out.h_rec.size();
+                    out.h_rec.resize(base + (size_t)npair * REC, 0);
+                    for (int q = 0; q < npair; ++q) {
+                        unsigned char* rec = &out.h_rec[base + (size_t)q * REC];
+                        const int ka = k + 2 * q;
+                        const bool has_b = ka + 1 < k1;
+                        const int kb = has_b ? ka + 1 : ka;          // padding repeats the column
+                        int hdr[4] = {p.col_idx[ka] - c * kc, p.col_idx[kb] - c * kc, 0, 0};
+                        float* w = reinterpret_cast<float*>(rec + (g == 1 ? 8 : 16));
+                        for (int j = 0; j < g; ++j) {
+                            w[j] = value(ka, j);
+                            w[g + j] = has_b ? value(kb, j) : 0.0f;
+                        }
+                        std::memcpy(rec, hdr, g == 1 ? 8 : 16);
+                    }
+                }
+                local += npair;
+                cursor[r] = k1;
+            }
+            roff[rpg] = local;
+            rec_count += local;
+            wcap = std::max(wcap, local);
+        }
+    }
+    out.h_slice[(size_t)n_rg * nch] = rec_count;
+    out.n_rec = rec_count;
+    out.wcap = wcap;
 }
 
 }  // namespace alcs
@@ -143,9 +179,9 @@ ALCS_API int alcs_pack(const void* w, const uint8_t* block_mask, int cout, int c
     // count kept blocks first so that overflow is detected before anything is allocated
     uint64_t nb64 = 0;
     for (size_t i = 0, e = (size_t)rows * cin; i < e; ++i) nb64 += block_mask[i] != 0;
-    // the device schedules pad every (row, 32-channel chunk) segment by at most one block and
+    // the launch schedules pad every (row, 16-channel chunk) segment by at most one block and
     // index values as block * g with int32
-    const uint64_t worst = (nb64 + (uint64_t)rows * (uint64_t)((cin + 31) / 32)) * (uint64_t)g;
+    const uint64_t worst = (nb64 + ((uint64_t)rows + 4) * (uint64_t)((cin + 15) / 16)) * (uint64_t)g;
     if (worst >= (uint64_t)std::numeric_limits<int32_t>::max()) return ALCS_ERR_SHAPE;
     alcs_packed* p = new (std::nothrow) alcs_packed();
     if (!p) return ALCS_ERR_ALLOC;

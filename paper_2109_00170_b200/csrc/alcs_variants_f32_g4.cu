@@ -5,21 +5,26 @@
 namespace alcs {
 
 static const KernelVariant kTable[] = {
-    //            XT   f16 G  P RW  NW MINB
-    ALCS_VARIANT(float, 0, 4, 8, 1, 8, 2),
-    ALCS_VARIANT(float, 0, 4, 8, 2, 8, 2),
-    ALCS_VARIANT(float, 0, 4, 8, 3, 8, 1),
-    ALCS_VARIANT(float, 0, 4, 8, 4, 8, 1),
-    ALCS_VARIANT(float, 0, 4, 8, 1, 16, 1),
-    ALCS_VARIANT(float, 0, 4, 8, 2, 16, 1),
-    ALCS_VARIANT(float, 0, 4, 8, 3, 16, 1),
-    ALCS_VARIANT(float, 0, 4, 4, 1, 8, 4),
-    ALCS_VARIANT(float, 0, 4, 4, 2, 8, 4),
-    ALCS_VARIANT(float, 0, 4, 4, 2, 8, 2),
-    ALCS_VARIANT(float, 0, 4, 4, 4, 8, 2),
-    ALCS_VARIANT(float, 0, 4, 4, 8, 8, 1),
-    ALCS_VARIANT(float, 0, 4, 4, 4, 16, 1),
-    ALCS_VARIANT(float, 0, 4, 4, 6, 16, 1),
+    //           XT   f16  G  P RW  NW MINB
+    ALCS_VARIANT(float, 0, 4, 8, 1, 7, 2),
+    ALCS_VARIANT(float, 0, 4, 8, 2, 7, 2),
+    ALCS_VARIANT(float, 0, 4, 8, 3, 7, 1),
+    ALCS_VARIANT(float, 0, 4, 8, 4, 7, 1),
+    ALCS_VARIANT(float, 0, 4, 8, 2, 11, 1),
+    ALCS_VARIANT(float, 0, 4, 8, 3, 11, 1),
+    ALCS_VARIANT(float, 0, 4, 8, 4, 11, 1),
+    ALCS_VARIANT(float, 0, 4, 8, 1, 15, 1),
+    ALCS_VARIANT(float, 0, 4, 8, 2, 15, 1),
+    ALCS_VARIANT(float, 0, 4, 8, 3, 15, 1),
+    ALCS_VARIANT(float, 0, 4, 4, 1, 7, 4),
+    ALCS_VARIANT(float, 0, 4, 4, 2, 7, 4),
+    ALCS_VARIANT(float, 0, 4, 4, 2, 7, 2),
+    ALCS_VARIANT(float, 0, 4, 4, 4, 7, 2),
+    ALCS_VARIANT(float, 0, 4, 4, 8, 7, 1),
+    ALCS_VARIANT(float, 0, 4, 4, 4, 11, 1),
+    ALCS_VARIANT(float, 0, 4, 4, 6, 11, 1),
+    ALCS_VARIANT(float, 0, 4, 4, 4, 15, 1),
+    ALCS_VARIANT(float, 0, 4, 4, 6, 15, 1),
 };
 
 const KernelVariant* variants_f32_g4(int* n)

@@ -99,7 +99,7 @@ StageLayout stage_layout(const KernelVariant& v, const Schedule& sc, int elt)
 {
     StageLayout L;
     L.off_rec = sc.kc * 32 * v.p * elt;                              // X tile first
-    L.off_rowoff = L.off_rec + sc.wcap * alcs::record_bytes(v.g);
+    L.off_rowoff = L.off_rec + sc.wcap * 16;
     L.stage_bytes = L.off_rowoff + ((sc.rpg + 1) * 4 + 15) / 16 * 16;
     return L;
 }
@@ -172,7 +172,7 @@ double model_cost(const alcs_packed* w, const KernelVariant& v, const Schedule& 
     const long long rounds = (items + slots - 1) / slots;
     const int vg = (v.p * elt >= 16) ? 16 / elt : v.p;
     const int ng = v.p / vg;
-    const double pairs_item = (double)sc.n_rec / sc.n_rg;
+    const double pairs_item = (double)sc.n_rec * 16.0 / alcs::record_bytes(v.g) / sc.n_rg;
     const double seg_item = (double)sc.rpg * sc.nch;
     const double fma_issue = pairs_item * (2.0 * v.g * v.p + 2 * ng + 6 + (elt == 2 ? v.p : 0)) / 4.0 + seg_item * 14.0 / 4.0;
     const double lsu = pairs_item * (2.0 * ng * (vg * elt * 32 / 128.0) + 1 + v.g / 2.0) +
@@ -384,15 +384,23 @@ int check_device(const alcs_packed* w)
 int resolve_plan(const alcs_packed* w, int n, int h, int wd, unsigned flags, long long q,
                  const alcs_launch_cfg* cfg, Plan* plan)
 {
-    if (cfg) return cfg_to_plan(w, q, cfg, plan);
-    const alcs::ShapeKey key{n, h, wd, flags};
+    alcs::ShapeKey key{n, h, wd, flags};
+    if (cfg) {
+        const int c[7] = {cfg->pixels_per_lane, cfg->rows_per_warp, cfg->warps, cfg->chunk_channels,
+                          cfg->stages, cfg->row_groups, cfg->min_blocks};
+        for (int i = 0; i < 7; ++i) key.c[i] = c[i];
+    }
     {
         std::lock_guard<std::mutex> lk(w->mu);
         auto it = w->plan_cache.find(key);
         if (it != w->plan_cache.end()) { *plan = it->second; return ALCS_OK; }
     }
-    auto it = w->tuned.find(key);
-    const int rc = cfg_to_plan(w, q, it != w->tuned.end() ? &it->second : nullptr, plan);
+    const alcs_launch_cfg* use = cfg;
+    if (!use) {
+        auto it = w->tuned.find(key);
+        if (it != w->tuned.end()) use = &it->second;
+    }
+    const int rc = cfg_to_plan(w, q, use, plan);
     if (rc) return rc;
     std::lock_guard<std::mutex> lk(w->mu);
     w->plan_cache[key] = *plan;

@@ -26,16 +26,18 @@ constexpr int kChunkings[kNumChunkings] = {16, 32, 64, 128, 0};
 // number of blocks whatever the distribution of row lengths.  rowmap[rg][t] is the block row that
 // is local row t of row group rg (-1 = none).
 //
-// The kept blocks are stored as "pair records" ordered [row group][chunk][local row][pair]: two
-// chunk-local column indices followed by their two g-wide value vectors (fp32; fp16 weights are
-// widened exactly).  A local row with an odd number of blocks in a chunk gets a padding block
-// that repeats its last column with zero weights.  slice[rg*nch + k] is the first record of the
-// (row group, chunk) slice, so the producer warp copies one contiguous range per stage;
-// rowoff[rg][k][t] is where local row t starts inside that slice (rowoff[..][rpg] = its length).
+// The kept blocks are stored as segments ordered [row group][chunk][local row].  The segment of a
+// local row with blocks in a chunk is a 16-byte lead entry (the chunk-local columns of its first
+// two blocks) followed by one "pair record" per two blocks: the columns of the NEXT pair, then the
+// two g-wide value vectors of this pair (fp32; fp16 weights are widened exactly).  An odd block
+// count gets a padding block that repeats the last column with zero weights.  slice[rg*nch + k]
+// is where the (row group, chunk) slice starts, so the producer warp copies one contiguous range
+// per stage; rowoff[rg][k][t] is where local row t starts inside that slice (rowoff[..][rpg] =
+// its length).  All offsets are in 16-byte units.
 struct Schedule {
     int kc = 0, nch = 0, n_rg = 0, rpg = 0;
-    int wcap = 0;                  // longest slice, in records
-    int n_rec = 0;                 // total records
+    int wcap = 0;                  // longest slice, in 16-byte units
+    int n_rec = 0;                 // total length of all slices, in 16-byte units
     // host copies (kept until uploaded)
     std::vector<unsigned char> h_rec;
     std::vector<int> h_slice, h_rowoff, h_rowmap;
@@ -59,11 +61,17 @@ struct Plan {
     double cost = 0;       // model estimate, seconds
 };
 
+// Key of the plan cache: the problem shape plus the requested configuration (all zero = automatic).
 struct ShapeKey {
     int n, h, wd;
     unsigned flags;
+    int c[7] = {0, 0, 0, 0, 0, 0, 0};
     bool operator<(const ShapeKey& o) const {
-        return std::tie(n, h, wd, flags) < std::tie(o.n, o.h, o.wd, o.flags);
+        if (std::tie(n, h, wd, flags) != std::tie(o.n, o.h, o.wd, o.flags))
+            return std::tie(n, h, wd, flags) < std::tie(o.n, o.h, o.wd, o.flags);
+        for (int i = 0; i < 7; ++i)
+            if (c[i] != o.c[i]) return c[i] < o.c[i];
+        return false;
     }
 };
 

@@ -36,21 +36,23 @@
 namespace alcs {
 
 constexpr int kMaxStages = 8;
-constexpr int kWaitLimit = 1 << 22;     // polls of mbarrier.try_wait before giving up
+constexpr int kWaitLimit = 1 << 21;     // polls of mbarrier.try_wait before giving up (about a second)
 constexpr int kErrFullWait = 1;         // a consumer gave up waiting for data
 constexpr int kErrEmptyWait = 2;        // the producer gave up waiting for a free stage
 
-// bytes of one pair record: header (2 column indices, padded to 16 bytes unless G == 1, where
-// the two values share the header's 16 bytes) followed by 2*G fp32 values
+// Bytes of one pair record: a header with the two column indices of the NEXT pair of the segment
+// (padded to 16 bytes unless G == 1, where the two values share the header's 16 bytes) followed
+// by the 2*G fp32 values of this pair.  A segment starts with a 16-byte lead entry that holds the
+// column indices of its first pair.
 __host__ __device__ constexpr int record_bytes(int g) { return g == 1 ? 16 : 16 + 8 * g; }
 
 struct ConvArgs {
     const void* x;            // [n][cin][hw] of XT
     void* y;                  // [n][cout][hw] of XT, or float if y_f32
     const float* bias;        // [cout] or nullptr
-    const unsigned char* rec; // pair records, ordered [row group][chunk][local row][pair]
-    const int* slice;         // [n_rg*nch + 1] first record of each (row group, chunk) slice
-    const int* rowoff;        // [n_rg][nch][rpg+1] record offsets of the local rows inside a slice
+    const unsigned char* rec; // segments of pair records, ordered [row group][chunk][local row]
+    const int* slice;         // [n_rg*nch + 1] start of each (row group, chunk) slice, in 16-byte units
+    const int* rowoff;        // [n_rg][nch][rpg+1] start of each local row's segment inside a slice (16-byte units)
     const int* rowmap;        // [n_rg][rpg] block row of each local row, -1 = none
     int* err;                 // device error word (0 = ok)
     int rows, cin, cout, hw;
@@ -95,18 +97,21 @@ __device__ __forceinline__ void mbar_arrive_on_copies(uint32_t bar)
 {
     asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];\n" ::"r"(bar) : "memory");
 }
-// Bounded wait for the phase with the given parity to complete.
+// Bounded wait for the phase with the given parity to complete.  Each poll lets the hardware
+// suspend the warp for up to about a microsecond, and failed polls back off with nanosleep, so a
+// waiting warp does not take issue slots from the warps that compute.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
 {
     for (int it = 0; it < kWaitLimit; ++it) {
         uint32_t done;
         asm volatile(
-            "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+            "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
             " selp.u32 %0, 1, 0, p;\n}\n"
             : "=r"(done)
-            : "r"(bar), "r"(parity)
+            : "r"(bar), "r"(parity), "r"(1000u)
             : "memory");
         if (done) return true;
+        if (it > 4) __nanosleep(it > 64 ? 256 : 64);
     }
     return false;
 }
@@ -151,6 +156,21 @@ struct XVec<__half, 4> {
     }
 };
 
+// The P pixels a lane owns of one staged channel row: P/VG vector loads, 32*VG elements apart.
+template <typename XT, int P>
+__device__ __forceinline__ void load_x(const unsigned char* p, float (&x)[P])
+{
+    constexpr int SZ = (int)sizeof(XT);
+    constexpr int VG = (P * SZ >= 16) ? 16 / SZ : P;
+#pragma unroll
+    for (int gi = 0; gi < P / VG; ++gi) {
+        float v[VG];
+        XVec<XT, VG>::load(p + gi * (32 * VG * SZ), v);
+#pragma unroll
+        for (int t = 0; t < VG; ++t) x[gi * VG + t] = v[t];
+    }
+}
+
 // One pair record from shared memory (same address in every lane: broadcasts).
 template <int G>
 __device__ __forceinline__ void load_record(const unsigned char* p, int& c0, int& c1, float (&w0)[G],
@@ -175,6 +195,92 @@ __device__ __forceinline__ void load_record(const unsigned char* p, int& c0, int
         for (int i = 0; i < G / 4; ++i) {
             const float4 v = *reinterpret_cast<const float4*>(p + 16 + 4 * G + 16 * i);
             w1[4 * i] = v.x; w1[4 * i + 1] = v.y; w1[4 * i + 2] = v.z; w1[4 * i + 3] = v.w;
+        }
+    }
+}
+
+// G (>= 4) weights of one block from shared memory (warp-uniform address).
+template <int G>
+__device__ __forceinline__ void load_w(const unsigned char* p, float (&w)[G])
+{
+#pragma unroll
+    for (int i = 0; i < G / 4; ++i) {
+        const float4 v = *reinterpret_cast<const float4*>(p + 16 * i);
+        w[4 * i] = v.x; w[4 * i + 1] = v.y; w[4 * i + 2] = v.z; w[4 * i + 3] = v.w;
+    }
+}
+
+// acc[j][t] += w[j] * x[t]: the G x P outer-product update of one block.
+template <int G, int P>
+__device__ __forceinline__ void fma_block(float (&acc)[G][P], const float (&w)[G], const float (&x)[P])
+{
+#pragma unroll
+    for (int j = 0; j < G; ++j)
+#pragma unroll
+        for (int t = 0; t < P; ++t) acc[j][t] = fmaf(w[j], x[t], acc[j][t]);
+}
+
+// Multiply-accumulate one (block row, chunk) segment of pair records into the lane's G x P
+// accumulators.  xs points at this lane's first pixel vector of the staged X tile; [rp, re) is the
+// segment in shared memory.
+template <typename XT, int G, int P>
+__device__ __forceinline__ void consume_segment(float (&acc)[G][P], const unsigned char* xs,
+                                                const unsigned char* rp, const unsigned char* re)
+{
+    constexpr int ROWB = 32 * P * (int)sizeof(XT);
+    constexpr int REC = record_bytes(G);
+    // A segment is a 16-byte lead entry with the columns of pair 0, then one record per
+    // pair holding the columns of the NEXT pair and the weights of this one.  So the
+    // loads issued while pair i is multiplied (record i+1, X vectors of pair i+1)
+    // depend only on data that arrived while pair i-1 was multiplied.  Two register
+    // sets (A, B) alternate; nothing is copied between them.
+    const int2 lead = *reinterpret_cast<const int2*>(rp);
+    rp += 16;
+    int ca0 = lead.x, ca1 = lead.y, cb0 = 0, cb1 = 0;
+    if constexpr (G <= 4) {
+        float wA0[G], wA1[G], wB0[G], wB1[G];
+        float xA0[P], xA1[P], xB0[P], xB1[P];
+        load_record<G>(rp, cb0, cb1, wA0, wA1);
+        load_x<XT, P>(xs + ca0 * ROWB, xA0);
+        load_x<XT, P>(xs + ca1 * ROWB, xA1);
+        while (true) {
+            const bool moreB = rp + REC < re;
+            if (moreB) {
+                load_record<G>(rp + REC, ca0, ca1, wB0, wB1);
+                load_x<XT, P>(xs + cb0 * ROWB, xB0);
+                load_x<XT, P>(xs + cb1 * ROWB, xB1);
+            }
+            fma_block<G, P>(acc, wA0, xA0);
+            fma_block<G, P>(acc, wA1, xA1);
+            if (!moreB) break;
+            const bool moreA = rp + 2 * REC < re;
+            if (moreA) {
+                load_record<G>(rp + 2 * REC, cb0, cb1, wA0, wA1);
+                load_x<XT, P>(xs + ca0 * ROWB, xA0);
+                load_x<XT, P>(xs + ca1 * ROWB, xA1);
+            }
+            fma_block<G, P>(acc, wB0, xB0);
+            fma_block<G, P>(acc, wB1, xB1);
+            if (!moreA) break;
+            rp += 2 * REC;
+        }
+    } else {
+        // Wide groups: every X word already feeds 8 or 16 FMAs and the accumulators
+        // fill most of the register file, so nothing but the next pair's columns is
+        // fetched ahead; the weights of each block are loaded just before its FMAs.
+        while (true) {
+            float x0[P], x1[P], w[G];
+            load_x<XT, P>(xs + ca0 * ROWB, x0);
+            load_x<XT, P>(xs + ca1 * ROWB, x1);
+            const int2 nx = *reinterpret_cast<const int2*>(rp);
+            load_w<G>(rp + 16, w);
+            fma_block<G, P>(acc, w, x0);
+            load_w<G>(rp + 16 + 4 * G, w);
+            fma_block<G, P>(acc, w, x1);
+            if (rp + REC >= re) break;
+            ca0 = nx.x;
+            ca1 = nx.y;
+            rp += REC;
         }
     }
 }
@@ -219,7 +325,6 @@ __device__ __forceinline__ void produce(const ConvArgs& a, unsigned char* smem, 
     constexpr int VPR = T / EV;             // copies per channel row
     constexpr int NCOL = VPR >= 32 ? VPR / 32 : 1;   // copies per channel row per lane
     constexpr int RP = VPR >= 32 ? 1 : 32 / VPR;     // channel rows the warp covers per pass
-    constexpr int REC = record_bytes(G);
     const int vlane = lane % VPR;           // (== lane when VPR >= 32)
     const int rlane = lane / VPR;           // first channel row of this lane (0 when VPR >= 32)
 
@@ -280,8 +385,8 @@ __device__ __forceinline__ void produce(const ConvArgs& a, unsigned char* smem, 
             }
             // the row group's pair records of this chunk and their per-row offsets
             const int r0 = __ldg(slice + k);
-            const int n16 = (__ldg(slice + k + 1) - r0) * (REC / 16);
-            const unsigned char* rsrc = a.rec + (size_t)r0 * REC;
+            const int n16 = __ldg(slice + k + 1) - r0;
+            const unsigned char* rsrc = a.rec + (size_t)r0 * 16;
             for (int i = lane; i < n16; i += 32) cp_async_16(st + a.off_rec + i * 16, rsrc + (size_t)i * 16);
             const int* osrc = rowoff + (size_t)k * (a.rpg + 1);
             for (int i = lane; i <= a.rpg; i += 32) cp_async_4(st + a.off_rowoff + i * 4, osrc + i);
@@ -369,35 +474,9 @@ __global__ void __launch_bounds__((NW + 1) * 32, MINB) spconv1x1_kernel(const Co
 #pragma unroll
             for (int s = 0; s < RW; ++s) {
                 if (lrow[s] >= a.rpg) continue;
-                const unsigned char* rp = recs + roff[lrow[s]] * REC;
-                const unsigned char* re = recs + roff[lrow[s] + 1] * REC;
-                for (; rp < re; rp += REC) {
-                    int c0, c1;
-                    float w0[G], w1[G];
-                    load_record<G>(rp, c0, c1, w0, w1);
-                    const unsigned char* x0p = xs + c0 * ROWB;
-                    const unsigned char* x1p = xs + c1 * ROWB;
-#pragma unroll
-                    for (int gi = 0; gi < NG; ++gi) {
-                        float xv[VG];
-                        XVec<XT, VG>::load(x0p + gi * (32 * VG * SZ), xv);
-#pragma unroll
-                        for (int j = 0; j < G; ++j)
-#pragma unroll
-                            for (int t = 0; t < VG; ++t)
-                                acc[s][j][gi * VG + t] = fmaf(w0[j], xv[t], acc[s][j][gi * VG + t]);
-                    }
-#pragma unroll
-                    for (int gi = 0; gi < NG; ++gi) {
-                        float xv[VG];
-                        XVec<XT, VG>::load(x1p + gi * (32 * VG * SZ), xv);
-#pragma unroll
-                        for (int j = 0; j < G; ++j)
-#pragma unroll
-                            for (int t = 0; t < VG; ++t)
-                                acc[s][j][gi * VG + t] = fmaf(w1[j], xv[t], acc[s][j][gi * VG + t]);
-                    }
-                }
+                const unsigned char* rp = recs + roff[lrow[s]] * 16;
+                const unsigned char* re = recs + roff[lrow[s] + 1] * 16;
+                if (rp < re) consume_segment<XT, G, P>(acc[s], xs, rp, re);
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32 + 8 * kMaxStages + 8 * st);   // stage st may be refilled

@@ -104,6 +104,7 @@ void build_schedule(const alcs_packed& p, int kc, int n_rg, bool with_records, S
             out.h_slice[(size_t)rg * nch + c] = rec_count;
             int* roff = &out.h_rowoff[((size_t)rg * nch + c) * (rpg + 1)];
             const int lim = (c + 1) * kc;
+            const int c0 = c * kc;
             int local = 0;
             for (int t = 0; t < rpg; ++t) {
                 roff[t] = local;
@@ -114,24 +115,34 @@ void build_schedule(const alcs_packed& p, int kc, int n_rg, bool with_records, S
                 int k1 = k;
                 while (k1 < kend && p.col_idx[k1] < lim) ++k1;
                 const int npair = (k1 - k + 1) / 2;
-                if (with_records) {
+                const int seg16 = npair ? 1 + npair * (REC / 16) : 0;   // lead entry + records
+                if (with_records && npair) {
                     const size_t base = out.h_rec.size();
-                    out.h_rec.resize(base + (size_t)npair * REC, 0);
+                    out.h_rec.resize(base + (size_t)seg16 * 16, 0);
+                    auto cols_of = [&](int q, int* c) {       // chunk-local columns of pair q
+                        const int ka = k + 2 * q;
+                        const int kb = ka + 1 < k1 ? ka + 1 : ka;    // padding repeats the column
+                        c[0] = p.col_idx[ka] - c0;
+                        c[1] = p.col_idx[kb] - c0;
+                    };
+                    int lead[4] = {0, 0, 0, 0};
+                    cols_of(0, lead);
+                    std::memcpy(&out.h_rec[base], lead, 16);
                     for (int q = 0; q < npair; ++q) {
-                        unsigned char* rec = &out.h_rec[base + (size_t)q * REC];
+                        unsigned char* rec = &out.h_rec[base + 16 + (size_t)q * REC];
                         const int ka = k + 2 * q;
                         const bool has_b = ka + 1 < k1;
-                        const int kb = has_b ? ka + 1 : ka;          // padding repeats the column
-                        int hdr[4] = {p.col_idx[ka] - c * kc, p.col_idx[kb] - c * kc, 0, 0};
+                        int hdr[4] = {0, 0, 0, 0};
+                        if (q + 1 < npair) cols_of(q + 1, hdr);       // columns of the next pair
                         float* w = reinterpret_cast<float*>(rec + (g == 1 ? 8 : 16));
                         for (int j = 0; j < g; ++j) {
                             w[j] = value(ka, j);
-                            w[g + j] = has_b ? value(kb, j) : 0.0f;
+                            w[g + j] = has_b ? value(ka + 1, j) : 0.0f;
                         }
                         std::memcpy(rec, hdr, g == 1 ? 8 : 16);
                     }
                 }
-                local += npair;
+                local += seg16;
                 cursor[r] = k1;
             }
             roff[rpg] = local;

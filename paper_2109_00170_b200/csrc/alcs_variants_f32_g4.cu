@@ -6,25 +6,30 @@ namespace alcs {
 
 static const KernelVariant kTable[] = {
     //           XT   f16  G  P RW  NW MINB
-    ALCS_VARIANT(float, 0, 4, 8, 1, 7, 2),
-    ALCS_VARIANT(float, 0, 4, 8, 2, 7, 2),
-    ALCS_VARIANT(float, 0, 4, 8, 3, 7, 1),
-    ALCS_VARIANT(float, 0, 4, 8, 4, 7, 1),
-    ALCS_VARIANT(float, 0, 4, 8, 2, 11, 1),
-    ALCS_VARIANT(float, 0, 4, 8, 3, 11, 1),
-    ALCS_VARIANT(float, 0, 4, 8, 4, 11, 1),
+    ALCS_VARIANT(float, 0, 4, 8, 1, 7, 1),
+    ALCS_VARIANT(float, 0, 4, 8, 1, 11, 1),
+    ALCS_VARIANT(float, 0, 4, 8, 1, 13, 1),
     ALCS_VARIANT(float, 0, 4, 8, 1, 15, 1),
-    ALCS_VARIANT(float, 0, 4, 8, 2, 15, 1),
-    ALCS_VARIANT(float, 0, 4, 8, 3, 15, 1),
-    ALCS_VARIANT(float, 0, 4, 4, 1, 7, 4),
-    ALCS_VARIANT(float, 0, 4, 4, 2, 7, 4),
-    ALCS_VARIANT(float, 0, 4, 4, 2, 7, 2),
-    ALCS_VARIANT(float, 0, 4, 4, 4, 7, 2),
-    ALCS_VARIANT(float, 0, 4, 4, 8, 7, 1),
+    ALCS_VARIANT(float, 0, 4, 8, 2, 7, 1),
+    ALCS_VARIANT(float, 0, 4, 8, 2, 11, 1),
+    ALCS_VARIANT(float, 0, 4, 8, 2, 13, 1),
+    ALCS_VARIANT(float, 0, 4, 8, 3, 7, 1),
+    ALCS_VARIANT(float, 0, 4, 8, 3, 11, 1),
+    ALCS_VARIANT(float, 0, 4, 8, 4, 7, 1),
+    ALCS_VARIANT(float, 0, 4, 8, 1, 7, 2),
+    ALCS_VARIANT(float, 0, 4, 4, 2, 7, 1),
+    ALCS_VARIANT(float, 0, 4, 4, 4, 7, 1),
+    ALCS_VARIANT(float, 0, 4, 4, 2, 11, 1),
     ALCS_VARIANT(float, 0, 4, 4, 4, 11, 1),
-    ALCS_VARIANT(float, 0, 4, 4, 6, 11, 1),
+    ALCS_VARIANT(float, 0, 4, 4, 2, 15, 1),
     ALCS_VARIANT(float, 0, 4, 4, 4, 15, 1),
-    ALCS_VARIANT(float, 0, 4, 4, 6, 15, 1),
+    ALCS_VARIANT(float, 0, 4, 4, 6, 7, 1),
+    ALCS_VARIANT(float, 0, 4, 4, 6, 11, 1),
+    ALCS_VARIANT(float, 0, 4, 4, 4, 7, 2),
+    ALCS_VARIANT(float, 0, 4, 4, 2, 7, 2),
+    ALCS_VARIANT(float, 0, 4, 16, 1, 7, 1),
+    ALCS_VARIANT(float, 0, 4, 16, 1, 11, 1),
+    ALCS_VARIANT(float, 0, 4, 16, 2, 7, 1),
 };
 
 const KernelVariant* variants_f32_g4(int* n)

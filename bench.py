@@ -179,7 +179,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--layers", default="", help="comma-separated layer indices (default: all)")
     ap.add_argument("--cfg", default="", help="force one launch configuration for every layer: "
-                    "pixels_per_lane,rows_per_warp,warps,chunk_channels,stages,row_groups,min_blocks")
+                    "pixels_per_lane,rows_per_warp,warps,chunk_channels,stages,row_groups,min_blocks[,copy_mode]")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "alcs" else args.warmup
     wl = args.workload
@@ -220,7 +220,7 @@ def main():
         flags = A.ALCS_RELU if s.relu else 0
         forced = None
         if args.cfg:
-            keys = ("pixels_per_lane", "rows_per_warp", "warps", "chunk_channels", "stages", "row_groups", "min_blocks")
+            keys = ("pixels_per_lane", "rows_per_warp", "warps", "chunk_channels", "stages", "row_groups", "min_blocks", "copy_mode")
             forced = dict(zip(keys, (int(v) for v in args.cfg.split(","))))
             cfg = forced
         else:

@@ -157,9 +157,11 @@ ALCS_API void alcs_packed_free(alcs_packed* p);
  *   stages            pipeline depth (2..8)
  *   row_groups        how many work items share one pixel tile, each taking a subset of rows
  *   min_blocks        thread blocks per SM the kernel is compiled for (1 or 2)
+ *   copy_mode         how X tiles reach shared memory: 1 = per-lane cp.async, 2 = bulk (TMA) copies
+ *                     of whole pixel runs (needs 16-byte aligned rows; otherwise 1 is used)
  */
 typedef struct {
-    int pixels_per_lane, rows_per_warp, warps, chunk_channels, stages, row_groups, min_blocks;
+    int pixels_per_lane, rows_per_warp, warps, chunk_channels, stages, row_groups, min_blocks, copy_mode;
 } alcs_launch_cfg;
 
 /*

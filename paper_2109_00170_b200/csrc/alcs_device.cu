@@ -100,7 +100,7 @@ StageLayout stage_layout(const KernelVariant& v, const Schedule& sc, int elt)
     StageLayout L;
     L.off_rec = sc.kc * 32 * v.p * elt;                              // X tile first
     L.off_rowoff = L.off_rec + sc.wcap * 16;
-    L.stage_bytes = L.off_rowoff + ((sc.rpg + 1) * 4 + 15) / 16 * 16;
+    L.stage_bytes = L.off_rowoff + sc.ros * 4;
     return L;
 }
 
@@ -197,7 +197,7 @@ int occupancy_of(const VariantInfo& vi, size_t smem)
 }
 
 // Enumerate every valid launch configuration for this shape, cheapest (by the model) first.
-int enumerate_plans(const alcs_packed* w, long long q, std::vector<Plan>& out)
+int enumerate_plans(const alcs_packed* w, long long q, int hw, std::vector<Plan>& out)
 {
     DeviceInfo di;
     int rc = device_info(w->device, &di);
@@ -242,7 +242,17 @@ int enumerate_plans(const alcs_packed* w, long long q, std::vector<Plan>& out)
                     p.cost = model_cost(w, v, *sc, q, di.sms, occ);
                     // deeper rings only help while there are chunks to prefetch; prefer the shallowest
                     p.cost *= 1.0 + 0.01 * stages;
+                    // Bulk copies pay a fixed cost per copy, so they win when a tile row is one long
+                    // run (images at least as large as the tile) and lose when it is cut into pieces.
+                    const bool rows_aligned = ((size_t)hw * elt) % 16 == 0;
+                    p.bulk = (rows_aligned && hw >= 32 * v.p) ? 1 : 0;
                     out.push_back(p);
+                    if (rows_aligned) {
+                        Plan p2 = p;
+                        p2.bulk = 1 - p.bulk;
+                        p2.cost *= 1.25;
+                        out.push_back(p2);
+                    }
                 }
             }
         }
@@ -261,13 +271,14 @@ void plan_to_cfg(const Plan& p, alcs_launch_cfg* c)
     c->stages = p.stages;
     c->row_groups = p.n_rg;
     c->min_blocks = v.minb;
+    c->copy_mode = p.bulk ? 2 : 1;
 }
 
 // Resolve a (possibly partial) configuration into a concrete plan.
-int cfg_to_plan(const alcs_packed* w, long long q, const alcs_launch_cfg* c, Plan* out)
+int cfg_to_plan(const alcs_packed* w, long long q, int hw, const alcs_launch_cfg* c, Plan* out)
 {
     std::vector<Plan> all;
-    int rc = enumerate_plans(w, q, all);
+    int rc = enumerate_plans(w, q, hw, all);
     if (rc) return rc;
     if (!c) { *out = all[0]; return ALCS_OK; }
     auto variant_ok = [&](const Plan& p) {
@@ -278,6 +289,7 @@ int cfg_to_plan(const alcs_packed* w, long long q, const alcs_launch_cfg* c, Pla
         if (c->min_blocks && c->min_blocks != v.minb) return false;
         if (c->chunk_channels && std::min(c->chunk_channels, w->cin) != p.kc) return false;
         if (c->stages && c->stages != p.stages) return false;
+        if (c->copy_mode && (c->copy_mode == 2) != (p.bulk == 1)) return false;
         return true;
     };
     for (const Plan& p : all)
@@ -362,6 +374,8 @@ int launch_plan(const alcs_packed* w, const Plan& p, const void* x, void* y, int
     int ld = 16;
     while (ld > elt && (((size_t)hw * elt) % ld || (uintptr_t)x % ld)) ld >>= 1;
     a.ld_bytes = ld;
+    a.bulk = (ld == 16 && p.bulk) ? 1 : 0;
+    a.ros = sc->ros;
     const int vg = (v.p * elt >= 16) ? 16 / elt : v.p;
     a.st_vec = (hw % vg == 0 && (uintptr_t)y % 16 == 0) ? 1 : 0;
     const long long items = (long long)a.n_tiles * a.n_rg;
@@ -386,9 +400,9 @@ int resolve_plan(const alcs_packed* w, int n, int h, int wd, unsigned flags, lon
 {
     alcs::ShapeKey key{n, h, wd, flags};
     if (cfg) {
-        const int c[7] = {cfg->pixels_per_lane, cfg->rows_per_warp, cfg->warps, cfg->chunk_channels,
-                          cfg->stages, cfg->row_groups, cfg->min_blocks};
-        for (int i = 0; i < 7; ++i) key.c[i] = c[i];
+        const int c[8] = {cfg->pixels_per_lane, cfg->rows_per_warp, cfg->warps, cfg->chunk_channels,
+                          cfg->stages, cfg->row_groups, cfg->min_blocks, cfg->copy_mode};
+        for (int i = 0; i < 8; ++i) key.c[i] = c[i];
     }
     {
         std::lock_guard<std::mutex> lk(w->mu);
@@ -400,7 +414,7 @@ int resolve_plan(const alcs_packed* w, int n, int h, int wd, unsigned flags, lon
         auto it = w->tuned.find(key);
         if (it != w->tuned.end()) use = &it->second;
     }
-    const int rc = cfg_to_plan(w, q, use, plan);
+    const int rc = cfg_to_plan(w, q, h * wd, use, plan);
     if (rc) return rc;
     std::lock_guard<std::mutex> lk(w->mu);
     w->plan_cache[key] = *plan;
@@ -494,6 +508,7 @@ ALCS_API int alcs_variant_get(int index, alcs_dtype* dt, int* g, alcs_launch_cfg
         cfg->rows_per_warp = v.rw;
         cfg->warps = v.nw;
         cfg->min_blocks = v.minb;
+        cfg->copy_mode = 0;
     }
     return ALCS_OK;
 }
@@ -549,7 +564,7 @@ ALCS_API int alcs_spconv1x1_tune(alcs_packed* w, const void* x, void* y, int n, 
     if (q == 0) return ALCS_OK;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     std::vector<Plan> all;
-    rc = enumerate_plans(w, q, all);
+    rc = enumerate_plans(w, q, h * wd, all);
     if (rc) return rc;
     const size_t max_try = 160;
     if (all.size() > max_try) all.resize(max_try);

@@ -36,6 +36,7 @@ constexpr int kChunkings[kNumChunkings] = {16, 32, 64, 128, 0};
 // its length).  All offsets are in 16-byte units.
 struct Schedule {
     int kc = 0, nch = 0, n_rg = 0, rpg = 0;
+    int ros = 0;                   // ints per (row group, chunk) row of rowoff: rpg + 1 rounded up to 4
     int wcap = 0;                  // longest slice, in 16-byte units
     int n_rec = 0;                 // total length of all slices, in 16-byte units
     // host copies (kept until uploaded)
@@ -56,6 +57,7 @@ struct Plan {
     int kc = 0;            // schedule key: channels per chunk ...
     int n_rg = 0;          // ... and number of row groups
     int stages = 0;
+    int bulk = 0;          // 1: bulk (TMA) copies of X, 0: per-lane cp.async
     int occ = 1;           // resident thread blocks per SM
     size_t smem = 0;
     double cost = 0;       // model estimate, seconds
@@ -65,11 +67,11 @@ struct Plan {
 struct ShapeKey {
     int n, h, wd;
     unsigned flags;
-    int c[7] = {0, 0, 0, 0, 0, 0, 0};
+    int c[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     bool operator<(const ShapeKey& o) const {
         if (std::tie(n, h, wd, flags) != std::tie(o.n, o.h, o.wd, o.flags))
             return std::tie(n, h, wd, flags) < std::tie(o.n, o.h, o.wd, o.flags);
-        for (int i = 0; i < 7; ++i)
+        for (int i = 0; i < 8; ++i)
             if (c[i] != o.c[i]) return c[i] < o.c[i];
         return false;
     }

@@ -52,7 +52,7 @@ struct ConvArgs {
     const float* bias;        // [cout] or nullptr
     const unsigned char* rec; // segments of pair records, ordered [row group][chunk][local row]
     const int* slice;         // [n_rg*nch + 1] start of each (row group, chunk) slice, in 16-byte units
-    const int* rowoff;        // [n_rg][nch][rpg+1] start of each local row's segment inside a slice (16-byte units)
+    const int* rowoff;        // [n_rg][nch][ros] start of each local row's segment inside a slice (16-byte units)
     const int* rowmap;        // [n_rg][rpg] block row of each local row, -1 = none
     int* err;                 // device error word (0 = ok)
     int rows, cin, cout, hw;
@@ -62,6 +62,8 @@ struct ConvArgs {
     int relu;
     int y_f32;                // only meaningful for XT = __half
     int ld_bytes;             // bytes per X staging copy: 16, 8, 4 or 2
+    int bulk;                 // 1: the producer uses bulk (TMA) copies; needs ld_bytes == 16
+    int ros;                  // stride of rowoff per (row group, chunk), in ints (multiple of 4)
     int st_vec;               // 1 if vector stores are allowed
     // shared-memory layout (bytes): [mbarriers | stage 0 | stage 1 | ...]
     int off_rec, off_rowoff, stage_bytes;
@@ -96,6 +98,20 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 __device__ __forceinline__ void mbar_arrive_on_copies(uint32_t bar)
 {
     asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];\n" ::"r"(bar) : "memory");
+}
+// One arrival that also announces `bytes` of bulk-copy traffic still to land on `bar`.
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("{\n .reg .b64 t;\n mbarrier.arrive.expect_tx.shared::cta.b64 t, [%0], %1;\n}\n" ::"r"(bar), "r"(bytes)
+                 : "memory");
+}
+// Bulk asynchronous copy global -> shared memory (TMA, untiled): 16-byte aligned addresses, size a
+// multiple of 16; its bytes are counted down on `bar` when they have landed.  No multicast.
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
 }
 // Bounded wait for the phase with the given parity to complete.  Each poll lets the hardware
 // suspend the warp for up to about a microsecond, and failed polls back off with nanosleep, so a
@@ -223,7 +239,7 @@ __device__ __forceinline__ void fma_block(float (&acc)[G][P], const float (&w)[G
 // Multiply-accumulate one (block row, chunk) segment of pair records into the lane's G x P
 // accumulators.  xs points at this lane's first pixel vector of the staged X tile; [rp, re) is the
 // segment in shared memory.
-template <typename XT, int G, int P>
+template <typename XT, int G, int P, bool DEEP>
 __device__ __forceinline__ void consume_segment(float (&acc)[G][P], const unsigned char* xs,
                                                 const unsigned char* rp, const unsigned char* re)
 {
@@ -237,7 +253,7 @@ __device__ __forceinline__ void consume_segment(float (&acc)[G][P], const unsign
     const int2 lead = *reinterpret_cast<const int2*>(rp);
     rp += 16;
     int ca0 = lead.x, ca1 = lead.y, cb0 = 0, cb1 = 0;
-    if constexpr (G <= 4) {
+    if constexpr (G <= 4 && DEEP) {
         float wA0[G], wA1[G], wB0[G], wB1[G];
         float xA0[P], xA1[P], xB0[P], xB1[P];
         load_record<G>(rp, cb0, cb1, wA0, wA1);
@@ -262,6 +278,32 @@ __device__ __forceinline__ void consume_segment(float (&acc)[G][P], const unsign
             fma_block<G, P>(acc, wB0, xB0);
             fma_block<G, P>(acc, wB1, xB1);
             if (!moreA) break;
+            rp += 2 * REC;
+        }
+    } else if constexpr (G <= 4) {
+        // Register-lean flavour for thread blocks with many warps: only the records are fetched
+        // ahead (two alternating weight sets); the X vectors of a pair are loaded when the
+        // previous pair's FMAs have been issued, and other warps cover that latency.
+        float wA0[G], wA1[G], wB0[G], wB1[G];
+        float x0[P], x1[P];
+        load_record<G>(rp, cb0, cb1, wA0, wA1);
+        load_x<XT, P>(xs + ca0 * ROWB, x0);
+        load_x<XT, P>(xs + ca1 * ROWB, x1);
+        while (true) {
+            const bool moreB = rp + REC < re;
+            if (moreB) load_record<G>(rp + REC, ca0, ca1, wB0, wB1);
+            fma_block<G, P>(acc, wA0, x0);
+            fma_block<G, P>(acc, wA1, x1);
+            if (!moreB) break;
+            load_x<XT, P>(xs + cb0 * ROWB, x0);
+            load_x<XT, P>(xs + cb1 * ROWB, x1);
+            const bool moreA = rp + 2 * REC < re;
+            if (moreA) load_record<G>(rp + 2 * REC, cb0, cb1, wA0, wA1);
+            fma_block<G, P>(acc, wB0, x0);
+            fma_block<G, P>(acc, wB1, x1);
+            if (!moreA) break;
+            load_x<XT, P>(xs + ca0 * ROWB, x0);
+            load_x<XT, P>(xs + ca1 * ROWB, x1);
             rp += 2 * REC;
         }
     } else {
@@ -350,7 +392,7 @@ __device__ __forceinline__ void produce(const ConvArgs& a, unsigned char* smem, 
             src[i] = static_cast<const unsigned char*>(a.x) + ((size_t)n * a.cin * a.hw + p) * SZ;
         }
         const int* slice = a.slice + rg * a.nch;
-        const int* rowoff = a.rowoff + (size_t)rg * a.nch * (a.rpg + 1);
+        const int* rowoff = a.rowoff + (size_t)rg * a.nch * a.ros;
 
         for (int k = 0; k < a.nch; ++k, ++kk) {
             const int s = kk % S;
@@ -388,13 +430,87 @@ __device__ __forceinline__ void produce(const ConvArgs& a, unsigned char* smem, 
             const int n16 = __ldg(slice + k + 1) - r0;
             const unsigned char* rsrc = a.rec + (size_t)r0 * 16;
             for (int i = lane; i < n16; i += 32) cp_async_16(st + a.off_rec + i * 16, rsrc + (size_t)i * 16);
-            const int* osrc = rowoff + (size_t)k * (a.rpg + 1);
+            const int* osrc = rowoff + (size_t)k * a.ros;
             for (int i = lane; i <= a.rpg; i += 32) cp_async_4(st + a.off_rowoff + i * 4, osrc + i);
             if constexpr (LDB == 2) __threadfence_block();
             mbar_arrive_on_copies(smem_u32 + 8 * s);      // "full" completes when all 32 lanes' copies land
         }
     }
     cp_async_wait_all();
+}
+
+// ---- producer, bulk-copy flavour ---------------------------------------------------------------
+// Used when every (image, channel) row of X starts on a 16-byte boundary and is a multiple of 16
+// bytes long.  One bulk copy moves a whole run of consecutive pixels of one channel (a tile row,
+// split where the tile crosses from one image into the next); the lanes of the producer warp
+// share the channel rows of the chunk.  Lane 0 announces the chunk's byte count on the "full"
+// mbarrier, which completes when all of them have landed.
+template <typename XT, int G, int P>
+__device__ __forceinline__ void produce_bulk(const ConvArgs& a, unsigned char* smem, int lane)
+{
+    constexpr int T = 32 * P;
+    constexpr int SZ = (int)sizeof(XT);
+    constexpr int ROWB = T * SZ;
+    const size_t ch_bytes = (size_t)a.hw * SZ;
+    const uint32_t smem_u32 = (uint32_t)__cvta_generic_to_shared(smem);
+    const uint32_t ring = smem_u32 + 16 * kMaxStages;
+    const int S = a.stages;
+    const int items = a.n_tiles * a.n_rg;
+    int kk = 0;
+
+    for (int item = blockIdx.x; item < items; item += gridDim.x) {
+        const int tile = item / a.n_rg;
+        const int rg = item - tile * a.n_rg;
+        const int q0 = tile * T;
+        const int vt = min(T, a.q_total - q0);          // valid pixels of this tile
+        const int n0 = q0 / a.hw;
+        const int p0 = q0 - n0 * a.hw;
+        const unsigned char* xbase = static_cast<const unsigned char*>(a.x) + ((size_t)n0 * a.cin * a.hw + p0) * SZ;
+        const int* slice = a.slice + rg * a.nch;
+        const int* rowoff = a.rowoff + (size_t)rg * a.nch * a.ros;
+
+        for (int k = 0; k < a.nch; ++k, ++kk) {
+            const int s = kk % S;
+            if (kk >= S) {
+                if (!mbar_wait(smem_u32 + 8 * kMaxStages + 8 * s, ((kk / S) - 1) & 1)) {
+                    if (lane == 0) atomicExch(a.err, kErrEmptyWait);
+                    goto drain;
+                }
+            }
+            {
+                const uint32_t st = ring + s * a.stage_bytes;
+                const uint32_t bar = smem_u32 + 8 * s;
+                const int cbase = k * a.kc;
+                const int nrows = min(a.kc, a.cin - cbase);
+                const int r0 = __ldg(slice + k);
+                const int rbytes = (__ldg(slice + k + 1) - r0) * 16;
+                if (lane == 0) mbar_arrive_expect_tx(bar, (uint32_t)(nrows * vt * SZ + rbytes + a.ros * 4));
+                __syncwarp();
+                // X: channel rows lane, lane+32, ...; each row is one copy per image it touches
+                for (int c = lane; c < nrows; c += 32) {
+                    const unsigned char* src = xbase + (size_t)(cbase + c) * ch_bytes;
+                    uint32_t dst = st + c * ROWB;
+                    int left = vt, p = p0;
+                    while (left > 0) {
+                        const int len = min(a.hw - p, left);
+                        bulk_copy_g2s(dst, src, (uint32_t)(len * SZ), bar);
+                        dst += len * SZ;
+                        // next image: same channel, pixel 0
+                        src += (size_t)len * SZ + (size_t)(a.cin - 1) * ch_bytes;
+                        left -= len;
+                        p = 0;
+                    }
+                }
+                if (lane == 0 && rbytes > 0) bulk_copy_g2s(st + a.off_rec, a.rec + (size_t)r0 * 16, (uint32_t)rbytes, bar);
+                if (lane == 1)
+                    bulk_copy_g2s(st + a.off_rowoff, rowoff + (size_t)k * a.ros, (uint32_t)(a.ros * 4), bar);
+            }
+        }
+    }
+drain:
+    // Do not leave while copies of this warp may still be landing: wait (bounded) for the last
+    // fills of every stage.
+    for (int j = max(0, kk - S); j < kk; ++j) mbar_wait(smem_u32 + 8 * (j % S), (j / S) & 1);
 }
 
 template <typename XT, int G, int P, int RW, int NW, int MINB>
@@ -404,8 +520,9 @@ __global__ void __launch_bounds__((NW + 1) * 32, MINB) spconv1x1_kernel(const Co
     constexpr int SZ = (int)sizeof(XT);
     constexpr int VG = (P * SZ >= 16) ? 16 / SZ : P;  // elements per shared-memory vector load
     constexpr int NG = P / VG;                        // vector groups per lane
-    constexpr int ROWB = T * SZ;                      // bytes of one staged channel row
-    constexpr int REC = record_bytes(G);
+    // registers a thread may use, and whether the deep software pipeline fits in them
+    constexpr int kRegCap = 65536 / ((NW + 1) * 32 * MINB) > 255 ? 255 : 65536 / ((NW + 1) * 32 * MINB) / 8 * 8;
+    constexpr bool kDeep = RW * G * P + 4 * G + 4 * P + 28 <= kRegCap;
 
     extern __shared__ __align__(16) unsigned char smem[];   // [full[8] | empty[8] | ring]
 
@@ -417,13 +534,17 @@ __global__ void __launch_bounds__((NW + 1) * 32, MINB) spconv1x1_kernel(const Co
 
     if (tid == 0) {
         for (int s = 0; s < S; ++s) {
-            mbar_init(smem_u32 + 8 * s, 32);                        // full: the 32 producer lanes
+            mbar_init(smem_u32 + 8 * s, a.bulk ? 1 : 32);           // full: one announcing arrival, or the 32 producer lanes
             mbar_init(smem_u32 + 8 * kMaxStages + 8 * s, NW);       // empty: one arrival per consumer warp
         }
     }
     __syncthreads();
 
     if (warp == NW) {   // ---- producer warp -------------------------------------------------
+        if (a.bulk) {
+            produce_bulk<XT, G, P>(a, smem, lane);
+            return;
+        }
         switch (a.ld_bytes) {
             case 16: produce<XT, G, P, 16>(a, smem, lane); break;
             case 8: produce<XT, G, P, 8>(a, smem, lane); break;
@@ -476,7 +597,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, MINB) spconv1x1_kernel(const Co
                 if (lrow[s] >= a.rpg) continue;
                 const unsigned char* rp = recs + roff[lrow[s]] * 16;
                 const unsigned char* re = recs + roff[lrow[s] + 1] * 16;
-                if (rp < re) consume_segment<XT, G, P>(acc[s], xs, rp, re);
+                if (rp < re) consume_segment<XT, G, P, kDeep>(acc[s], xs, rp, re);
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32 + 8 * kMaxStages + 8 * st);   // stage st may be refilled

@@ -79,7 +79,9 @@ void build_schedule(const alcs_packed& p, int kc, int n_rg, bool with_records, S
     }
 
     out.h_slice.assign((size_t)n_rg * nch + 1, 0);
-    out.h_rowoff.assign((size_t)n_rg * nch * (rpg + 1), 0);
+    const int ros = (rpg + 1 + 3) & ~3;          // padded so that one row of offsets is a multiple of 16 bytes
+    out.ros = ros;
+    out.h_rowoff.assign((size_t)n_rg * nch * ros, 0);
     out.h_rec.clear();
     std::vector<int> cursor(R);
     int rec_count = 0, wcap = 0;
@@ -102,7 +104,7 @@ void build_schedule(const alcs_packed& p, int kc, int n_rg, bool with_records, S
         }
         for (int c = 0; c < nch; ++c) {
             out.h_slice[(size_t)rg * nch + c] = rec_count;
-            int* roff = &out.h_rowoff[((size_t)rg * nch + c) * (rpg + 1)];
+            int* roff = &out.h_rowoff[((size_t)rg * nch + c) * ros];
             const int lim = (c + 1) * kc;
             const int c0 = c * kc;
             int local = 0;

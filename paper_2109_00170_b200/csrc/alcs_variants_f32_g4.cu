@@ -5,6 +5,11 @@
 namespace alcs {
 
 static const KernelVariant kTable[] = {
+    ALCS_VARIANT(float, 0, 4, 8, 1, 23, 1),
+    ALCS_VARIANT(float, 0, 4, 8, 1, 19, 1),
+    ALCS_VARIANT(float, 0, 4, 4, 2, 23, 1),
+    ALCS_VARIANT(float, 0, 4, 8, 2, 15, 1),
+    ALCS_VARIANT(float, 0, 4, 8, 4, 11, 1),
     //           XT   f16  G  P RW  NW MINB
     ALCS_VARIANT(float, 0, 4, 8, 1, 7, 1),
     ALCS_VARIANT(float, 0, 4, 8, 1, 11, 1),

@@ -208,6 +208,15 @@ ALCS_API int alcs_spconv1x1_tune(alcs_packed* w, const void* x, void* y, int n, 
                         alcs_launch_cfg* best);
 
 /*
+ * alcs_spconv1x1_set_cfg: make later alcs_spconv1x1 / alcs_stack_create calls with this
+ * (n, h, wd, flags) use the given configuration, e.g. one that alcs_spconv1x1_tune found in an
+ * earlier process.  Fields left 0 are chosen by the library.  Host only; returns UNSUPPORTED if no
+ * compiled kernel variant fits it.
+ */
+ALCS_API int alcs_spconv1x1_set_cfg(alcs_packed* w, int n, int h, int wd, unsigned flags,
+                                    const alcs_launch_cfg* cfg);
+
+/*
  * alcs_spconv1x1_host: the same operation on HOST buffers x_host / y_host / bias_host, staged
  * through a caller-provided device workspace of at least alcs_spconv1x1_host_workspace() bytes
  * (256-byte aligned).  Enqueues H2D copies, the kernel and the D2H copy on cuda_stream and

@@ -25,7 +25,7 @@ EXPORTS = ["alcs_strerror", "alcs_last_cuda_error", "alcs_version", "alcs_pack",
            "alcs_packed_view", "alcs_packed_serialize", "alcs_packed_deserialize",
            "alcs_packed_upload", "alcs_packed_status", "alcs_packed_free", "alcs_variant_count", "alcs_variant_get",
            "alcs_spconv1x1", "alcs_spconv1x1_cfg",
-           "alcs_spconv1x1_plan", "alcs_spconv1x1_tune", "alcs_spconv1x1_host_workspace",
+           "alcs_spconv1x1_plan", "alcs_spconv1x1_tune", "alcs_spconv1x1_set_cfg", "alcs_spconv1x1_host_workspace",
            "alcs_spconv1x1_host", "alcs_stack_create", "alcs_stack_run", "alcs_stack_destroy"]
 
 
@@ -82,6 +82,7 @@ def lib():
     L.alcs_spconv1x1_cfg.argtypes = [vp, vp, vp, i, i, i, vp, u, C.POINTER(LaunchCfg), vp]
     L.alcs_spconv1x1_plan.argtypes = [vp, i, i, i, u, C.POINTER(LaunchCfg)]
     L.alcs_spconv1x1_tune.argtypes = [vp, vp, vp, i, i, i, vp, u, vp, C.POINTER(LaunchCfg)]
+    L.alcs_spconv1x1_set_cfg.argtypes = [vp, i, i, i, u, C.POINTER(LaunchCfg)]
     L.alcs_spconv1x1_host_workspace.argtypes = [vp, i, i, i, u]
     L.alcs_spconv1x1_host_workspace.restype = sz
     L.alcs_spconv1x1_host.argtypes = [vp, vp, vp, i, i, i, vp, u, vp, sz, vp]
@@ -265,6 +266,12 @@ def alcs_spconv1x1_tune(w: Packed, x, y, n: int, h: int, wd: int, bias=None, fla
     _check(lib().alcs_spconv1x1_tune(w.handle, _addr(x), _addr(y), n, h, wd, _addr(bias), flags,
                                      _stream(stream), C.byref(c)), "alcs_spconv1x1_tune")
     return c.as_dict()
+
+
+def alcs_spconv1x1_set_cfg(w: Packed, n: int, h: int, wd: int, flags: int, cfg) -> None:
+    """Use `cfg` (a dict or LaunchCfg, e.g. from a tuning cache) for later calls with this shape."""
+    c = _cfg(cfg)
+    _check(lib().alcs_spconv1x1_set_cfg(w.handle, n, h, wd, flags, C.byref(c)), "alcs_spconv1x1_set_cfg")
 
 
 def alcs_spconv1x1_host_workspace(w: Packed, n: int, h: int, wd: int, flags: int = 0) -> int:

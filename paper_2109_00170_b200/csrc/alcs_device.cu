@@ -628,6 +628,26 @@ ALCS_API int alcs_spconv1x1_tune(alcs_packed* w, const void* x, void* y, int n, 
     return rc;
 }
 
+ALCS_API int alcs_spconv1x1_set_cfg(alcs_packed* w, int n, int h, int wd, unsigned flags,
+                                    const alcs_launch_cfg* cfg)
+{
+    if (!w || !cfg || n < 0 || h < 0 || wd < 0) return ALCS_ERR_INVALID_ARG;
+    if (flags & ~(ALCS_RELU | ALCS_Y_F32)) return ALCS_ERR_INVALID_ARG;
+    if (w->device < 0) return ALCS_ERR_STATE;
+    const long long q = (long long)n * h * wd;
+    if ((long long)h * wd > (1ll << 30) || q > (1ll << 30)) return ALCS_ERR_SHAPE;
+    Plan plan;
+    const int rc = cfg_to_plan(w, std::max(1ll, q), h * wd, cfg, &plan);
+    if (rc) return rc;
+    alcs_launch_cfg full;
+    plan_to_cfg(plan, &full);
+    std::lock_guard<std::mutex> lk(w->mu);
+    const alcs::ShapeKey key{n, h, wd, flags};
+    w->tuned[key] = full;
+    w->plan_cache[key] = plan;
+    return ALCS_OK;
+}
+
 ALCS_API size_t alcs_spconv1x1_host_workspace(const alcs_packed* w, int n, int h, int wd, unsigned flags)
 {
     if (!w || n < 0 || h < 0 || wd < 0) return 0;

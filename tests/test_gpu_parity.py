@@ -211,6 +211,24 @@ def test_tuned_configuration_is_used_and_correct(alcs):
     assert_parity(Y, Yref, A, "f32")
 
 
+def test_set_cfg_is_used_by_later_calls(alcs):
+    """A configuration applied with alcs_spconv1x1_set_cfg (e.g. from a tuning cache) becomes the
+    plan of later automatic calls for that shape, and the result is still right."""
+    W, M, X, b = _rand(26, 4, 128, 128, 196, 4, 0.25)
+    p = alcs.alcs_packed_upload(alcs.alcs_pack(W, M, 4), 0)
+    cfg = dict(pixels_per_lane=4, rows_per_warp=2, warps=7, chunk_channels=32, stages=3, row_groups=0,
+               min_blocks=0, copy_mode=1)
+    alcs.alcs_spconv1x1_set_cfg(p, 4, 14, 14, alcs.ALCS_RELU, cfg)
+    plan = alcs.alcs_spconv1x1_plan(p, 4, 14, 14, alcs.ALCS_RELU)
+    for k in ("pixels_per_lane", "rows_per_warp", "warps", "chunk_channels", "stages", "copy_mode"):
+        assert plan[k] == cfg[k]
+    Yref, A = oracle.conv1x1(W, M, X, b, True, 4, want_scale=True)
+    assert_parity(run_gpu(alcs, W, M, X, b, True, 4, h=14, wd=14, packed=p), Yref, A, "f32")
+    with pytest.raises(alcs.AlcsError) as e:
+        alcs.alcs_spconv1x1_set_cfg(p, 4, 14, 14, 0, dict(pixels_per_lane=5))
+    assert e.value.status == alcs.ALCS_ERR_UNSUPPORTED
+
+
 def test_host_buffer_entry_point(alcs):
     import torch
     W, M, X, b = _rand(23, 4, 64, 128, 196, 4, 0.3)

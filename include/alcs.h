@@ -159,14 +159,16 @@ ALCS_API void alcs_packed_free(alcs_packed* p);
  *   min_blocks        thread blocks per SM the kernel is compiled for (1 or 2)
  *   copy_mode         how X tiles reach shared memory: 1 = per-lane cp.async, 2 = bulk (TMA) copies
  *                     of whole pixel runs (needs 16-byte aligned rows; otherwise 1 is used)
+ *   producer_warps    warps of the thread block that only move data (1..4)
  */
 typedef struct {
-    int pixels_per_lane, rows_per_warp, warps, chunk_channels, stages, row_groups, min_blocks, copy_mode;
+    int pixels_per_lane, rows_per_warp, warps, chunk_channels, stages, row_groups, min_blocks, copy_mode,
+        producer_warps;
 } alcs_launch_cfg;
 
 /*
  * Introspection of the compiled kernel variants (host only): alcs_variant_count() entries, each a
- * (dtype, g, pixels_per_lane, rows_per_warp, warps, min_blocks) combination that
+ * (dtype, g, pixels_per_lane, rows_per_warp, warps, min_blocks, producer_warps) combination that
  * alcs_spconv1x1_cfg accepts; the other fields of *cfg are set to 0.
  */
 ALCS_API int alcs_variant_count(void);

@@ -189,7 +189,7 @@ double model_cost(const alcs_packed* w, const KernelVariant& v, const Schedule& 
 int occupancy_of(const VariantInfo& vi, size_t smem)
 {
     int occ = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, vi.v.fn, (vi.v.nw + 1) * 32, smem) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, vi.v.fn, (vi.v.nw + vi.v.npw) * 32, smem) != cudaSuccess) {
         (void)cudaGetLastError();
         return 0;
     }
@@ -272,6 +272,7 @@ void plan_to_cfg(const Plan& p, alcs_launch_cfg* c)
     c->row_groups = p.n_rg;
     c->min_blocks = v.minb;
     c->copy_mode = p.bulk ? 2 : 1;
+    c->producer_warps = v.npw;
 }
 
 // Resolve a (possibly partial) configuration into a concrete plan.
@@ -287,6 +288,7 @@ int cfg_to_plan(const alcs_packed* w, long long q, int hw, const alcs_launch_cfg
         if (c->rows_per_warp && c->rows_per_warp != v.rw) return false;
         if (c->warps && c->warps != v.nw) return false;
         if (c->min_blocks && c->min_blocks != v.minb) return false;
+        if (c->producer_warps && c->producer_warps != v.npw) return false;
         if (c->chunk_channels && std::min(c->chunk_channels, w->cin) != p.kc) return false;
         if (c->stages && c->stages != p.stages) return false;
         if (c->copy_mode && (c->copy_mode == 2) != (p.bulk == 1)) return false;
@@ -383,7 +385,7 @@ int launch_plan(const alcs_packed* w, const Plan& p, const void* x, void* y, int
     // persistent thread blocks: as many as can be resident, each walks items with that stride
     const long long grid = std::min<long long>(items, (long long)di.sms * std::max(1, p.occ));
     void* args[] = {&a};
-    ALCS_CUDA(cudaLaunchKernel(v.fn, dim3((unsigned)grid), dim3((v.nw + 1) * 32), args, p.smem, st));
+    ALCS_CUDA(cudaLaunchKernel(v.fn, dim3((unsigned)grid), dim3((v.nw + v.npw) * 32), args, p.smem, st));
     return ALCS_OK;
 }
 
@@ -400,9 +402,9 @@ int resolve_plan(const alcs_packed* w, int n, int h, int wd, unsigned flags, lon
 {
     alcs::ShapeKey key{n, h, wd, flags};
     if (cfg) {
-        const int c[8] = {cfg->pixels_per_lane, cfg->rows_per_warp, cfg->warps, cfg->chunk_channels,
-                          cfg->stages, cfg->row_groups, cfg->min_blocks, cfg->copy_mode};
-        for (int i = 0; i < 8; ++i) key.c[i] = c[i];
+        const int c[9] = {cfg->pixels_per_lane, cfg->rows_per_warp, cfg->warps, cfg->chunk_channels,
+                          cfg->stages, cfg->row_groups, cfg->min_blocks, cfg->copy_mode, cfg->producer_warps};
+        for (int i = 0; i < 9; ++i) key.c[i] = c[i];
     }
     {
         std::lock_guard<std::mutex> lk(w->mu);
@@ -509,6 +511,7 @@ ALCS_API int alcs_variant_get(int index, alcs_dtype* dt, int* g, alcs_launch_cfg
         cfg->warps = v.nw;
         cfg->min_blocks = v.minb;
         cfg->copy_mode = 0;
+        cfg->producer_warps = v.npw;
     }
     return ALCS_OK;
 }
@@ -566,7 +569,7 @@ ALCS_API int alcs_spconv1x1_tune(alcs_packed* w, const void* x, void* y, int n, 
     std::vector<Plan> all;
     rc = enumerate_plans(w, q, h * wd, all);
     if (rc) return rc;
-    const size_t max_try = 160;
+    const size_t max_try = 400;
     if (all.size() > max_try) all.resize(max_try);
     // a buffer larger than L2, rewritten before every timed launch so that each candidate is
     // timed with cold caches, as it will run inside a network

@@ -67,11 +67,11 @@ struct Plan {
 struct ShapeKey {
     int n, h, wd;
     unsigned flags;
-    int c[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    int c[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
     bool operator<(const ShapeKey& o) const {
         if (std::tie(n, h, wd, flags) != std::tie(o.n, o.h, o.wd, o.flags))
             return std::tie(n, h, wd, flags) < std::tie(o.n, o.h, o.wd, o.flags);
-        for (int i = 0; i < 8; ++i)
+        for (int i = 0; i < 9; ++i)
             if (c[i] != o.c[i]) return c[i] < o.c[i];
         return false;
     }

@@ -9,7 +9,7 @@
 //   thread block = persistent: walks items blockIdx.x, blockIdx.x + gridDim.x, ...
 //   consumer warp= RW block rows at a time, all T pixels of the tile
 //   lane         = P pixels of each of those rows: G*P fp32 accumulators per row in registers
-//   producer warp= one extra warp that only moves data
+//   producer warps= one or more extra warps that only move data
 //
 // The input channels are walked in chunks of KC channels.  For each (item, chunk) the producer
 // warp copies, with cp.async, the X tile ([KC][T] elements) and the row group's slice of the
@@ -172,9 +172,10 @@ struct XVec<__half, 4> {
     }
 };
 
-// The P pixels a lane owns of one staged channel row: P/VG vector loads, 32*VG elements apart.
+// The P pixels a lane owns of one staged channel row, as P/2 adjacent pairs: P/VG vector loads,
+// 32*VG elements apart.
 template <typename XT, int P>
-__device__ __forceinline__ void load_x(const unsigned char* p, float (&x)[P])
+__device__ __forceinline__ void load_x(const unsigned char* p, float2 (&x)[P / 2])
 {
     constexpr int SZ = (int)sizeof(XT);
     constexpr int VG = (P * SZ >= 16) ? 16 / SZ : P;
@@ -183,7 +184,7 @@ __device__ __forceinline__ void load_x(const unsigned char* p, float (&x)[P])
         float v[VG];
         XVec<XT, VG>::load(p + gi * (32 * VG * SZ), v);
 #pragma unroll
-        for (int t = 0; t < VG; ++t) x[gi * VG + t] = v[t];
+        for (int t = 0; t < VG / 2; ++t) x[gi * (VG / 2) + t] = make_float2(v[2 * t], v[2 * t + 1]);
     }
 }
 
@@ -226,21 +227,26 @@ __device__ __forceinline__ void load_w(const unsigned char* p, float (&w)[G])
     }
 }
 
-// acc[j][t] += w[j] * x[t]: the G x P outer-product update of one block.
+// acc[j][t] += w[j] * x[t]: the G x P outer-product update of one block, two pixels per
+// instruction with the packed fp32 FMA of sm_100 (each half is an IEEE fused multiply-add, so
+// the result equals the scalar fmaf bit for bit).  Fewer issue slots per FMA leave room for the
+// shared-memory loads and the loop bookkeeping.
 template <int G, int P>
-__device__ __forceinline__ void fma_block(float (&acc)[G][P], const float (&w)[G], const float (&x)[P])
+__device__ __forceinline__ void fma_block(float2 (&acc)[G][P / 2], const float (&w)[G], const float2 (&x)[P / 2])
 {
 #pragma unroll
-    for (int j = 0; j < G; ++j)
+    for (int j = 0; j < G; ++j) {
+        const float2 w2 = make_float2(w[j], w[j]);
 #pragma unroll
-        for (int t = 0; t < P; ++t) acc[j][t] = fmaf(w[j], x[t], acc[j][t]);
+        for (int t = 0; t < P / 2; ++t) acc[j][t] = __ffma2_rn(w2, x[t], acc[j][t]);
+    }
 }
 
 // Multiply-accumulate one (block row, chunk) segment of pair records into the lane's G x P
 // accumulators.  xs points at this lane's first pixel vector of the staged X tile; [rp, re) is the
 // segment in shared memory.
 template <typename XT, int G, int P, bool DEEP>
-__device__ __forceinline__ void consume_segment(float (&acc)[G][P], const unsigned char* xs,
+__device__ __forceinline__ void consume_segment(float2 (&acc)[G][P / 2], const unsigned char* xs,
                                                 const unsigned char* rp, const unsigned char* re)
 {
     constexpr int ROWB = 32 * P * (int)sizeof(XT);
@@ -255,7 +261,7 @@ __device__ __forceinline__ void consume_segment(float (&acc)[G][P], const unsign
     int ca0 = lead.x, ca1 = lead.y, cb0 = 0, cb1 = 0;
     if constexpr (G <= 4 && DEEP) {
         float wA0[G], wA1[G], wB0[G], wB1[G];
-        float xA0[P], xA1[P], xB0[P], xB1[P];
+        float2 xA0[P / 2], xA1[P / 2], xB0[P / 2], xB1[P / 2];
         load_record<G>(rp, cb0, cb1, wA0, wA1);
         load_x<XT, P>(xs + ca0 * ROWB, xA0);
         load_x<XT, P>(xs + ca1 * ROWB, xA1);
@@ -285,7 +291,7 @@ __device__ __forceinline__ void consume_segment(float (&acc)[G][P], const unsign
         // ahead (two alternating weight sets); the X vectors of a pair are loaded when the
         // previous pair's FMAs have been issued, and other warps cover that latency.
         float wA0[G], wA1[G], wB0[G], wB1[G];
-        float x0[P], x1[P];
+        float2 x0[P / 2], x1[P / 2];
         load_record<G>(rp, cb0, cb1, wA0, wA1);
         load_x<XT, P>(xs + ca0 * ROWB, x0);
         load_x<XT, P>(xs + ca1 * ROWB, x1);
@@ -311,7 +317,8 @@ __device__ __forceinline__ void consume_segment(float (&acc)[G][P], const unsign
         // fill most of the register file, so nothing but the next pair's columns is
         // fetched ahead; the weights of each block are loaded just before its FMAs.
         while (true) {
-            float x0[P], x1[P], w[G];
+            float2 x0[P / 2], x1[P / 2];
+            float w[G];
             load_x<XT, P>(xs + ca0 * ROWB, x0);
             load_x<XT, P>(xs + ca1 * ROWB, x1);
             const int2 nx = *reinterpret_cast<const int2*>(rp);
@@ -358,7 +365,7 @@ __device__ __forceinline__ void store_one(YT* p, float v)
 // LDB = bytes per X copy.  Each lane owns NCOL fixed pixel vectors of the tile and walks the
 // channels of the chunk, so its source pointers are computed once per item.
 template <typename XT, int G, int P, int LDB>
-__device__ __forceinline__ void produce(const ConvArgs& a, unsigned char* smem, int lane)
+__device__ __forceinline__ void produce(const ConvArgs& a, unsigned char* smem, int lane, int pw, int npw)
 {
     constexpr int T = 32 * P;
     constexpr int SZ = (int)sizeof(XT);
@@ -413,14 +420,14 @@ __device__ __forceinline__ void produce(const ConvArgs& a, unsigned char* smem, 
                 const unsigned char* sp = src[i] + (size_t)cbase * ch_bytes;
                 const uint32_t dp = st + (vlane + 32 * i) * LDB;
                 if constexpr (LDB == 16) {
-                    for (int c = rlane; c < nrows; c += RP) cp_async_16(dp + c * ROWB, sp + c * ch_bytes);
+                    for (int c = rlane + pw * RP; c < nrows; c += RP * npw) cp_async_16(dp + c * ROWB, sp + c * ch_bytes);
                 } else if constexpr (LDB == 8) {
-                    for (int c = rlane; c < nrows; c += RP) cp_async_8(dp + c * ROWB, sp + c * ch_bytes);
+                    for (int c = rlane + pw * RP; c < nrows; c += RP * npw) cp_async_8(dp + c * ROWB, sp + c * ch_bytes);
                 } else if constexpr (LDB == 4) {
-                    for (int c = rlane; c < nrows; c += RP) cp_async_4(dp + c * ROWB, sp + c * ch_bytes);
+                    for (int c = rlane + pw * RP; c < nrows; c += RP * npw) cp_async_4(dp + c * ROWB, sp + c * ch_bytes);
                 } else {   // 2-byte elements at odd alignment: plain loads and shared-memory stores
                     unsigned char* d = smem + 16 * kMaxStages + s * a.stage_bytes + (vlane + 32 * i) * LDB;
-                    for (int c = rlane; c < nrows; c += RP)
+                    for (int c = rlane + pw * RP; c < nrows; c += RP * npw)
                         *reinterpret_cast<unsigned short*>(d + c * ROWB) =
                             __ldg(reinterpret_cast<const unsigned short*>(sp + c * ch_bytes));
                 }
@@ -429,11 +436,11 @@ __device__ __forceinline__ void produce(const ConvArgs& a, unsigned char* smem, 
             const int r0 = __ldg(slice + k);
             const int n16 = __ldg(slice + k + 1) - r0;
             const unsigned char* rsrc = a.rec + (size_t)r0 * 16;
-            for (int i = lane; i < n16; i += 32) cp_async_16(st + a.off_rec + i * 16, rsrc + (size_t)i * 16);
+            for (int i = lane + 32 * pw; i < n16; i += 32 * npw) cp_async_16(st + a.off_rec + i * 16, rsrc + (size_t)i * 16);
             const int* osrc = rowoff + (size_t)k * a.ros;
-            for (int i = lane; i <= a.rpg; i += 32) cp_async_4(st + a.off_rowoff + i * 4, osrc + i);
+            for (int i = lane + 32 * pw; i <= a.rpg; i += 32 * npw) cp_async_4(st + a.off_rowoff + i * 4, osrc + i);
             if constexpr (LDB == 2) __threadfence_block();
-            mbar_arrive_on_copies(smem_u32 + 8 * s);      // "full" completes when all 32 lanes' copies land
+            mbar_arrive_on_copies(smem_u32 + 8 * s);      // "full" completes when all producer lanes' copies land
         }
     }
     cp_async_wait_all();
@@ -446,7 +453,7 @@ __device__ __forceinline__ void produce(const ConvArgs& a, unsigned char* smem, 
 // share the channel rows of the chunk.  Lane 0 announces the chunk's byte count on the "full"
 // mbarrier, which completes when all of them have landed.
 template <typename XT, int G, int P>
-__device__ __forceinline__ void produce_bulk(const ConvArgs& a, unsigned char* smem, int lane)
+__device__ __forceinline__ void produce_bulk(const ConvArgs& a, unsigned char* smem, int lane, int pw, int npw)
 {
     constexpr int T = 32 * P;
     constexpr int SZ = (int)sizeof(XT);
@@ -484,10 +491,10 @@ __device__ __forceinline__ void produce_bulk(const ConvArgs& a, unsigned char* s
                 const int nrows = min(a.kc, a.cin - cbase);
                 const int r0 = __ldg(slice + k);
                 const int rbytes = (__ldg(slice + k + 1) - r0) * 16;
-                if (lane == 0) mbar_arrive_expect_tx(bar, (uint32_t)(nrows * vt * SZ + rbytes + a.ros * 4));
+                if (lane == 0 && pw == 0) mbar_arrive_expect_tx(bar, (uint32_t)(nrows * vt * SZ + rbytes + a.ros * 4));
                 __syncwarp();
                 // X: channel rows lane, lane+32, ...; each row is one copy per image it touches
-                for (int c = lane; c < nrows; c += 32) {
+                for (int c = lane + 32 * pw; c < nrows; c += 32 * npw) {
                     const unsigned char* src = xbase + (size_t)(cbase + c) * ch_bytes;
                     uint32_t dst = st + c * ROWB;
                     int left = vt, p = p0;
@@ -501,8 +508,8 @@ __device__ __forceinline__ void produce_bulk(const ConvArgs& a, unsigned char* s
                         p = 0;
                     }
                 }
-                if (lane == 0 && rbytes > 0) bulk_copy_g2s(st + a.off_rec, a.rec + (size_t)r0 * 16, (uint32_t)rbytes, bar);
-                if (lane == 1)
+                if (lane == 0 && pw == 0 && rbytes > 0) bulk_copy_g2s(st + a.off_rec, a.rec + (size_t)r0 * 16, (uint32_t)rbytes, bar);
+                if (lane == 1 && pw == 0)
                     bulk_copy_g2s(st + a.off_rowoff, rowoff + (size_t)k * a.ros, (uint32_t)(a.ros * 4), bar);
             }
         }
@@ -513,15 +520,17 @@ drain:
     for (int j = max(0, kk - S); j < kk; ++j) mbar_wait(smem_u32 + 8 * (j % S), (j / S) & 1);
 }
 
-template <typename XT, int G, int P, int RW, int NW, int MINB>
-__global__ void __launch_bounds__((NW + 1) * 32, MINB) spconv1x1_kernel(const ConvArgs a)
+template <typename XT, int G, int P, int RW, int NW, int MINB, int NPW>
+__global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_kernel(const ConvArgs a)
 {
     constexpr int T = 32 * P;                         // pixels per tile
     constexpr int SZ = (int)sizeof(XT);
     constexpr int VG = (P * SZ >= 16) ? 16 / SZ : P;  // elements per shared-memory vector load
     constexpr int NG = P / VG;                        // vector groups per lane
     // registers a thread may use, and whether the deep software pipeline fits in them
-    constexpr int kRegCap = 65536 / ((NW + 1) * 32 * MINB) > 255 ? 255 : 65536 / ((NW + 1) * 32 * MINB) / 8 * 8;
+    // (the register file is handed out as if the block had a multiple of 128 threads)
+    constexpr int kThreadsAlloc = ((NW + NPW) * 32 + 127) / 128 * 128;
+    constexpr int kRegCap = 65536 / (kThreadsAlloc * MINB) > 255 ? 255 : 65536 / (kThreadsAlloc * MINB) / 8 * 8;
     constexpr bool kDeep = RW * G * P + 4 * G + 4 * P + 28 <= kRegCap;
 
     extern __shared__ __align__(16) unsigned char smem[];   // [full[8] | empty[8] | ring]
@@ -534,23 +543,24 @@ __global__ void __launch_bounds__((NW + 1) * 32, MINB) spconv1x1_kernel(const Co
 
     if (tid == 0) {
         for (int s = 0; s < S; ++s) {
-            mbar_init(smem_u32 + 8 * s, a.bulk ? 1 : 32);           // full: one announcing arrival, or the 32 producer lanes
+            mbar_init(smem_u32 + 8 * s, a.bulk ? 1 : 32 * NPW);     // full: one announcing arrival, or every producer lane
             mbar_init(smem_u32 + 8 * kMaxStages + 8 * s, NW);       // empty: one arrival per consumer warp
         }
     }
     __syncthreads();
 
-    if (warp == NW) {   // ---- producer warp -------------------------------------------------
+    if (warp >= NW) {   // ---- producer warps ------------------------------------------------
+        const int pw = warp - NW;
         if (a.bulk) {
-            produce_bulk<XT, G, P>(a, smem, lane);
+            produce_bulk<XT, G, P>(a, smem, lane, pw, NPW);
             return;
         }
         switch (a.ld_bytes) {
-            case 16: produce<XT, G, P, 16>(a, smem, lane); break;
-            case 8: produce<XT, G, P, 8>(a, smem, lane); break;
-            case 4: produce<XT, G, P, 4>(a, smem, lane); break;
+            case 16: produce<XT, G, P, 16>(a, smem, lane, pw, NPW); break;
+            case 8: produce<XT, G, P, 8>(a, smem, lane, pw, NPW); break;
+            case 4: produce<XT, G, P, 4>(a, smem, lane, pw, NPW); break;
             default:
-                if constexpr (SZ == 2) produce<XT, G, P, 2>(a, smem, lane);
+                if constexpr (SZ == 2) produce<XT, G, P, 2>(a, smem, lane, pw, NPW);
                 break;
         }
         return;
@@ -574,13 +584,13 @@ __global__ void __launch_bounds__((NW + 1) * 32, MINB) spconv1x1_kernel(const Co
             rowid[s] = lrow[s] < a.rpg ? __ldg(a.rowmap + rg * a.rpg + lrow[s]) : -1;
         }
 
-        float acc[RW][G][P];
+        float2 acc[RW][G][P / 2];
 #pragma unroll
         for (int s = 0; s < RW; ++s)
 #pragma unroll
             for (int j = 0; j < G; ++j)
 #pragma unroll
-                for (int e = 0; e < P; ++e) acc[s][j][e] = 0.0f;
+                for (int e = 0; e < P / 2; ++e) acc[s][j][e] = make_float2(0.0f, 0.0f);
 
         for (int k = 0; k < a.nch; ++k, ++kk) {
             const int st = kk % S;
@@ -628,7 +638,8 @@ __global__ void __launch_bounds__((NW + 1) * 32, MINB) spconv1x1_kernel(const Co
                         float v[VG];
 #pragma unroll
                         for (int t = 0; t < VG; ++t) {
-                            v[t] = acc[s][j][gi * VG + t] + bv;
+                            const float2 a2 = acc[s][j][(gi * VG + t) / 2];
+                            v[t] = (((gi * VG + t) & 1) ? a2.y : a2.x) + bv;
                             if (a.relu) v[t] = fmaxf(v[t], 0.0f);
                         }
                         if (a.st_vec) {
@@ -658,12 +669,13 @@ __global__ void __launch_bounds__((NW + 1) * 32, MINB) spconv1x1_kernel(const Co
 
 // One entry of the table of compiled kernel variants.
 struct KernelVariant {
-    int is_f16, g, p, rw, nw, minb;
+    int is_f16, g, p, rw, nw, minb, npw;
     const void* fn;
 };
 
-#define ALCS_VARIANT(XT, ISF16, G, P, RW, NW, MINB) \
-    {ISF16, G, P, RW, NW, MINB, (const void*)&spconv1x1_kernel<XT, G, P, RW, NW, MINB>}
+#define ALCS_VARIANT_P(XT, ISF16, G, P, RW, NW, MINB, NPW) \
+    {ISF16, G, P, RW, NW, MINB, NPW, (const void*)&spconv1x1_kernel<XT, G, P, RW, NW, MINB, NPW>}
+#define ALCS_VARIANT(XT, ISF16, G, P, RW, NW, MINB) ALCS_VARIANT_P(XT, ISF16, G, P, RW, NW, MINB, 1)
 
 // Defined one per translation unit, concatenated by alcs_device.cu.
 const KernelVariant* variants_f32_g4(int* n);

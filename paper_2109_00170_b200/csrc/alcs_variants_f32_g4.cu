@@ -5,36 +5,45 @@
 namespace alcs {
 
 static const KernelVariant kTable[] = {
-    ALCS_VARIANT(float, 0, 4, 8, 1, 23, 1),
-    ALCS_VARIANT(float, 0, 4, 8, 1, 19, 1),
-    ALCS_VARIANT(float, 0, 4, 4, 2, 23, 1),
-    ALCS_VARIANT(float, 0, 4, 8, 2, 15, 1),
-    ALCS_VARIANT(float, 0, 4, 8, 4, 11, 1),
-    //           XT   f16  G  P RW  NW MINB
-    ALCS_VARIANT(float, 0, 4, 8, 1, 7, 1),
-    ALCS_VARIANT(float, 0, 4, 8, 1, 11, 1),
-    ALCS_VARIANT(float, 0, 4, 8, 1, 13, 1),
-    ALCS_VARIANT(float, 0, 4, 8, 1, 15, 1),
-    ALCS_VARIANT(float, 0, 4, 8, 2, 7, 1),
-    ALCS_VARIANT(float, 0, 4, 8, 2, 11, 1),
-    ALCS_VARIANT(float, 0, 4, 8, 2, 13, 1),
-    ALCS_VARIANT(float, 0, 4, 8, 3, 7, 1),
-    ALCS_VARIANT(float, 0, 4, 8, 3, 11, 1),
-    ALCS_VARIANT(float, 0, 4, 8, 4, 7, 1),
-    ALCS_VARIANT(float, 0, 4, 8, 1, 7, 2),
-    ALCS_VARIANT(float, 0, 4, 4, 2, 7, 1),
-    ALCS_VARIANT(float, 0, 4, 4, 4, 7, 1),
-    ALCS_VARIANT(float, 0, 4, 4, 2, 11, 1),
-    ALCS_VARIANT(float, 0, 4, 4, 4, 11, 1),
-    ALCS_VARIANT(float, 0, 4, 4, 2, 15, 1),
-    ALCS_VARIANT(float, 0, 4, 4, 4, 15, 1),
-    ALCS_VARIANT(float, 0, 4, 4, 6, 7, 1),
-    ALCS_VARIANT(float, 0, 4, 4, 6, 11, 1),
-    ALCS_VARIANT(float, 0, 4, 4, 4, 7, 2),
-    ALCS_VARIANT(float, 0, 4, 4, 2, 7, 2),
-    ALCS_VARIANT(float, 0, 4, 16, 1, 7, 1),
-    ALCS_VARIANT(float, 0, 4, 16, 1, 11, 1),
-    ALCS_VARIANT(float, 0, 4, 16, 2, 7, 1),
+    //             XT   f16  G  P RW  NW MINB NPW
+    ALCS_VARIANT_P(float, 0, 4, 8, 1, 7, 1, 1),
+    ALCS_VARIANT_P(float, 0, 4, 8, 2, 7, 1, 1),
+    ALCS_VARIANT_P(float, 0, 4, 8, 3, 7, 1, 1),
+    ALCS_VARIANT_P(float, 0, 4, 8, 4, 7, 1, 1),
+    ALCS_VARIANT_P(float, 0, 4, 8, 4, 6, 1, 2),
+    ALCS_VARIANT_P(float, 0, 4, 8, 1, 7, 2, 1),
+    ALCS_VARIANT_P(float, 0, 4, 8, 1, 11, 1, 1),
+    ALCS_VARIANT_P(float, 0, 4, 8, 2, 11, 1, 1),
+    ALCS_VARIANT_P(float, 0, 4, 8, 3, 11, 1, 1),
+    ALCS_VARIANT_P(float, 0, 4, 8, 2, 10, 1, 2),
+    ALCS_VARIANT_P(float, 0, 4, 8, 3, 10, 1, 2),
+    ALCS_VARIANT_P(float, 0, 4, 8, 1, 15, 1, 1),
+    ALCS_VARIANT_P(float, 0, 4, 8, 2, 15, 1, 1),
+    ALCS_VARIANT_P(float, 0, 4, 8, 1, 14, 1, 2),
+    ALCS_VARIANT_P(float, 0, 4, 8, 2, 14, 1, 2),
+    ALCS_VARIANT_P(float, 0, 4, 8, 2, 13, 1, 3),
+    ALCS_VARIANT_P(float, 0, 4, 8, 1, 13, 1, 3),
+    ALCS_VARIANT_P(float, 0, 4, 8, 1, 19, 1, 1),
+    ALCS_VARIANT_P(float, 0, 4, 8, 1, 18, 1, 2),
+    ALCS_VARIANT_P(float, 0, 4, 4, 2, 7, 1, 1),
+    ALCS_VARIANT_P(float, 0, 4, 4, 4, 7, 1, 1),
+    ALCS_VARIANT_P(float, 0, 4, 4, 6, 7, 1, 1),
+    ALCS_VARIANT_P(float, 0, 4, 4, 4, 7, 2, 1),
+    ALCS_VARIANT_P(float, 0, 4, 4, 2, 7, 2, 1),
+    ALCS_VARIANT_P(float, 0, 4, 4, 4, 6, 2, 2),
+    ALCS_VARIANT_P(float, 0, 4, 4, 2, 11, 1, 1),
+    ALCS_VARIANT_P(float, 0, 4, 4, 4, 11, 1, 1),
+    ALCS_VARIANT_P(float, 0, 4, 4, 6, 11, 1, 1),
+    ALCS_VARIANT_P(float, 0, 4, 4, 4, 10, 1, 2),
+    ALCS_VARIANT_P(float, 0, 4, 4, 6, 10, 1, 2),
+    ALCS_VARIANT_P(float, 0, 4, 4, 2, 15, 1, 1),
+    ALCS_VARIANT_P(float, 0, 4, 4, 4, 15, 1, 1),
+    ALCS_VARIANT_P(float, 0, 4, 4, 4, 14, 1, 2),
+    ALCS_VARIANT_P(float, 0, 4, 4, 2, 23, 1, 1),
+    ALCS_VARIANT_P(float, 0, 4, 16, 1, 7, 1, 1),
+    ALCS_VARIANT_P(float, 0, 4, 16, 1, 11, 1, 1),
+    ALCS_VARIANT_P(float, 0, 4, 16, 2, 7, 1, 1),
+    ALCS_VARIANT_P(float, 0, 4, 16, 1, 10, 1, 2),
 };
 
 const KernelVariant* variants_f32_g4(int* n)

@@ -177,9 +177,13 @@ ALCS_API int alcs_variant_get(int index, alcs_dtype* dt, int* g, alcs_launch_cfg
 /*
  * alcs_spconv1x1: x device [n][cin][h*wd], y device [n][cout][h*wd], both contiguous NCHW of the
  * packed dtype (y fp32 if ALCS_Y_F32); bias device fp32 [cout] or NULL; flags = ALCS_RELU |
- * ALCS_Y_F32.  x and y must not overlap and must be aligned to their element size; 16-byte
- * aligned buffers with h*wd a multiple of 4 (fp32) or 8 (fp16) take the vectorised path, anything
- * else a slower element-wise path with identical results.  Enqueues one kernel on cuda_stream;
+ * ALCS_Y_F32.  x and y must not overlap and must be aligned to their element size.  16-byte
+ * aligned buffers with h*wd a multiple of 4 (fp32) or 8 (fp16) are used in place.  If the rows of
+ * x are not a multiple of 16 bytes long (h*wd = 49, ...) x is first repacked, by a small kernel on
+ * the same stream, into scratch memory owned by w (allocated or grown by the first call that
+ * needs it; n*cin*round_up(h*wd)*element bytes) and y is stored element by element; results are
+ * identical.  Because that scratch belongs to w, two such convolutions with the SAME w must not
+ * run concurrently on different streams.  Enqueues one kernel on cuda_stream;
  * no allocation and no synchronisation once this shape has been seen (see alcs_packed_upload).  n == 0 or h*wd == 0 is a successful no-op.
  * Errors: INVALID_ARG, SHAPE (n*channels*pixels beyond int32 tiles), UNSUPPORTED (g), STATE (not
  * uploaded / wrong current device), CUDA.

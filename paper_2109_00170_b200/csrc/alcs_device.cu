@@ -244,8 +244,8 @@ int enumerate_plans(const alcs_packed* w, long long q, int hw, std::vector<Plan>
                     p.cost *= 1.0 + 0.01 * stages;
                     // Bulk copies pay a fixed cost per copy, so they win when a tile row is one long
                     // run (images at least as large as the tile) and lose when it is cut into pieces.
-                    const bool rows_aligned = ((size_t)hw * elt) % 16 == 0;
-                    p.bulk = (rows_aligned && hw >= 32 * v.p) ? 1 : 0;
+                    const bool rows_aligned = true;     // unaligned rows are repacked to aligned ones
+                    p.bulk = hw >= 32 * v.p ? 1 : 0;
                     out.push_back(p);
                     if (rows_aligned) {
                         Plan p2 = p;
@@ -321,6 +321,44 @@ int cfg_to_plan(const alcs_packed* w, long long q, int hw, const alcs_launch_cfg
     return ALCS_ERR_UNSUPPORTED;
 }
 
+// X whose (image, channel) rows are not a multiple of 16 bytes long (H*W = 49, ...) cannot be staged
+// with 16-byte copies.  Such inputs are first repacked into scratch memory with every row padded
+// with zeros to the next multiple of 16 bytes; the main kernel then runs on the padded pixel axis
+// and simply does not store the padding pixels.
+template <typename T>
+__global__ void repack_rows_kernel(const T* __restrict__ in, T* __restrict__ out, long long rows, int hw, int hwp)
+{
+    const long long total = rows * hwp;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
+         i += (long long)gridDim.x * blockDim.x) {
+        const long long r = i / hwp;
+        const int p = (int)(i - r * hwp);
+        out[i] = p < hw ? in[r * hw + p] : T(0);
+    }
+}
+
+// pixels per image after padding the rows of X to a multiple of 16 bytes
+int padded_hw(int hw, int elt) { const int m = 16 / elt; return (hw + m - 1) / m * m; }
+
+// Make sure the scratch of w can hold `bytes`.  Growing it frees the old block, which waits for
+// all earlier work on the device.
+int ensure_xpad(const alcs_packed* w, size_t bytes)
+{
+    std::lock_guard<std::mutex> lk(w->mu);
+    if (w->xpad_bytes >= bytes) return ALCS_OK;
+    if (w->d_xpad) cudaFree(w->d_xpad);
+    w->d_xpad = nullptr;
+    w->xpad_bytes = 0;
+    cudaError_t e = cudaMalloc(&w->d_xpad, bytes);
+    if (e != cudaSuccess) {
+        alcs::set_cuda_error_text(cudaGetErrorString(e));
+        (void)cudaGetLastError();
+        return ALCS_ERR_ALLOC;
+    }
+    w->xpad_bytes = bytes;
+    return ALCS_OK;
+}
+
 int check_conv_args(const alcs_packed* w, const void* x, const void* y, int n, int h, int wd,
                     unsigned flags, long long* q_out)
 {
@@ -358,12 +396,31 @@ int launch_plan(const alcs_packed* w, const Plan& p, const void* x, void* y, int
     if (rc) return rc;
     const int elt = (int)w->elt();
     const int hw = h * wd;
+    // Rows of X that are not a multiple of 16 bytes long: repack X into scratch with padded rows.
+    int hwx = hw;
+    const void* xk = x;
+    if (((size_t)hw * elt) % 16 != 0) {
+        const int hwp = padded_hw(hw, elt);
+        const size_t need = (size_t)n * w->cin * hwp * elt;
+        if ((long long)n * hwp <= (1ll << 30) && ensure_xpad(w, need) == ALCS_OK) {
+            const long long rows = (long long)n * w->cin;
+            const unsigned blocks = (unsigned)std::min<long long>((rows * hwp + 255) / 256, (long long)di.sms * 16);
+            if (elt == 4)
+                repack_rows_kernel<float><<<blocks, 256, 0, st>>>(static_cast<const float*>(x), static_cast<float*>(w->d_xpad), rows, hw, hwp);
+            else
+                repack_rows_kernel<unsigned short><<<blocks, 256, 0, st>>>(static_cast<const unsigned short*>(x),
+                                                                          static_cast<unsigned short*>(w->d_xpad), rows, hw, hwp);
+            ALCS_CUDA(cudaGetLastError());
+            xk = w->d_xpad;
+            hwx = hwp;
+        }   // else: fall back to element-wise staging of the unpadded rows
+    }
     ConvArgs a;
-    a.x = x; a.y = y; a.bias = bias;
+    a.x = xk; a.y = y; a.bias = bias;
     a.rec = sc->rec; a.slice = sc->slice; a.rowoff = sc->rowoff; a.rowmap = sc->rowmap;
     a.err = w->d_err;
-    a.rows = w->rows; a.cin = w->cin; a.cout = w->cout; a.hw = hw;
-    a.q_total = n * hw;
+    a.rows = w->rows; a.cin = w->cin; a.cout = w->cout; a.hw = hwx; a.hwy = hw;
+    a.q_total = n * hwx;
     const int T = 32 * v.p;
     a.n_tiles = (a.q_total + T - 1) / T;
     a.n_rg = sc->n_rg; a.rpg = sc->rpg;
@@ -374,12 +431,12 @@ int launch_plan(const alcs_packed* w, const Plan& p, const void* x, void* y, int
     a.off_rec = L.off_rec; a.off_rowoff = L.off_rowoff; a.stage_bytes = L.stage_bytes;
     // widest staging copy that every (image, channel) row start and length allows
     int ld = 16;
-    while (ld > elt && (((size_t)hw * elt) % ld || (uintptr_t)x % ld)) ld >>= 1;
+    while (ld > elt && (((size_t)hwx * elt) % ld || (uintptr_t)xk % ld)) ld >>= 1;
     a.ld_bytes = ld;
     a.bulk = (ld == 16 && p.bulk) ? 1 : 0;
     a.ros = sc->ros;
     const int vg = (v.p * elt >= 16) ? 16 / elt : v.p;
-    a.st_vec = (hw % vg == 0 && (uintptr_t)y % 16 == 0) ? 1 : 0;
+    a.st_vec = (hwx == hw && hw % vg == 0 && (uintptr_t)y % 16 == 0) ? 1 : 0;
     const long long items = (long long)a.n_tiles * a.n_rg;
     if (items > 0x7fffffffll) return ALCS_ERR_SHAPE;
     // persistent thread blocks: as many as can be resident, each walks items with that stride
@@ -482,6 +539,7 @@ ALCS_API void alcs_packed_free(alcs_packed* p)
         if (cudaGetDevice(&prev) == cudaSuccess && cudaSetDevice(p->device) == cudaSuccess) {
             for (auto& kv : p->sched) free_schedule_device(kv.second);
             cudaFree(p->d_err);
+            cudaFree(p->d_xpad);
             cudaSetDevice(prev);
         }
         (void)cudaGetLastError();
@@ -706,6 +764,10 @@ ALCS_API int alcs_stack_create(const alcs_layer* layers, int n_layers, unsigned 
         if (!rc && it.q > 0) {   // the schedule must be resident before any launch is captured
             Schedule* sc = get_schedule(L.w, it.plan.kc, it.plan.n_rg, true);
             rc = sc ? upload_schedule(L.w, sc, nullptr) : ALCS_ERR_ALLOC;
+            const int elt = (int)L.w->elt();
+            const long long hw = (long long)L.h * L.wd;
+            if (!rc && (hw * elt) % 16 != 0 && (long long)L.n * padded_hw((int)hw, elt) <= (1ll << 30))
+                rc = ensure_xpad(L.w, (size_t)L.n * L.w->cin * padded_hw((int)hw, elt) * elt);
         }
         if (rc) { delete s; return rc; }
         s->items.push_back(it);

@@ -88,6 +88,8 @@ struct alcs_packed {
     // device side (valid once uploaded)
     int device = -1;
     int* d_err = nullptr;             // device error word written by a kernel whose bounded wait ran out
+    mutable void* d_xpad = nullptr;   // scratch: X repacked to 16-byte aligned rows (grown on demand)
+    mutable size_t xpad_bytes = 0;
     mutable std::map<std::pair<int, int>, alcs::Schedule> sched;   // by (kc, n_rg), built on demand
     std::map<alcs::ShapeKey, alcs_launch_cfg> tuned;   // filled by alcs_spconv1x1_tune
     mutable std::map<alcs::ShapeKey, alcs::Plan> plan_cache;   // resolved plans, by shape

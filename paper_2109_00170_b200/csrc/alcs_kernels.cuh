@@ -55,7 +55,9 @@ struct ConvArgs {
     const int* rowoff;        // [n_rg][nch][ros] start of each local row's segment inside a slice (16-byte units)
     const int* rowmap;        // [n_rg][rpg] block row of each local row, -1 = none
     int* err;                 // device error word (0 = ok)
-    int rows, cin, cout, hw;
+    int rows, cin, cout;
+    int hw;                   // pixels per image in X (padded up when X was repacked to aligned rows)
+    int hwy;                  // pixels per image in Y (the real h*w, <= hw)
     int q_total;              // n * hw
     int n_tiles, n_rg, rpg;   // pixel tiles, row groups, local rows per row group (padded)
     int kc, nch, stages;
@@ -618,12 +620,14 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_kernel(const 
             using YT = std::remove_pointer_t<decltype(ybase)>;
             size_t yoff[NG];
             bool yok[NG];
+            int yn[NG], yp[NG];
 #pragma unroll
             for (int gi = 0; gi < NG; ++gi) {
                 const int q = q0 + gi * (32 * VG) + lane * VG;
                 yok[gi] = q < a.q_total;
-                const int n = q / a.hw;
-                yoff[gi] = (size_t)n * a.cout * a.hw + (q - n * a.hw);
+                yn[gi] = q / a.hw;
+                yp[gi] = q - yn[gi] * a.hw;
+                yoff[gi] = (size_t)yn[gi] * a.cout * a.hwy + yp[gi];
             }
 #pragma unroll
             for (int s = 0; s < RW; ++s) {
@@ -643,15 +647,17 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_kernel(const 
                             if (a.relu) v[t] = fmaxf(v[t], 0.0f);
                         }
                         if (a.st_vec) {
-                            if (yok[gi]) store_vec<YT, VG>(ybase + yoff[gi] + (size_t)co * a.hw, v);
+                            if (yok[gi]) store_vec<YT, VG>(ybase + yoff[gi] + (size_t)co * a.hwy, v);
                         } else {
+                            // element by element: the run may cross into the next image, and pixels
+                            // p >= hwy exist only as padding of the repacked X
+                            int nn = yn[gi], pp = yp[gi];
 #pragma unroll
                             for (int t = 0; t < VG; ++t) {
-                                const int q = q0 + gi * (32 * VG) + lane * VG + t;
-                                if (q < a.q_total) {
-                                    const int n = q / a.hw;
-                                    store_one<YT>(ybase + ((size_t)n * a.cout + co) * a.hw + (q - n * a.hw), v[t]);
-                                }
+                                while (pp >= a.hw) { pp -= a.hw; ++nn; }
+                                if (q0 + gi * (32 * VG) + lane * VG + t < a.q_total && pp < a.hwy)
+                                    store_one<YT>(ybase + ((size_t)nn * a.cout + co) * a.hwy + pp, v[t]);
+                                ++pp;
                             }
                         }
                     }

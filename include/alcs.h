@@ -48,7 +48,8 @@ typedef enum {
     ALCS_ERR_ALLOC = -4,        /* host or device allocation failed                                 */
     ALCS_ERR_CUDA = -5,         /* a CUDA runtime call failed; see alcs_last_cuda_error()           */
     ALCS_ERR_CORRUPT = -6,      /* a serialized blob failed validation                              */
-    ALCS_ERR_STATE = -7         /* object not in the required state (e.g. weights not uploaded)     */
+    ALCS_ERR_STATE = -7,        /* object not in the required state (e.g. weights not uploaded)     */
+    ALCS_ERR_TOO_LARGE = -8     /* problem needs more than the fixed scratch of alcs_spconv1x1_noalloc */
 } alcs_status;
 
 typedef enum {
@@ -232,6 +233,33 @@ ALCS_API size_t alcs_spconv1x1_host_workspace(const alcs_packed* w, int n, int h
 ALCS_API int alcs_spconv1x1_host(const alcs_packed* w, const void* x_host, void* y_host, int n, int h,
                         int wd, const float* bias_host, unsigned flags, void* workspace,
                         size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * alcs_spconv1x1_noalloc: the same convolution for callers that must not allocate device memory.
+ * (The paper has no counterpart to this entry point; it exists for the way this library is used.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a latency-critical serving
+ * loop, after the process has handed all free device memory to another allocator, or in a plugin
+ * whose host forbids allocation calls after initialisation.  alcs_spconv1x1 may allocate: the first
+ * call for a shape uploads the launch schedule, and inputs whose rows are not a multiple of 16
+ * bytes long (h*wd = 49, ...) are repacked into scratch that w allocates or grows on demand.  This
+ * entry point never calls cudaMalloc, cudaFree or any other allocating routine:
+ *   - the launch schedule for (n, h, wd, flags) must already be on the device, i.e. alcs_spconv1x1,
+ *     alcs_spconv1x1_tune or alcs_stack_create has been called once for that shape during set-up;
+ *     otherwise the call fails with ALCS_ERR_STATE and launches nothing;
+ *   - the repacked copy of x goes into one fixed array of ALCS_NOALLOC_SCRATCH_BYTES bytes that is
+ *     part of the library image (every GPU that loads the library holds it until the process exits).
+ *     A problem that needs more, n*cin*round_up(h*wd to 16 bytes)*element size, is rejected with
+ *     ALCS_ERR_TOO_LARGE; inputs with 16-byte-multiple rows need no scratch and have no size limit.
+ * The first call on each device looks up the address of that array (with that device current); make
+ * that first call before any stream capture begins.  All calls share the one array and it keeps
+ * what the previous call left there: every call rewrites the part it uses, padding included, but two
+ * calls that overlap on the GPU (different streams) race on it -- keep them on one stream or order
+ * them with events.  Arguments, results and error codes are otherwise those of alcs_spconv1x1.
+ */
+#define ALCS_NOALLOC_SCRATCH_BYTES (16u << 20)
+ALCS_API int alcs_spconv1x1_noalloc(const alcs_packed* w, const void* x, void* y, int n, int h, int wd,
+                                    const float* bias, unsigned flags, void* cuda_stream);
 
 /* ---------------------------------------------------------------------------------------------
  * Layer stack: a network's pointwise layers run back to back on one stream (paper, Section 3.3,

@@ -15,7 +15,8 @@ LIB_PATH = os.path.join(_PKG, "libalcs.so")
 
 ALCS_OK = 0
 ALCS_ERR_INVALID_ARG, ALCS_ERR_SHAPE, ALCS_ERR_UNSUPPORTED, ALCS_ERR_ALLOC = -1, -2, -3, -4
-ALCS_ERR_CUDA, ALCS_ERR_CORRUPT, ALCS_ERR_STATE = -5, -6, -7
+ALCS_ERR_CUDA, ALCS_ERR_CORRUPT, ALCS_ERR_STATE, ALCS_ERR_TOO_LARGE = -5, -6, -7, -8
+ALCS_NOALLOC_SCRATCH_BYTES = 16 << 20
 ALCS_F32, ALCS_F16 = 0, 1
 ALCS_RELU, ALCS_Y_F32 = 1, 2
 ALCS_STACK_GRAPH = 1
@@ -26,7 +27,7 @@ EXPORTS = ["alcs_strerror", "alcs_last_cuda_error", "alcs_version", "alcs_pack",
            "alcs_packed_upload", "alcs_packed_status", "alcs_packed_free", "alcs_variant_count", "alcs_variant_get",
            "alcs_spconv1x1", "alcs_spconv1x1_cfg",
            "alcs_spconv1x1_plan", "alcs_spconv1x1_tune", "alcs_spconv1x1_set_cfg", "alcs_spconv1x1_host_workspace",
-           "alcs_spconv1x1_host", "alcs_stack_create", "alcs_stack_run", "alcs_stack_destroy"]
+           "alcs_spconv1x1_host", "alcs_spconv1x1_noalloc", "alcs_stack_create", "alcs_stack_run", "alcs_stack_destroy"]
 
 
 class AlcsError(RuntimeError):
@@ -87,6 +88,7 @@ def lib():
     L.alcs_spconv1x1_host_workspace.argtypes = [vp, i, i, i, u]
     L.alcs_spconv1x1_host_workspace.restype = sz
     L.alcs_spconv1x1_host.argtypes = [vp, vp, vp, i, i, i, vp, u, vp, sz, vp]
+    L.alcs_spconv1x1_noalloc.argtypes = [vp, vp, vp, i, i, i, vp, u, vp]
     L.alcs_stack_create.argtypes = [C.POINTER(Layer), i, u, C.POINTER(vp)]
     L.alcs_stack_run.argtypes = [vp, vp]
     L.alcs_stack_destroy.argtypes = [vp]
@@ -285,6 +287,14 @@ def alcs_spconv1x1_host(w: Packed, x_host, y_host, n: int, h: int, wd: int, bias
     _check(lib().alcs_spconv1x1_host(w.handle, _addr(x_host), _addr(y_host), n, h, wd, _addr(bias_host),
                                      flags, _addr(workspace), workspace_bytes, _stream(stream)),
            "alcs_spconv1x1_host")
+
+
+def alcs_spconv1x1_noalloc(w: Packed, x, y, n: int, h: int, wd: int, bias=None, flags: int = 0, stream=None):
+    """alcs_spconv1x1 for callers that must not allocate device memory: the shape must have been run
+    once through alcs_spconv1x1 / tune / a stack before, and the repacked input (only needed when
+    h*wd rows are not 16-byte multiples) has to fit ALCS_NOALLOC_SCRATCH_BYTES."""
+    _check(lib().alcs_spconv1x1_noalloc(w.handle, _addr(x), _addr(y), n, h, wd, _addr(bias), flags, _stream(stream)),
+           "alcs_spconv1x1_noalloc")
 
 
 class Stack:

@@ -827,3 +827,118 @@ ALCS_API int alcs_stack_destroy(alcs_stack* s)
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// alcs_spconv1x1_noalloc: the convolution for callers that cannot allocate device memory.
+//
+// Everything this entry point needs beyond the caller's buffers is either already resident (the
+// launch schedule, put there by an earlier ordinary call for the same shape) or lives in the fixed
+// array below, which is part of the library image.  The array's name is only a handle in host
+// code: its device address is looked up once per device with cudaGetSymbolAddress and that pointer
+// is what the kernels receive.
+// ---------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_noalloc_scratch[ALCS_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+
+void* g_noalloc_ptr[64] = {nullptr};     // device address of g_noalloc_scratch, per device
+std::mutex g_noalloc_mu;
+
+// Device address of the fixed scratch array on the current device `dev` (looked up on first use).
+int noalloc_scratch_address(int dev, void** out)
+{
+    if (dev < 0 || dev >= 64) return ALCS_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lk(g_noalloc_mu);
+    if (!g_noalloc_ptr[dev]) {
+        void* p = nullptr;
+        ALCS_CUDA(cudaGetSymbolAddress(&p, g_noalloc_scratch));
+        g_noalloc_ptr[dev] = p;
+    }
+    *out = g_noalloc_ptr[dev];
+    return ALCS_OK;
+}
+
+}  // namespace
+
+extern "C" ALCS_API int alcs_spconv1x1_noalloc(const alcs_packed* w, const void* x, void* y, int n, int h, int wd,
+                                               const float* bias, unsigned flags, void* cuda_stream)
+{
+    long long q = 0;
+    int rc = check_conv_args(w, x, y, n, h, wd, flags, &q);
+    if (rc) return rc;
+    rc = check_device(w);
+    if (rc) return rc;
+    if (q == 0) return ALCS_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+
+    // The plan and its schedule must already be resident: looking them up allocates nothing.
+    Plan plan;
+    Schedule* sc = nullptr;
+    {
+        std::lock_guard<std::mutex> lk(w->mu);
+        auto it = w->plan_cache.find(alcs::ShapeKey{n, h, wd, flags});
+        if (it == w->plan_cache.end()) return ALCS_ERR_STATE;
+        plan = it->second;
+        auto si = w->sched.find(std::make_pair(plan.kc, plan.n_rg));
+        if (si == w->sched.end() || !si->second.uploaded) return ALCS_ERR_STATE;
+        sc = &si->second;
+    }
+    DeviceInfo di;
+    rc = device_info(w->device, &di);
+    if (rc) return rc;
+
+    const KernelVariant& v = g_variants[plan.variant].v;
+    const int elt = (int)w->elt();
+    const int hw = h * wd;
+    int hwx = hw;
+    const void* xk = x;
+    if (((size_t)hw * elt) % 16 != 0) {
+        // rows that cannot be staged with 16-byte copies: repack into the fixed array
+        const int hwp = padded_hw(hw, elt);
+        const unsigned long long need = (unsigned long long)n * w->cin * hwp * elt;
+        if (need > ALCS_NOALLOC_SCRATCH_BYTES || (long long)n * hwp > (1ll << 30)) return ALCS_ERR_TOO_LARGE;
+        void* scratch = nullptr;
+        rc = noalloc_scratch_address(w->device, &scratch);
+        if (rc) return rc;
+        const long long rows = (long long)n * w->cin;
+        const unsigned blocks = (unsigned)std::min<long long>((rows * hwp + 255) / 256, (long long)di.sms * 16);
+        // the kernel writes every element of the region it uses, zero padding included, so nothing
+        // left behind by an earlier call can leak into this one
+        if (elt == 4)
+            repack_rows_kernel<float><<<blocks, 256, 0, st>>>(static_cast<const float*>(x), static_cast<float*>(scratch), rows, hw, hwp);
+        else
+            repack_rows_kernel<unsigned short><<<blocks, 256, 0, st>>>(static_cast<const unsigned short*>(x),
+                                                                      static_cast<unsigned short*>(scratch), rows, hw, hwp);
+        ALCS_CUDA(cudaGetLastError());
+        xk = scratch;
+        hwx = hwp;
+    }
+
+    ConvArgs a;
+    a.x = xk; a.y = y; a.bias = bias;
+    a.rec = sc->rec; a.slice = sc->slice; a.rowoff = sc->rowoff; a.rowmap = sc->rowmap;
+    a.err = w->d_err;
+    a.rows = w->rows; a.cin = w->cin; a.cout = w->cout; a.hw = hwx; a.hwy = hw;
+    a.q_total = n * hwx;
+    const int T = 32 * v.p;
+    a.n_tiles = (a.q_total + T - 1) / T;
+    a.n_rg = sc->n_rg; a.rpg = sc->rpg;
+    a.kc = sc->kc; a.nch = sc->nch; a.stages = plan.stages;
+    a.relu = (flags & ALCS_RELU) ? 1 : 0;
+    a.y_f32 = (flags & ALCS_Y_F32) ? 1 : 0;
+    const StageLayout L = stage_layout(v, *sc, elt);
+    a.off_rec = L.off_rec; a.off_rowoff = L.off_rowoff; a.stage_bytes = L.stage_bytes;
+    int ld = 16;
+    while (ld > elt && (((size_t)hwx * elt) % ld || (uintptr_t)xk % ld)) ld >>= 1;
+    a.ld_bytes = ld;
+    a.bulk = (ld == 16 && plan.bulk) ? 1 : 0;
+    a.ros = sc->ros;
+    const int vg = (v.p * elt >= 16) ? 16 / elt : v.p;
+    a.st_vec = (hwx == hw && hw % vg == 0 && (uintptr_t)y % 16 == 0) ? 1 : 0;
+    const long long items = (long long)a.n_tiles * a.n_rg;
+    if (items > 0x7fffffffll) return ALCS_ERR_SHAPE;
+    const long long grid = std::min<long long>(items, (long long)di.sms * std::max(1, plan.occ));
+    void* args[] = {&a};
+    ALCS_CUDA(cudaLaunchKernel(v.fn, dim3((unsigned)grid), dim3((v.nw + v.npw) * 32), args, plan.smem, st));
+    return ALCS_OK;
+}

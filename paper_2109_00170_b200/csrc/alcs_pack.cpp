@@ -172,6 +172,7 @@ ALCS_API const char* alcs_strerror(int status)
         case ALCS_ERR_CUDA: return "ALCS_ERR_CUDA: CUDA runtime call failed";
         case ALCS_ERR_CORRUPT: return "ALCS_ERR_CORRUPT: serialized blob failed validation";
         case ALCS_ERR_STATE: return "ALCS_ERR_STATE: object not in the required state";
+        case ALCS_ERR_TOO_LARGE: return "ALCS_ERR_TOO_LARGE: the problem needs more scratch than alcs_spconv1x1_noalloc has (ALCS_NOALLOC_SCRATCH_BYTES)";
         default: return "unknown ALCS status";
     }
 }

@@ -16,8 +16,8 @@ namespace alcs {
 
 // Chunk sizes (input channels per pipeline stage) the planner considers.  0 stands for "the
 // whole Cin in one chunk" (used when Cin is small).
-constexpr int kNumChunkings = 5;
-constexpr int kChunkings[kNumChunkings] = {16, 32, 64, 128, 0};
+constexpr int kNumChunkings = 6;
+constexpr int kChunkings[kNumChunkings] = {16, 32, 64, 96, 128, 0};
 
 // Launch schedule for one (chunk size KC, number of row groups) pair.
 //
@@ -27,16 +27,15 @@ constexpr int kChunkings[kNumChunkings] = {16, 32, 64, 128, 0};
 // is local row t of row group rg (-1 = none).
 //
 // The kept blocks are stored as segments ordered [row group][chunk][local row].  The segment of a
-// local row with blocks in a chunk is a 16-byte lead entry (the chunk-local columns of its first
-// two blocks) followed by one "pair record" per two blocks: the columns of the NEXT pair, then the
-// two g-wide value vectors of this pair (fp32; fp16 weights are widened exactly).  An odd block
-// count gets a padding block that repeats the last column with zero weights.  slice[rg*nch + k]
-// is where the (row group, chunk) slice starts, so the producer warp copies one contiguous range
-// per stage; rowoff[rg][k][t] is where local row t starts inside that slice (rowoff[..][rpg] =
-// its length).  All offsets are in 16-byte units.
+// local row with blocks in a chunk is one "pair record" per two blocks: the chunk-local columns of
+// the NEXT pair, then the two g-wide value vectors of this pair (fp32; fp16 weights are widened
+// exactly).  An odd block count gets a padding block that repeats the last column with zero
+// weights.  slice[rg*nch + k] is where the (row group, chunk) slice starts, so the producer warp
+// copies one contiguous range per stage; rowoff[rg][k][t] = {where local row t starts inside that
+// slice, the columns of its first pair, its number of pairs}.  Offsets are in 16-byte units.
 struct Schedule {
     int kc = 0, nch = 0, n_rg = 0, rpg = 0;
-    int ros = 0;                   // ints per (row group, chunk) row of rowoff: rpg + 1 rounded up to 4
+    int ros = 0;                   // ints per (row group, chunk) row of rowoff: 4 per local row
     int wcap = 0;                  // longest slice, in 16-byte units
     int n_rec = 0;                 // total length of all slices, in 16-byte units
     // host copies (kept until uploaded)

@@ -52,7 +52,7 @@ struct ConvArgs {
     const float* bias;        // [cout] or nullptr
     const unsigned char* rec; // segments of pair records, ordered [row group][chunk][local row]
     const int* slice;         // [n_rg*nch + 1] start of each (row group, chunk) slice, in 16-byte units
-    const int* rowoff;        // [n_rg][nch][ros] start of each local row's segment inside a slice (16-byte units)
+    const int* rowoff;        // [n_rg][nch][rpg] int4 per local row: {segment start inside the slice (16-byte units), c0, c1, pairs}
     const int* rowmap;        // [n_rg][rpg] block row of each local row, -1 = none
     int* err;                 // device error word (0 = ok)
     int rows, cin, cout;
@@ -65,7 +65,7 @@ struct ConvArgs {
     int y_f32;                // only meaningful for XT = __half
     int ld_bytes;             // bytes per X staging copy: 16, 8, 4 or 2
     int bulk;                 // 1: the producer uses bulk (TMA) copies; needs ld_bytes == 16
-    int ros;                  // stride of rowoff per (row group, chunk), in ints (multiple of 4)
+    int ros;                  // ints of rowoff per (row group, chunk) = 4 * rpg
     int st_vec;               // 1 if vector stores are allowed
     // shared-memory layout (bytes): [mbarriers | stage 0 | stage 1 | ...]
     int off_rec, off_rowoff, stage_bytes;
@@ -244,23 +244,22 @@ __device__ __forceinline__ void fma_block(float2 (&acc)[G][P / 2], const float (
     }
 }
 
-// Multiply-accumulate one (block row, chunk) segment of pair records into the lane's G x P
-// accumulators.  xs points at this lane's first pixel vector of the staged X tile; [rp, re) is the
-// segment in shared memory.
+// Multiply-accumulate one (block row, chunk) segment of `npairs` pair records, starting at rp in
+// shared memory, into the lane's G x P accumulators.  xs points at this lane's first pixel vector
+// of the staged X tile; (ca0, ca1) are the columns of the first pair.
 template <typename XT, int G, int P, bool DEEP>
 __device__ __forceinline__ void consume_segment(float2 (&acc)[G][P / 2], const unsigned char* xs,
-                                                const unsigned char* rp, const unsigned char* re)
+                                                const unsigned char* rp, int npairs, int ca0, int ca1)
 {
     constexpr int ROWB = 32 * P * (int)sizeof(XT);
     constexpr int REC = record_bytes(G);
-    // A segment is a 16-byte lead entry with the columns of pair 0, then one record per
-    // pair holding the columns of the NEXT pair and the weights of this one.  So the
-    // loads issued while pair i is multiplied (record i+1, X vectors of pair i+1)
-    // depend only on data that arrived while pair i-1 was multiplied.  Two register
-    // sets (A, B) alternate; nothing is copied between them.
-    const int2 lead = *reinterpret_cast<const int2*>(rp);
-    rp += 16;
-    int ca0 = lead.x, ca1 = lead.y, cb0 = 0, cb1 = 0;
+    // A segment is one record per pair, holding the columns of the NEXT pair and the weights of
+    // this one; the columns of pair 0 (ca0, ca1) come with the segment's header.  So the loads
+    // issued while pair i is multiplied (record i+1, X vectors of pair i+1) depend only on data
+    // that arrived while pair i-1 was multiplied.  Two register sets (A, B) alternate; nothing is
+    // copied between them.
+    const unsigned char* re = rp + npairs * REC;
+    int cb0 = 0, cb1 = 0;
     if constexpr (G <= 4 && DEEP) {
         float wA0[G], wA1[G], wB0[G], wB1[G];
         float2 xA0[P / 2], xA1[P / 2], xB0[P / 2], xB1[P / 2];
@@ -440,7 +439,7 @@ __device__ __forceinline__ void produce(const ConvArgs& a, unsigned char* smem, 
             const unsigned char* rsrc = a.rec + (size_t)r0 * 16;
             for (int i = lane + 32 * pw; i < n16; i += 32 * npw) cp_async_16(st + a.off_rec + i * 16, rsrc + (size_t)i * 16);
             const int* osrc = rowoff + (size_t)k * a.ros;
-            for (int i = lane + 32 * pw; i <= a.rpg; i += 32 * npw) cp_async_4(st + a.off_rowoff + i * 4, osrc + i);
+            for (int i = lane + 32 * pw; i < a.rpg; i += 32 * npw) cp_async_16(st + a.off_rowoff + i * 16, osrc + 4 * i);
             if constexpr (LDB == 2) __threadfence_block();
             mbar_arrive_on_copies(smem_u32 + 8 * s);      // "full" completes when all producer lanes' copies land
         }
@@ -603,13 +602,12 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_kernel(const 
             const unsigned char* stage = ring + st * a.stage_bytes;
             const unsigned char* xs = stage + lane * (VG * SZ);
             const unsigned char* recs = stage + a.off_rec;
-            const int* roff = reinterpret_cast<const int*>(stage + a.off_rowoff);
+            const int4* roff = reinterpret_cast<const int4*>(stage + a.off_rowoff);
 #pragma unroll
             for (int s = 0; s < RW; ++s) {
                 if (lrow[s] >= a.rpg) continue;
-                const unsigned char* rp = recs + roff[lrow[s]] * 16;
-                const unsigned char* re = recs + roff[lrow[s] + 1] * 16;
-                if (rp < re) consume_segment<XT, G, P, kDeep>(acc[s], xs, rp, re);
+                const int4 hd = roff[lrow[s]];     // {segment start, first two columns, pairs}
+                if (hd.w > 0) consume_segment<XT, G, P, kDeep>(acc[s], xs, recs + hd.x * 16, hd.w, hd.y, hd.z);
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32 + 8 * kMaxStages + 8 * st);   // stage st may be refilled

@@ -79,7 +79,7 @@ void build_schedule(const alcs_packed& p, int kc, int n_rg, bool with_records, S
     }
 
     out.h_slice.assign((size_t)n_rg * nch + 1, 0);
-    const int ros = (rpg + 1 + 3) & ~3;          // padded so that one row of offsets is a multiple of 16 bytes
+    const int ros = rpg * 4;                     // one int4 {offset, first two columns, pair count} per local row
     out.ros = ros;
     out.h_rowoff.assign((size_t)n_rg * nch * ros, 0);
     out.h_rec.clear();
@@ -109,7 +109,8 @@ void build_schedule(const alcs_packed& p, int kc, int n_rg, bool with_records, S
             const int c0 = c * kc;
             int local = 0;
             for (int t = 0; t < rpg; ++t) {
-                roff[t] = local;
+                int* hd = roff + 4 * t;                 // {segment start (16-byte units), c0, c1, pairs}
+                hd[0] = local; hd[1] = hd[2] = hd[3] = 0;
                 const int r = out.h_rowmap[(size_t)rg * rpg + t];
                 if (r < 0) continue;
                 int k = cursor[r];
@@ -117,21 +118,20 @@ void build_schedule(const alcs_packed& p, int kc, int n_rg, bool with_records, S
                 int k1 = k;
                 while (k1 < kend && p.col_idx[k1] < lim) ++k1;
                 const int npair = (k1 - k + 1) / 2;
-                const int seg16 = npair ? 1 + npair * (REC / 16) : 0;   // lead entry + records
+                const int seg16 = npair * (REC / 16);
+                auto cols_of = [&](int q, int* c) {       // chunk-local columns of pair q
+                    const int ka = k + 2 * q;
+                    const int kb = ka + 1 < k1 ? ka + 1 : ka;    // padding repeats the column
+                    c[0] = p.col_idx[ka] - c0;
+                    c[1] = p.col_idx[kb] - c0;
+                };
+                if (npair) cols_of(0, hd + 1);
+                hd[3] = npair;
                 if (with_records && npair) {
                     const size_t base = out.h_rec.size();
                     out.h_rec.resize(base + (size_t)seg16 * 16, 0);
-                    auto cols_of = [&](int q, int* c) {       // chunk-local columns of pair q
-                        const int ka = k + 2 * q;
-                        const int kb = ka + 1 < k1 ? ka + 1 : ka;    // padding repeats the column
-                        c[0] = p.col_idx[ka] - c0;
-                        c[1] = p.col_idx[kb] - c0;
-                    };
-                    int lead[4] = {0, 0, 0, 0};
-                    cols_of(0, lead);
-                    std::memcpy(&out.h_rec[base], lead, 16);
                     for (int q = 0; q < npair; ++q) {
-                        unsigned char* rec = &out.h_rec[base + 16 + (size_t)q * REC];
+                        unsigned char* rec = &out.h_rec[base + (size_t)q * REC];
                         const int ka = k + 2 * q;
                         const bool has_b = ka + 1 < k1;
                         int hdr[4] = {0, 0, 0, 0};
@@ -147,7 +147,6 @@ void build_schedule(const alcs_packed& p, int kc, int n_rg, bool with_records, S
                 local += seg16;
                 cursor[r] = k1;
             }
-            roff[rpg] = local;
             rec_count += local;
             wcap = std::max(wcap, local);
         }

@@ -476,6 +476,7 @@ def main():
         "roofline": roof,
         "stack_roofline": {"sum_t_roof_us": round(sum_roof, 1), "sum_layer_us": round(sum_us, 1),
                            "frac": round(sum_roof / sum_us, 4), "min_layer_frac": min(r["frac"] for r in rows),
+                           "step_frac": round(sum_roof / (ms_step * 1e3), 4),
                            "us_per_layer": round(ms_step * 1e3 / nl, 2)},
         "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": nl * args.steps, "clocks": clocks,
         "batch1": batch1, "layers": rows,

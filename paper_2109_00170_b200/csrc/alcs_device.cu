@@ -442,7 +442,19 @@ int launch_plan(const alcs_packed* w, const Plan& p, const void* x, void* y, int
     // persistent thread blocks: as many as can be resident, each walks items with that stride
     const long long grid = std::min<long long>(items, (long long)di.sms * std::max(1, p.occ));
     void* args[] = {&a};
-    ALCS_CUDA(cudaLaunchKernel(v.fn, dim3((unsigned)grid), dim3((v.nw + v.npw) * 32), args, p.smem, st));
+    // programmatic dependent launch: this kernel's set-up may overlap the tail of the kernel before
+    // it on the stream; it waits for that kernel before it reads X or writes Y
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3((unsigned)grid);
+    lc.blockDim = dim3((v.nw + v.npw) * 32);
+    lc.dynamicSmemBytes = p.smem;
+    lc.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    ALCS_CUDA(cudaLaunchKernelExC(&lc, v.fn, args));
     return ALCS_OK;
 }
 

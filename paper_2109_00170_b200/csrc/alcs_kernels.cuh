@@ -115,6 +115,15 @@ __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uin
                  "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
 }
+// Programmatic dependent launch: a kernel launched with the programmatic-serialization attribute
+// may start while the previous kernel on the stream is still draining.  grid_dep_wait() blocks until
+// that previous kernel has completed and its writes are visible; everything that touches X, Y or the
+// repack scratch comes after it, so only set-up work (barrier init, the first weight copies)
+// overlaps the predecessor's tail.  grid_dep_launch() lets the NEXT kernel start its own set-up.
+// Both are no-ops for an ordinary launch.
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
+
 // Bounded wait for the phase with the given parity to complete.  Each poll lets the hardware
 // suspend the warp for up to about a microsecond, and failed polls back off with nanosleep, so a
 // waiting warp does not take issue slots from the warps that compute.
@@ -385,6 +394,7 @@ __device__ __forceinline__ void produce(const ConvArgs& a, unsigned char* smem, 
     const int items = a.n_tiles * a.n_rg;
     int kk = 0;                             // running (item, chunk) counter = ring position
 
+    bool dep_ok = false;                    // has the predecessor kernel been waited for yet?
     for (int item = blockIdx.x; item < items; item += gridDim.x) {
         const int tile = item / a.n_rg;
         const int rg = item - tile * a.n_rg;
@@ -412,6 +422,16 @@ __device__ __forceinline__ void produce(const ConvArgs& a, unsigned char* smem, 
                 }
             }
             const uint32_t st = ring + s * a.stage_bytes;
+            // the row group's pair records of this chunk and their per-row offsets
+            const int r0 = __ldg(slice + k);
+            const int n16 = __ldg(slice + k + 1) - r0;
+            const unsigned char* rsrc = a.rec + (size_t)r0 * 16;
+            for (int i = lane + 32 * pw; i < n16; i += 32 * npw) cp_async_16(st + a.off_rec + i * 16, rsrc + (size_t)i * 16);
+            const int* osrc = rowoff + (size_t)k * a.ros;
+            for (int i = lane + 32 * pw; i < a.rpg; i += 32 * npw) cp_async_16(st + a.off_rowoff + i * 16, osrc + 4 * i);
+            // X (or its repacked copy) is the predecessor kernel's output: wait for it once, after the
+            // first weight copies are already in flight
+            if (!dep_ok) { grid_dep_wait(); dep_ok = true; }
             // X tile of this chunk
             const int cbase = k * a.kc;
             const int nrows = min(a.kc, a.cin - cbase);
@@ -433,13 +453,6 @@ __device__ __forceinline__ void produce(const ConvArgs& a, unsigned char* smem, 
                             __ldg(reinterpret_cast<const unsigned short*>(sp + c * ch_bytes));
                 }
             }
-            // the row group's pair records of this chunk and their per-row offsets
-            const int r0 = __ldg(slice + k);
-            const int n16 = __ldg(slice + k + 1) - r0;
-            const unsigned char* rsrc = a.rec + (size_t)r0 * 16;
-            for (int i = lane + 32 * pw; i < n16; i += 32 * npw) cp_async_16(st + a.off_rec + i * 16, rsrc + (size_t)i * 16);
-            const int* osrc = rowoff + (size_t)k * a.ros;
-            for (int i = lane + 32 * pw; i < a.rpg; i += 32 * npw) cp_async_16(st + a.off_rowoff + i * 16, osrc + 4 * i);
             if constexpr (LDB == 2) __threadfence_block();
             mbar_arrive_on_copies(smem_u32 + 8 * s);      // "full" completes when all producer lanes' copies land
         }
@@ -466,6 +479,7 @@ __device__ __forceinline__ void produce_bulk(const ConvArgs& a, unsigned char* s
     const int items = a.n_tiles * a.n_rg;
     int kk = 0;
 
+    bool dep_ok = false;                    // has the predecessor kernel been waited for yet?
     for (int item = blockIdx.x; item < items; item += gridDim.x) {
         const int tile = item / a.n_rg;
         const int rg = item - tile * a.n_rg;
@@ -494,6 +508,12 @@ __device__ __forceinline__ void produce_bulk(const ConvArgs& a, unsigned char* s
                 const int rbytes = (__ldg(slice + k + 1) - r0) * 16;
                 if (lane == 0 && pw == 0) mbar_arrive_expect_tx(bar, (uint32_t)(nrows * vt * SZ + rbytes + a.ros * 4));
                 __syncwarp();
+                if (lane == 0 && pw == 0 && rbytes > 0) bulk_copy_g2s(st + a.off_rec, a.rec + (size_t)r0 * 16, (uint32_t)rbytes, bar);
+                if (lane == 1 && pw == 0)
+                    bulk_copy_g2s(st + a.off_rowoff, rowoff + (size_t)k * a.ros, (uint32_t)(a.ros * 4), bar);
+                // X (or its repacked copy) is the predecessor kernel's output: wait for it once,
+                // after the first weight copies are already in flight
+                if (!dep_ok) { grid_dep_wait(); dep_ok = true; }
                 // X: channel rows lane, lane+32, ...; each row is one copy per image it touches
                 for (int c = lane + 32 * pw; c < nrows; c += 32 * npw) {
                     const unsigned char* src = xbase + (size_t)(cbase + c) * ch_bytes;
@@ -509,9 +529,7 @@ __device__ __forceinline__ void produce_bulk(const ConvArgs& a, unsigned char* s
                         p = 0;
                     }
                 }
-                if (lane == 0 && pw == 0 && rbytes > 0) bulk_copy_g2s(st + a.off_rec, a.rec + (size_t)r0 * 16, (uint32_t)rbytes, bar);
-                if (lane == 1 && pw == 0)
-                    bulk_copy_g2s(st + a.off_rowoff, rowoff + (size_t)k * a.ros, (uint32_t)(a.ros * 4), bar);
+
             }
         }
     }
@@ -549,6 +567,7 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_kernel(const 
         }
     }
     __syncthreads();
+    grid_dep_launch();
 
     if (warp >= NW) {   // ---- producer warps ------------------------------------------------
         const int pw = warp - NW;
@@ -614,6 +633,7 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_kernel(const 
         }
 
         // ---- epilogue: bias, ReLU, store ----------------------------------------------------
+        grid_dep_wait();    // (long satisfied: the data consumed above was loaded after the producer's wait)
         auto epilogue = [&](auto* ybase) {
             using YT = std::remove_pointer_t<decltype(ybase)>;
             size_t yoff[NG];

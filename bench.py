@@ -31,7 +31,7 @@ from alcs_workloads import config_layers, make_bias, make_mask, make_weights, ma
 
 METRIC = "nonzero-GFLOP/s & % of roofline, SIMD-sparse 1x1 conv stack, 1 B200, b=1/64"
 UNIT = "GFLOP/s"
-WORKLOADS = {"mbv1_b64": 2, "mbv1_b1": 1, "c1": 0, "rn50_b32": 3}
+WORKLOADS = {"mbv1_b64": 2, "mbv1_b1": 1, "c1": 0, "rn50_b32": 3, "sweep_b256": 4}
 SM_COUNT, FP32_LANES = 148, 128
 
 
@@ -196,6 +196,29 @@ def run_reference(args, specs, wl):
         "gpu_launches": 0}))
 
 
+def rank_env():
+    """(rank, world size, local rank) as torchrun exports them; a plain run is rank 0 of 1."""
+    return (int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1")),
+            int(os.environ.get("LOCAL_RANK", "0")))
+
+
+def max_over_ranks(ms, world, device=None):
+    """The slowest rank's time: what a multi-GPU step costs.  No-op for one rank."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(ms)], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_gflops(flops_per_rank, world, ms_per_step):
+    """Weak scaling: every rank runs its own batch (replicas, no exchange), so the job's
+    throughput is the ranks' work added up over the slowest rank's time."""
+    return world * flops_per_rank / (ms_per_step * 1e-3) / 1e9
+
+
 def measure_batch1(A, torch, dev, stream, steps, hbm_gbs, fp32_tf):
     """The same stack at batch 1 (the paper's latency setting), replayed as one CUDA graph.  A layer's
     roofline time is below a microsecond there, so the run is launch- and latency-bound; reported
@@ -277,9 +300,7 @@ def main():
     import torch.distributed as dist
     import paper_2109_00170_b200 as A
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = rank_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
     torch.cuda.set_device(local)
@@ -386,12 +407,9 @@ def main():
     per_layer_ms = [statistics.mean(evs[k][i].elapsed_time(evs[k][i + 1]) for k in range(args.steps)) for i in range(nl)]
     per_layer_min = [min(evs[k][i].elapsed_time(evs[k][i + 1]) for k in range(args.steps)) for i in range(nl)]
 
-    if world > 1:
-        t = torch.tensor([ms_total], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, world, dev)
     ms_step = ms_total / args.steps
-    value = world * total_flops / (ms_step * 1e-3) / 1e9
+    value = whole_job_gflops(total_flops, world, ms_step)
 
     # ---- end to end: host buffers through alcs_spconv1x1_host, copies inside the timed region --
     e2e = None
@@ -417,12 +435,8 @@ def main():
         f1.record(stream)
         barrier()
         ms_e2e = f0.elapsed_time(f1)
-        if world > 1:
-            t = torch.tensor([ms_e2e], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e2e = float(t.item())
-        ms_e2e /= args.e2e_steps
-        e2e = {"value": world * total_flops / (ms_e2e * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms_e2e,
+        ms_e2e = max_over_ranks(ms_e2e, world, dev) / args.e2e_steps
+        e2e = {"value": whole_job_gflops(total_flops, world, ms_e2e), "unit": UNIT, "ms_per_step": ms_e2e,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": args.e2e_steps}
 
     if rank != 0:

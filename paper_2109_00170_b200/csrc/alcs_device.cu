@@ -224,7 +224,13 @@ int enumerate_plans(const alcs_packed* w, long long q, int hw, std::vector<Plan>
             last_kc = kc;
             if ((size_t)kc * 32 * v.p * elt * 2 > (size_t)smem_max) continue;
             int last_rpg = -1;
-            for (int n_rg = rg_min; n_rg <= std::min(w->rows, rg_min * 4 + 2); ++n_rg) {
+            // Row-group counts to consider: every count up to a few times the minimum, and, when
+            // the pixel tiles alone are too few to occupy the GPU (small batches), a geometric
+            // ladder of larger counts up to about two work items per SM.
+            const long long tiles = (q + 32 * v.p - 1) / (32 * v.p);
+            const int rg_dense = std::min(w->rows, rg_min * 4 + 2);
+            const int rg_hi = std::max<long long>(rg_dense, std::min<long long>(w->rows, (2ll * di.sms + tiles - 1) / tiles));
+            for (int n_rg = rg_min; n_rg <= rg_hi; n_rg = n_rg < rg_dense ? n_rg + 1 : std::max(n_rg + 1, n_rg * 5 / 4)) {
                 const int rpg = (w->rows + n_rg - 1) / n_rg;
                 if (rpg == last_rpg || rpg > cap) continue;
                 last_rpg = rpg;

@@ -9,8 +9,8 @@ LAUNCHES.csv is the `--csv --log-file` output of
         python bench.py --steps 2 --warmup 3 --no-cpu-baseline --e2e-steps 0 --no-batch1
 
 and BENCH.json is the JSON line the same command printed when run without ncu.  The launches inside
-the "alcs_timed" range are the layers of the stack in order, repeated `steps` times, so launch i is
-layer i mod n_layers.  Per-launch times under ncu are cold-cache and serialised: the SHARES are what
+the "alcs_timed" range are the layers of the stack in order, repeated `steps` times, so convolution launch i
+is layer i mod n_layers (a row-repacking launch belongs to the convolution after it).  Per-launch times under ncu are cold-cache and serialised: the SHARES are what
 can be compared with the live CUDA-event timings, not the absolutes.
 """
 from __future__ import annotations
@@ -77,19 +77,25 @@ def main():
         sys.exit("no JSON line in " + a.bench_json)
     layers = bench["layers"]
     nl = len(layers)
-    if not launches or len(launches) % nl:
-        sys.exit(f"{len(launches)} launches do not divide into {nl} layers")
-    reps = len(launches) // nl
+    # A layer whose X rows are not a multiple of 16 bytes launches the row-repacking kernel first;
+    # that launch is counted with the convolution that follows it.
+    n_conv = sum(1 for name, _ in launches if "spconv1x1_kernel" in name)
+    if not n_conv or n_conv % nl:
+        sys.exit(f"{n_conv} convolution launches do not divide into {nl} layers")
+    reps = n_conv // nl
 
     per_kernel = defaultdict(lambda: [0, 0.0])
     per_layer = [dict(t=0.0, rd=0.0, wr=0.0) for _ in range(nl)]
     total = 0.0
-    for i, (name, m) in enumerate(launches):
+    i = 0
+    for name, m in launches:
         t = m.get("gpu__time_duration.sum", 0.0)
         short = re.sub(r"^void\s+|alcs::|\(.*\)$", "", name)
         per_kernel[short][0] += 1
         per_kernel[short][1] += t
         L = per_layer[i % nl]
+        if "spconv1x1_kernel" in name:
+            i += 1
         L["t"] += t / reps
         L["rd"] += m.get("dram__bytes_read.sum", 0.0) / reps
         L["wr"] += m.get("dram__bytes_write.sum", 0.0) / reps

@@ -161,10 +161,14 @@ ALCS_API void alcs_packed_free(alcs_packed* p);
  *   copy_mode         how X tiles reach shared memory: 1 = per-lane cp.async, 2 = bulk (TMA) copies
  *                     of whole pixel runs (needs 16-byte aligned rows; otherwise 1 is used)
  *   producer_warps    warps of the thread block that only move data (1..4)
+ *   math_mode         1 = fp32 FMA on the CUDA cores; 2 = tensor cores (fp16 weights and activations
+ *                     only): 16 kept blocks of a block row times the 16 input rows they select is a
+ *                     dense 16 x g by 16 x pixels contraction, run as warp-level MMA with fp32
+ *                     accumulation
  */
 typedef struct {
     int pixels_per_lane, rows_per_warp, warps, chunk_channels, stages, row_groups, min_blocks, copy_mode,
-        producer_warps;
+        producer_warps, math_mode;
 } alcs_launch_cfg;
 
 /*

@@ -60,6 +60,8 @@ void init_variants_locked()
     for (int i = 0; i < n; ++i) g_variants.push_back({t[i]});
     t = alcs::variants_f16(&n);
     for (int i = 0; i < n; ++i) g_variants.push_back({t[i]});
+    t = alcs::variants_f16_mma(&n);
+    for (int i = 0; i < n; ++i) g_variants.push_back({t[i]});
 }
 
 int device_info(int dev, DeviceInfo* out)
@@ -93,28 +95,36 @@ using alcs::Schedule;
 
 struct StageLayout {
     int off_rec, off_rowoff, stage_bytes;
+    int tail_bytes;     // shared memory after the ring (epilogue scratch of the tensor-core kernels)
 };
 
 StageLayout stage_layout(const KernelVariant& v, const Schedule& sc, int elt)
 {
     StageLayout L;
-    L.off_rec = sc.kc * 32 * v.p * elt;                              // X tile first
+    // X tile first; the tensor-core kernels pad every channel row by 16 bytes
+    L.off_rec = sc.kc * (32 * v.p * elt + (v.mma ? 16 : 0));
     L.off_rowoff = L.off_rec + sc.wcap * 16;
     L.stage_bytes = L.off_rowoff + sc.ros * 4;
+    L.tail_bytes = v.mma ? v.nw * 8 * (32 * v.p * 2 + 16) : 0;     // [8 channels][T pixels] fp16 per consumer warp
     return L;
 }
 
-size_t plan_smem(const StageLayout& L, int stages) { return 16 * alcs::kMaxStages + (size_t)stages * L.stage_bytes; }
+size_t plan_smem(const StageLayout& L, int stages)
+{
+    return 16 * alcs::kMaxStages + (size_t)stages * L.stage_bytes + L.tail_bytes;
+}
 
 // The schedule for (kc, n_rg): sizes only (with_records = false) or complete.  Cached in w.
-Schedule* get_schedule(const alcs_packed* w, int kc, int n_rg, bool with_records)
+Schedule* get_schedule(const alcs_packed* w, int kc, int n_rg, bool with_records, int mma)
 {
     if (kc <= 0 || kc > w->cin) kc = w->cin;
     std::lock_guard<std::mutex> lk(w->mu);
-    Schedule& sc = w->sched[std::make_pair(kc, n_rg)];
+    Schedule& sc = w->sched[alcs::sched_key(kc, n_rg, mma)];
     try {
-        if (sc.n_rg == 0 || (with_records && !sc.uploaded && sc.h_rec.empty() && sc.n_rec > 0))
-            alcs::build_schedule(*w, kc, n_rg, with_records, sc);
+        if (sc.n_rg == 0 || (with_records && !sc.uploaded && sc.h_rec.empty() && sc.n_rec > 0)) {
+            if (mma) alcs::build_schedule_mma(*w, kc, n_rg, with_records, sc);
+            else alcs::build_schedule(*w, kc, n_rg, with_records, sc);
+        }
     } catch (const std::bad_alloc&) {
         return nullptr;
     }
@@ -170,6 +180,22 @@ double model_cost(const alcs_packed* w, const KernelVariant& v, const Schedule& 
     const long long items = n_tiles * sc.n_rg;
     const long long slots = (long long)sms * occ;
     const long long rounds = (items + slots - 1) / slots;
+    if (v.mma) {
+        // shared-memory wavefronts dominate: per step and 16-pixel tile one 4-wavefront ldmatrix
+        // (about 1.4 with the residual bank conflicts), plus the staging writes of the tile
+        const double steps_item = (double)sc.n_rec * 16.0 / alcs::step_record_bytes(v.g) / sc.n_rg;
+        const double lsu = steps_item * (2.0 * v.p * 4 * 1.4 + 3 + 2.0 * (v.g > 8 ? 2 : 1)) +
+                           (double)sc.nch * sc.kc * T * elt / 128.0;
+        const double issue = steps_item * (2.0 * v.p * (1 + (v.g > 8 ? 2 : 1)) * 2 + 12) / 4.0 +
+                             (double)sc.rpg * sc.nch * 14.0 / 4.0;
+        const double l2b = ((double)w->cin * T * elt + steps_item * alcs::step_record_bytes(v.g)) / (16.0 * v.npw);
+        const double warps = (double)v.nw * occ;
+        const double hide = std::min(1.0, 0.4 + warps / 20.0);
+        const double item_cycles = std::max(std::max(issue, lsu) / hide, l2b) + 2500.0;
+        const double t_sm = (double)rounds * occ * item_cycles / 1.9e9;
+        const double bytes = (double)q * (w->cin + w->cout) * elt;
+        return std::max(t_sm, bytes / 6.0e12);
+    }
     const int vg = (v.p * elt >= 16) ? 16 / elt : v.p;
     const int ng = v.p / vg;
     const double pairs_item = (double)sc.n_rec * 16.0 / alcs::record_bytes(v.g) / sc.n_rg;
@@ -234,7 +260,7 @@ int enumerate_plans(const alcs_packed* w, long long q, int hw, std::vector<Plan>
                 const int rpg = (w->rows + n_rg - 1) / n_rg;
                 if (rpg == last_rpg || rpg > cap) continue;
                 last_rpg = rpg;
-                const Schedule* sc = get_schedule(w, kc, n_rg, false);
+                const Schedule* sc = get_schedule(w, kc, n_rg, false, v.mma);
                 if (!sc) return ALCS_ERR_ALLOC;
                 const StageLayout L = stage_layout(v, *sc, elt);
                 for (int stages = 2; stages <= alcs::kMaxStages; ++stages) {
@@ -279,6 +305,7 @@ void plan_to_cfg(const Plan& p, alcs_launch_cfg* c)
     c->min_blocks = v.minb;
     c->copy_mode = p.bulk ? 2 : 1;
     c->producer_warps = v.npw;
+    c->math_mode = v.mma ? 2 : 1;
 }
 
 // Resolve a (possibly partial) configuration into a concrete plan.
@@ -295,6 +322,7 @@ int cfg_to_plan(const alcs_packed* w, long long q, int hw, const alcs_launch_cfg
         if (c->warps && c->warps != v.nw) return false;
         if (c->min_blocks && c->min_blocks != v.minb) return false;
         if (c->producer_warps && c->producer_warps != v.npw) return false;
+        if (c->math_mode && (c->math_mode == 2) != (v.mma == 1)) return false;
         if (c->chunk_channels && std::min(c->chunk_channels, w->cin) != p.kc) return false;
         if (c->stages && c->stages != p.stages) return false;
         if (c->copy_mode && (c->copy_mode == 2) != (p.bulk == 1)) return false;
@@ -312,7 +340,7 @@ int cfg_to_plan(const alcs_packed* w, long long q, int hw, const alcs_launch_cfg
             const KernelVariant& v = g_variants[p0.variant].v;
             const int rpg = (w->rows + c->row_groups - 1) / c->row_groups;
             if (rpg > v.nw * v.rw) continue;
-            const Schedule* sc = get_schedule(w, p0.kc, c->row_groups, false);
+            const Schedule* sc = get_schedule(w, p0.kc, c->row_groups, false, v.mma);
             if (!sc) return ALCS_ERR_ALLOC;
             Plan p = p0;
             p.n_rg = sc->n_rg;
@@ -331,15 +359,23 @@ int cfg_to_plan(const alcs_packed* w, long long q, int hw, const alcs_launch_cfg
 // with 16-byte copies.  Such inputs are first repacked into scratch memory with every row padded
 // with zeros to the next multiple of 16 bytes; the main kernel then runs on the padded pixel axis
 // and simply does not store the padding pixels.
+// Each thread writes one 16-byte piece of a padded row (EPV elements), reading its elements one
+// by one: the source rows start at arbitrary element offsets.
 template <typename T>
 __global__ void repack_rows_kernel(const T* __restrict__ in, T* __restrict__ out, long long rows, int hw, int hwp)
 {
-    const long long total = rows * hwp;
+    constexpr int EPV = 16 / (int)sizeof(T);
+    const int vpr = hwp / EPV;                       // 16-byte pieces per padded row
+    const long long total = rows * vpr;
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
          i += (long long)gridDim.x * blockDim.x) {
-        const long long r = i / hwp;
-        const int p = (int)(i - r * hwp);
-        out[i] = p < hw ? in[r * hw + p] : T(0);
+        const long long r = i / vpr;
+        const int p0 = (int)(i - r * vpr) * EPV;
+        const T* src = in + r * hw + p0;
+        alignas(16) T v[EPV];
+#pragma unroll
+        for (int t = 0; t < EPV; ++t) v[t] = p0 + t < hw ? __ldg(src + t) : T(0);
+        *reinterpret_cast<uint4*>(out + r * hwp + p0) = *reinterpret_cast<const uint4*>(v);
     }
 }
 
@@ -391,7 +427,7 @@ int launch_plan(const alcs_packed* w, const Plan& p, const void* x, void* y, int
                 const float* bias, unsigned flags, cudaStream_t st)
 {
     const KernelVariant& v = g_variants[p.variant].v;
-    Schedule* sc = get_schedule(w, p.kc, p.n_rg, true);
+    Schedule* sc = get_schedule(w, p.kc, p.n_rg, true, v.mma);
     if (!sc) return ALCS_ERR_ALLOC;
     if (!sc->uploaded) {
         const int rc = upload_schedule(w, sc, st);
@@ -410,7 +446,7 @@ int launch_plan(const alcs_packed* w, const Plan& p, const void* x, void* y, int
         const size_t need = (size_t)n * w->cin * hwp * elt;
         if ((long long)n * hwp <= (1ll << 30) && ensure_xpad(w, need) == ALCS_OK) {
             const long long rows = (long long)n * w->cin;
-            const unsigned blocks = (unsigned)std::min<long long>((rows * hwp + 255) / 256, (long long)di.sms * 16);
+            const unsigned blocks = (unsigned)std::min<long long>((rows * (hwp * elt / 16) + 255) / 256, (long long)di.sms * 16);
             if (elt == 4)
                 repack_rows_kernel<float><<<blocks, 256, 0, st>>>(static_cast<const float*>(x), static_cast<float*>(w->d_xpad), rows, hw, hwp);
             else
@@ -477,9 +513,10 @@ int resolve_plan(const alcs_packed* w, int n, int h, int wd, unsigned flags, lon
 {
     alcs::ShapeKey key{n, h, wd, flags};
     if (cfg) {
-        const int c[9] = {cfg->pixels_per_lane, cfg->rows_per_warp, cfg->warps, cfg->chunk_channels,
-                          cfg->stages, cfg->row_groups, cfg->min_blocks, cfg->copy_mode, cfg->producer_warps};
-        for (int i = 0; i < 9; ++i) key.c[i] = c[i];
+        const int c[10] = {cfg->pixels_per_lane, cfg->rows_per_warp, cfg->warps, cfg->chunk_channels,
+                           cfg->stages, cfg->row_groups, cfg->min_blocks, cfg->copy_mode, cfg->producer_warps,
+                           cfg->math_mode};
+        for (int i = 0; i < 10; ++i) key.c[i] = c[i];
     }
     {
         std::lock_guard<std::mutex> lk(w->mu);
@@ -588,6 +625,7 @@ ALCS_API int alcs_variant_get(int index, alcs_dtype* dt, int* g, alcs_launch_cfg
         cfg->min_blocks = v.minb;
         cfg->copy_mode = 0;
         cfg->producer_warps = v.npw;
+        cfg->math_mode = v.mma ? 2 : 1;
     }
     return ALCS_OK;
 }
@@ -694,10 +732,11 @@ ALCS_API int alcs_spconv1x1_tune(alcs_packed* w, const void* x, void* y, int n, 
     }
     {   // release the device copies of the schedules that did not win
         std::lock_guard<std::mutex> lk(w->mu);
+        auto key_of = [&](const Plan& pl) { return alcs::sched_key(pl.kc, pl.n_rg, g_variants[pl.variant].v.mma); };
         for (auto& kv : w->sched)
-            if (kv.second.uploaded && !(kv.first.first == all[best_i].kc && kv.first.second == all[best_i].n_rg)) {
+            if (kv.second.uploaded && kv.first != key_of(all[best_i])) {
                 bool used = false;
-                for (auto& pc : w->plan_cache) used |= (pc.second.kc == kv.first.first && pc.second.n_rg == kv.first.second);
+                for (auto& pc : w->plan_cache) used |= (key_of(pc.second) == kv.first);
                 if (!used) { free_schedule_device(kv.second); kv.second.n_rg = 0; }
             }
     }
@@ -780,7 +819,7 @@ ALCS_API int alcs_stack_create(const alcs_layer* layers, int n_layers, unsigned 
         if (!rc) rc = check_device(L.w);
         if (!rc && it.q > 0) rc = resolve_plan(L.w, L.n, L.h, L.wd, L.flags, it.q, nullptr, &it.plan);
         if (!rc && it.q > 0) {   // the schedule must be resident before any launch is captured
-            Schedule* sc = get_schedule(L.w, it.plan.kc, it.plan.n_rg, true);
+            Schedule* sc = get_schedule(L.w, it.plan.kc, it.plan.n_rg, true, g_variants[it.plan.variant].v.mma);
             rc = sc ? upload_schedule(L.w, sc, nullptr) : ALCS_ERR_ALLOC;
             const int elt = (int)L.w->elt();
             const long long hw = (long long)L.h * L.wd;
@@ -897,7 +936,7 @@ extern "C" ALCS_API int alcs_spconv1x1_noalloc(const alcs_packed* w, const void*
         auto it = w->plan_cache.find(alcs::ShapeKey{n, h, wd, flags});
         if (it == w->plan_cache.end()) return ALCS_ERR_STATE;
         plan = it->second;
-        auto si = w->sched.find(std::make_pair(plan.kc, plan.n_rg));
+        auto si = w->sched.find(alcs::sched_key(plan.kc, plan.n_rg, g_variants[plan.variant].v.mma));
         if (si == w->sched.end() || !si->second.uploaded) return ALCS_ERR_STATE;
         sc = &si->second;
     }
@@ -919,7 +958,7 @@ extern "C" ALCS_API int alcs_spconv1x1_noalloc(const alcs_packed* w, const void*
         rc = noalloc_scratch_address(w->device, &scratch);
         if (rc) return rc;
         const long long rows = (long long)n * w->cin;
-        const unsigned blocks = (unsigned)std::min<long long>((rows * hwp + 255) / 256, (long long)di.sms * 16);
+        const unsigned blocks = (unsigned)std::min<long long>((rows * (hwp * elt / 16) + 255) / 256, (long long)di.sms * 16);
         // the kernel writes every element of the region it uses, zero padding included, so nothing
         // left behind by an earlier call can leak into this one
         if (elt == 4)

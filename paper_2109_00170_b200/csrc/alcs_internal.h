@@ -33,8 +33,16 @@ constexpr int kChunkings[kNumChunkings] = {16, 32, 64, 96, 128, 0};
 // weights.  slice[rg*nch + k] is where the (row group, chunk) slice starts, so the producer warp
 // copies one contiguous range per stage; rowoff[rg][k][t] = {where local row t starts inside that
 // slice, the columns of its first pair, its number of pairs}.  Offsets are in 16-byte units.
+//
+// The tensor-core flavour (mma = 1, fp16 weights, g = 8 or 16) keeps the same slices and row
+// headers but stores a segment as "step records" of 16 blocks each: the 16 chunk-local columns
+// (uint16), then per 8 output channels the 16x8 weight tile in the register order of the
+// m16n8k16 B operand.  The blocks of a segment are ordered so that the 8 columns of each half step
+// differ modulo 8 wherever the segment allows it (their shared-memory rows then lie in different
+// banks); missing blocks are zero-weight padding.  A row header is {segment start, steps, 0, 0}.
 struct Schedule {
     int kc = 0, nch = 0, n_rg = 0, rpg = 0;
+    int mma = 0;                   // 1: step records for the tensor-core kernels
     int ros = 0;                   // ints per (row group, chunk) row of rowoff: 4 per local row
     int wcap = 0;                  // longest slice, in 16-byte units
     int n_rec = 0;                 // total length of all slices, in 16-byte units
@@ -66,11 +74,11 @@ struct Plan {
 struct ShapeKey {
     int n, h, wd;
     unsigned flags;
-    int c[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
+    int c[10] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
     bool operator<(const ShapeKey& o) const {
         if (std::tie(n, h, wd, flags) != std::tie(o.n, o.h, o.wd, o.flags))
             return std::tie(n, h, wd, flags) < std::tie(o.n, o.h, o.wd, o.flags);
-        for (int i = 0; i < 9; ++i)
+        for (int i = 0; i < 10; ++i)
             if (c[i] != o.c[i]) return c[i] < o.c[i];
         return false;
     }
@@ -89,7 +97,8 @@ struct alcs_packed {
     int* d_err = nullptr;             // device error word written by a kernel whose bounded wait ran out
     mutable void* d_xpad = nullptr;   // scratch: X repacked to 16-byte aligned rows (grown on demand)
     mutable size_t xpad_bytes = 0;
-    mutable std::map<std::pair<int, int>, alcs::Schedule> sched;   // by (kc, n_rg), built on demand
+    // by (kc, n_rg), built on demand; the tensor-core flavour of a schedule is stored under -kc
+    mutable std::map<std::pair<int, int>, alcs::Schedule> sched;
     std::map<alcs::ShapeKey, alcs_launch_cfg> tuned;   // filled by alcs_spconv1x1_tune
     mutable std::map<alcs::ShapeKey, alcs::Plan> plan_cache;   // resolved plans, by shape
     mutable std::mutex mu;                                      // guards plan_cache and sched
@@ -101,6 +110,10 @@ namespace alcs {
 // Host-side helpers implemented in alcs_pack.cpp (no CUDA).
 float half_bits_to_float(uint16_t h);
 void build_schedule(const alcs_packed& p, int kc, int n_rg, bool with_records, Schedule& out);
+void build_schedule_mma(const alcs_packed& p, int kc, int n_rg, bool with_records, Schedule& out);
+inline std::pair<int, int> sched_key(int kc, int n_rg, int mma) { return std::make_pair(mma ? -kc : kc, n_rg); }
+// bytes of one step record of the tensor-core flavour
+constexpr int step_record_bytes(int g) { return 32 + 32 * (g < 8 ? 8 : g); }
 
 }  // namespace alcs
 

@@ -374,12 +374,13 @@ __device__ __forceinline__ void store_one(YT* p, float v)
 // ---- producer: one warp copies (item, chunk) after (item, chunk) into the ring ---------------
 // LDB = bytes per X copy.  Each lane owns NCOL fixed pixel vectors of the tile and walks the
 // channels of the chunk, so its source pointers are computed once per item.
-template <typename XT, int G, int P, int LDB>
+// XPAD = bytes of padding after each channel row of the tile in shared memory.
+template <typename XT, int G, int P, int LDB, int XPAD = 0>
 __device__ __forceinline__ void produce(const ConvArgs& a, unsigned char* smem, int lane, int pw, int npw)
 {
     constexpr int T = 32 * P;
     constexpr int SZ = (int)sizeof(XT);
-    constexpr int ROWB = T * SZ;
+    constexpr int ROWB = T * SZ + XPAD;
     constexpr int EV = LDB / SZ;            // elements per copy
     constexpr int VPR = T / EV;             // copies per channel row
     constexpr int NCOL = VPR >= 32 ? VPR / 32 : 1;   // copies per channel row per lane
@@ -466,12 +467,12 @@ __device__ __forceinline__ void produce(const ConvArgs& a, unsigned char* smem, 
 // split where the tile crosses from one image into the next); the lanes of the producer warp
 // share the channel rows of the chunk.  Lane 0 announces the chunk's byte count on the "full"
 // mbarrier, which completes when all of them have landed.
-template <typename XT, int G, int P>
+template <typename XT, int G, int P, int XPAD = 0>
 __device__ __forceinline__ void produce_bulk(const ConvArgs& a, unsigned char* smem, int lane, int pw, int npw)
 {
     constexpr int T = 32 * P;
     constexpr int SZ = (int)sizeof(XT);
-    constexpr int ROWB = T * SZ;
+    constexpr int ROWB = T * SZ + XPAD;
     const size_t ch_bytes = (size_t)a.hw * SZ;
     const uint32_t smem_u32 = (uint32_t)__cvta_generic_to_shared(smem);
     const uint32_t ring = smem_u32 + 16 * kMaxStages;
@@ -692,19 +693,22 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_kernel(const 
 }
 
 // One entry of the table of compiled kernel variants.
+// mma = 1: the tensor-core kernel (fp16 only), which takes the step-record flavour of the schedule.
 struct KernelVariant {
     int is_f16, g, p, rw, nw, minb, npw;
     const void* fn;
+    int mma;
 };
 
 #define ALCS_VARIANT_P(XT, ISF16, G, P, RW, NW, MINB, NPW) \
-    {ISF16, G, P, RW, NW, MINB, NPW, (const void*)&spconv1x1_kernel<XT, G, P, RW, NW, MINB, NPW>}
+    {ISF16, G, P, RW, NW, MINB, NPW, (const void*)&spconv1x1_kernel<XT, G, P, RW, NW, MINB, NPW>, 0}
 #define ALCS_VARIANT(XT, ISF16, G, P, RW, NW, MINB) ALCS_VARIANT_P(XT, ISF16, G, P, RW, NW, MINB, 1)
 
 // Defined one per translation unit, concatenated by alcs_device.cu.
 const KernelVariant* variants_f32_g4(int* n);
 const KernelVariant* variants_f32_other(int* n);
 const KernelVariant* variants_f16(int* n);
+const KernelVariant* variants_f16_mma(int* n);
 
 }  // namespace alcs
 

@@ -156,6 +156,137 @@ void build_schedule(const alcs_packed& p, int kc, int n_rg, bool with_records, S
     out.wcap = wcap;
 }
 
+// Tensor-core flavour of the schedule (fp16 weights): see the comment on Schedule.
+void build_schedule_mma(const alcs_packed& p, int kc, int n_rg, bool with_records, Schedule& out)
+{
+    if (kc <= 0 || kc > p.cin) kc = p.cin;
+    const int R = p.rows, g = p.g;
+    const int gp = g < 8 ? 8 : g;                 // output channels per block after padding to an 8-wide tile
+    n_rg = std::max(1, std::min(n_rg, R));
+    const int nch = (p.cin + kc - 1) / kc;
+    const int rpg = (R + n_rg - 1) / n_rg;
+    const int REC = step_record_bytes(g);
+    out.kc = kc; out.nch = nch; out.n_rg = n_rg; out.rpg = rpg; out.mma = 1;
+
+    std::vector<int> order(R);
+    std::iota(order.begin(), order.end(), 0);
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+        return p.row_ptr[a + 1] - p.row_ptr[a] > p.row_ptr[b + 1] - p.row_ptr[b];
+    });
+    out.h_rowmap.assign((size_t)n_rg * rpg, -1);
+    for (int i = 0; i < R; ++i) {
+        const int t = i / n_rg, j = i % n_rg;
+        const int rg = (t & 1) ? n_rg - 1 - j : j;
+        out.h_rowmap[(size_t)rg * rpg + t] = order[i];
+    }
+
+    out.h_slice.assign((size_t)n_rg * nch + 1, 0);
+    const int ros = rpg * 4;
+    out.ros = ros;
+    out.h_rowoff.assign((size_t)n_rg * nch * ros, 0);
+    out.h_rec.clear();
+    std::vector<int> cursor(R);
+    int rec_count = 0, wcap = 0;
+    std::vector<int> slot;                         // slot -> index into col_idx, or -1 - column for padding
+    for (int rg = 0; rg < n_rg; ++rg) {
+        for (int t = 0; t < rpg; ++t) {
+            const int r = out.h_rowmap[(size_t)rg * rpg + t];
+            if (r >= 0) cursor[r] = p.row_ptr[r];
+        }
+        for (int c = 0; c < nch; ++c) {
+            out.h_slice[(size_t)rg * nch + c] = rec_count;
+            int* roff = &out.h_rowoff[((size_t)rg * nch + c) * ros];
+            const int c0 = c * kc;
+            const int lim = c0 + kc;
+            const int nrows = std::min(kc, p.cin - c0);      // channels present in this chunk
+            int local = 0;
+            for (int t = 0; t < rpg; ++t) {
+                int* hd = roff + 4 * t;                      // {segment start (16-byte units), steps, 0, 0}
+                hd[0] = local; hd[1] = hd[2] = hd[3] = 0;
+                const int r = out.h_rowmap[(size_t)rg * rpg + t];
+                if (r < 0) continue;
+                const int k = cursor[r];
+                const int kend = p.row_ptr[r + 1];
+                int k1 = k;
+                while (k1 < kend && p.col_idx[k1] < lim) ++k1;
+                const int nblk = k1 - k;
+                const int nstep = (nblk + 15) / 16;
+                hd[1] = nstep;
+                cursor[r] = k1;
+                if (!nstep) continue;
+                if (with_records) {
+                    // deal the blocks to the 2*nstep half steps: members of one residue class (column
+                    // modulo 8) are spread over the half steps as evenly as the room allows
+                    const int noct = 2 * nstep;
+                    slot.assign((size_t)noct * 8, 0);
+                    std::vector<int> fill(noct, 0);
+                    std::vector<int> has((size_t)noct * 8, 0);            // [half step][residue] count
+                    std::vector<int> cls[8];
+                    for (int kk = k; kk < k1; ++kk) cls[(p.col_idx[kk] - c0) & 7].push_back(kk);
+                    int cord[8] = {0, 1, 2, 3, 4, 5, 6, 7};
+                    std::stable_sort(cord, cord + 8, [&](int a, int b) { return cls[a].size() > cls[b].size(); });
+                    for (int ci = 0; ci < 8; ++ci) {
+                        const int res = cord[ci];
+                        for (int kk : cls[res]) {
+                            int best = -1;
+                            for (int o = 0; o < noct; ++o) {
+                                if (fill[o] >= 8) continue;
+                                if (best < 0 || has[(size_t)o * 8 + res] < has[(size_t)best * 8 + res] ||
+                                    (has[(size_t)o * 8 + res] == has[(size_t)best * 8 + res] && fill[o] < fill[best]))
+                                    best = o;
+                            }
+                            slot[(size_t)best * 8 + fill[best]++] = kk;
+                            ++has[(size_t)best * 8 + res];
+                        }
+                    }
+                    for (int o = 0; o < noct; ++o) {
+                        while (fill[o] < 8) {       // padding: a zero-weight block on a column whose residue is free
+                            int col = 0;
+                            for (int res = 0; res < 8; ++res)
+                                if (!has[(size_t)o * 8 + res] && res < nrows) { col = res; break; }
+                            ++has[(size_t)o * 8 + (col & 7)];
+                            slot[(size_t)o * 8 + fill[o]++] = -1 - col;
+                        }
+                    }
+                    const size_t base = out.h_rec.size();
+                    out.h_rec.resize(base + (size_t)nstep * REC, 0);
+                    for (int s = 0; s < nstep; ++s) {
+                        unsigned char* rec = &out.h_rec[base + (size_t)s * REC];
+                        uint16_t cols[16];
+                        uint16_t wv[16][16];                 // [column of the step][output channel of the block]
+                        std::memset(wv, 0, sizeof wv);
+                        for (int i = 0; i < 16; ++i) {
+                            const int e = slot[(size_t)s * 16 + i];
+                            if (e < 0) { cols[i] = (uint16_t)(-1 - e); continue; }
+                            cols[i] = (uint16_t)(p.col_idx[e] - c0);
+                            std::memcpy(wv[i], &p.vals[(size_t)e * g * 2], (size_t)g * 2);
+                        }
+                        std::memcpy(rec, cols, 32);
+                        // B operand of m16n8k16, per tile of 8 output channels: lane l = 4*n + t holds
+                        // W[2t][n], W[2t+1][n], W[2t+8][n], W[2t+9][n]
+                        for (int nb = 0; nb < gp / 8; ++nb) {
+                            uint16_t* frag = reinterpret_cast<uint16_t*>(rec + 32 + nb * 256);
+                            for (int l = 0; l < 32; ++l) {
+                                const int n = nb * 8 + (l >> 2), tq = l & 3;
+                                frag[l * 4 + 0] = wv[2 * tq][n];
+                                frag[l * 4 + 1] = wv[2 * tq + 1][n];
+                                frag[l * 4 + 2] = wv[2 * tq + 8][n];
+                                frag[l * 4 + 3] = wv[2 * tq + 9][n];
+                            }
+                        }
+                    }
+                }
+                local += nstep * (REC / 16);
+            }
+            rec_count += local;
+            wcap = std::max(wcap, local);
+        }
+    }
+    out.h_slice[(size_t)n_rg * nch] = rec_count;
+    out.n_rec = rec_count;
+    out.wcap = wcap;
+}
+
 }  // namespace alcs
 
 extern "C" {

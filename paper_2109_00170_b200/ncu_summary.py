@@ -79,7 +79,7 @@ def main():
     nl = len(layers)
     # A layer whose X rows are not a multiple of 16 bytes launches the row-repacking kernel first;
     # that launch is counted with the convolution that follows it.
-    n_conv = sum(1 for name, _ in launches if "spconv1x1_kernel" in name)
+    n_conv = sum(1 for name, _ in launches if "spconv1x1_" in name)
     if not n_conv or n_conv % nl:
         sys.exit(f"{n_conv} convolution launches do not divide into {nl} layers")
     reps = n_conv // nl
@@ -94,7 +94,7 @@ def main():
         per_kernel[short][0] += 1
         per_kernel[short][1] += t
         L = per_layer[i % nl]
-        if "spconv1x1_kernel" in name:
+        if "spconv1x1_" in name:
             i += 1
         L["t"] += t / reps
         L["rd"] += m.get("dram__bytes_read.sum", 0.0) / reps

@@ -165,10 +165,13 @@ ALCS_API void alcs_packed_free(alcs_packed* p);
  *                     only): 16 kept blocks of a block row times the 16 input rows they select is a
  *                     dense 16 x g by 16 x pixels contraction, run as warp-level MMA with fp32
  *                     accumulation
+ *   consumer_groups   1 = all consumer warps work on one work item at a time; 2 = two halves of the
+ *                     consumer warps take the thread block's work items alternately (tensor-core
+ *                     kernels only), so that one half multiplies while the other half stores
  */
 typedef struct {
     int pixels_per_lane, rows_per_warp, warps, chunk_channels, stages, row_groups, min_blocks, copy_mode,
-        producer_warps, math_mode;
+        producer_warps, math_mode, consumer_groups;
 } alcs_launch_cfg;
 
 /*

@@ -42,7 +42,7 @@ class AlcsError(RuntimeError):
 class LaunchCfg(C.Structure):
     _fields_ = [(k, C.c_int) for k in ("pixels_per_lane", "rows_per_warp", "warps",
                                        "chunk_channels", "stages", "row_groups", "min_blocks", "copy_mode",
-                                       "producer_warps", "math_mode")]
+                                       "producer_warps", "math_mode", "consumer_groups")]
 
     def as_dict(self):
         return {k: getattr(self, k) for k, _ in self._fields_}

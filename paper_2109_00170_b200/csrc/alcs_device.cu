@@ -191,7 +191,7 @@ double model_cost(const alcs_packed* w, const KernelVariant& v, const Schedule& 
         const double l2b = ((double)w->cin * T * elt + steps_item * alcs::step_record_bytes(v.g)) / (16.0 * v.npw);
         const double warps = (double)v.nw * occ;
         const double hide = std::min(1.0, 0.4 + warps / 20.0);
-        const double item_cycles = std::max(std::max(issue, lsu) / hide, l2b) + 2500.0;
+        const double item_cycles = (std::max(std::max(issue, lsu) / hide, l2b) + 2500.0) * (v.groups == 2 && rounds > 1 ? 0.7 : 1.0);
         const double t_sm = (double)rounds * occ * item_cycles / 1.9e9;
         const double bytes = (double)q * (w->cin + w->cout) * elt;
         return std::max(t_sm, bytes / 6.0e12);
@@ -240,7 +240,7 @@ int enumerate_plans(const alcs_packed* w, long long q, int hw, std::vector<Plan>
         if (v.is_f16 != (w->dt == ALCS_F16) || v.g != w->g) continue;
         rc = prepare_variant(g_variants[vi]);
         if (rc) return rc;
-        const int cap = v.nw * v.rw;
+        const int cap = v.nw / v.groups * v.rw;
         const int rg_min = (w->rows + cap - 1) / cap;
         int last_kc = -1;
         for (int ci = 0; ci < alcs::kNumChunkings; ++ci) {
@@ -264,6 +264,7 @@ int enumerate_plans(const alcs_packed* w, long long q, int hw, std::vector<Plan>
                 if (!sc) return ALCS_ERR_ALLOC;
                 const StageLayout L = stage_layout(v, *sc, elt);
                 for (int stages = 2; stages <= alcs::kMaxStages; ++stages) {
+                    if (stages % v.groups) continue;        // every consumer group gets the same share of the ring
                     const size_t smem = plan_smem(L, stages);
                     if (smem > (size_t)smem_max) break;
                     const int occ = occupancy_of(g_variants[vi], smem);
@@ -306,6 +307,7 @@ void plan_to_cfg(const Plan& p, alcs_launch_cfg* c)
     c->copy_mode = p.bulk ? 2 : 1;
     c->producer_warps = v.npw;
     c->math_mode = v.mma ? 2 : 1;
+    c->consumer_groups = v.groups;
 }
 
 // Resolve a (possibly partial) configuration into a concrete plan.
@@ -323,6 +325,7 @@ int cfg_to_plan(const alcs_packed* w, long long q, int hw, const alcs_launch_cfg
         if (c->min_blocks && c->min_blocks != v.minb) return false;
         if (c->producer_warps && c->producer_warps != v.npw) return false;
         if (c->math_mode && (c->math_mode == 2) != (v.mma == 1)) return false;
+        if (c->consumer_groups && c->consumer_groups != v.groups) return false;
         if (c->chunk_channels && std::min(c->chunk_channels, w->cin) != p.kc) return false;
         if (c->stages && c->stages != p.stages) return false;
         if (c->copy_mode && (c->copy_mode == 2) != (p.bulk == 1)) return false;
@@ -339,7 +342,7 @@ int cfg_to_plan(const alcs_packed* w, long long q, int hw, const alcs_launch_cfg
             if (!variant_ok(p0)) continue;
             const KernelVariant& v = g_variants[p0.variant].v;
             const int rpg = (w->rows + c->row_groups - 1) / c->row_groups;
-            if (rpg > v.nw * v.rw) continue;
+            if (rpg > v.nw / v.groups * v.rw) continue;
             const Schedule* sc = get_schedule(w, p0.kc, c->row_groups, false, v.mma);
             if (!sc) return ALCS_ERR_ALLOC;
             Plan p = p0;
@@ -513,10 +516,10 @@ int resolve_plan(const alcs_packed* w, int n, int h, int wd, unsigned flags, lon
 {
     alcs::ShapeKey key{n, h, wd, flags};
     if (cfg) {
-        const int c[10] = {cfg->pixels_per_lane, cfg->rows_per_warp, cfg->warps, cfg->chunk_channels,
+        const int c[11] = {cfg->pixels_per_lane, cfg->rows_per_warp, cfg->warps, cfg->chunk_channels,
                            cfg->stages, cfg->row_groups, cfg->min_blocks, cfg->copy_mode, cfg->producer_warps,
-                           cfg->math_mode};
-        for (int i = 0; i < 10; ++i) key.c[i] = c[i];
+                           cfg->math_mode, cfg->consumer_groups};
+        for (int i = 0; i < 11; ++i) key.c[i] = c[i];
     }
     {
         std::lock_guard<std::mutex> lk(w->mu);
@@ -626,6 +629,7 @@ ALCS_API int alcs_variant_get(int index, alcs_dtype* dt, int* g, alcs_launch_cfg
         cfg->copy_mode = 0;
         cfg->producer_warps = v.npw;
         cfg->math_mode = v.mma ? 2 : 1;
+        cfg->consumer_groups = v.groups;
     }
     return ALCS_OK;
 }

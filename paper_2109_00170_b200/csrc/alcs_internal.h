@@ -74,11 +74,11 @@ struct Plan {
 struct ShapeKey {
     int n, h, wd;
     unsigned flags;
-    int c[10] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+    int c[11] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
     bool operator<(const ShapeKey& o) const {
         if (std::tie(n, h, wd, flags) != std::tie(o.n, o.h, o.wd, o.flags))
             return std::tie(n, h, wd, flags) < std::tie(o.n, o.h, o.wd, o.flags);
-        for (int i = 0; i < 10; ++i)
+        for (int i = 0; i < 11; ++i)
             if (c[i] != o.c[i]) return c[i] < o.c[i];
         return false;
     }

@@ -375,7 +375,10 @@ __device__ __forceinline__ void store_one(YT* p, float v)
 // LDB = bytes per X copy.  Each lane owns NCOL fixed pixel vectors of the tile and walks the
 // channels of the chunk, so its source pointers are computed once per item.
 // XPAD = bytes of padding after each channel row of the tile in shared memory.
-template <typename XT, int G, int P, int LDB, int XPAD = 0>
+// GR = consumer groups: with 2, the items of the thread block belong alternately to group 0 and
+// group 1, and each group has its own half of the ring (stages and barriers), so that a barrier
+// is only ever used by one group, one phase after the other.
+template <typename XT, int G, int P, int LDB, int XPAD = 0, int GR = 1>
 __device__ __forceinline__ void produce(const ConvArgs& a, unsigned char* smem, int lane, int pw, int npw)
 {
     constexpr int T = 32 * P;
@@ -391,9 +394,10 @@ __device__ __forceinline__ void produce(const ConvArgs& a, unsigned char* smem, 
     const size_t ch_bytes = (size_t)a.hw * SZ;
     const uint32_t smem_u32 = (uint32_t)__cvta_generic_to_shared(smem);
     const uint32_t ring = smem_u32 + 16 * kMaxStages;
-    const int S = a.stages;
+    const int S = a.stages / GR;            // stages of one group's ring
     const int items = a.n_tiles * a.n_rg;
-    int kk = 0;                             // running (item, chunk) counter = ring position
+    int kk = 0;                             // running (item, chunk) counter = position in the group's ring
+    int kk_other = 0, turn = 0;             // (GR == 2) the other group's counter; whose item this is
 
     bool dep_ok = false;                    // has the predecessor kernel been waited for yet?
     for (int item = blockIdx.x; item < items; item += gridDim.x) {
@@ -414,7 +418,7 @@ __device__ __forceinline__ void produce(const ConvArgs& a, unsigned char* smem, 
         const int* rowoff = a.rowoff + (size_t)rg * a.nch * a.ros;
 
         for (int k = 0; k < a.nch; ++k, ++kk) {
-            const int s = kk % S;
+            const int s = turn * S + kk % S;
             if (kk >= S) {                  // wait until the consumers have released this stage
                 if (!mbar_wait(smem_u32 + 8 * kMaxStages + 8 * s, ((kk / S) - 1) & 1)) {
                     if (lane == 0) atomicExch(a.err, kErrEmptyWait);
@@ -457,6 +461,10 @@ __device__ __forceinline__ void produce(const ConvArgs& a, unsigned char* smem, 
             if constexpr (LDB == 2) __threadfence_block();
             mbar_arrive_on_copies(smem_u32 + 8 * s);      // "full" completes when all producer lanes' copies land
         }
+        if constexpr (GR == 2) {            // the next item is the other group's
+            const int t = kk; kk = kk_other; kk_other = t;
+            turn ^= 1;
+        }
     }
     cp_async_wait_all();
 }
@@ -467,7 +475,7 @@ __device__ __forceinline__ void produce(const ConvArgs& a, unsigned char* smem, 
 // split where the tile crosses from one image into the next); the lanes of the producer warp
 // share the channel rows of the chunk.  Lane 0 announces the chunk's byte count on the "full"
 // mbarrier, which completes when all of them have landed.
-template <typename XT, int G, int P, int XPAD = 0>
+template <typename XT, int G, int P, int XPAD = 0, int GR = 1>
 __device__ __forceinline__ void produce_bulk(const ConvArgs& a, unsigned char* smem, int lane, int pw, int npw)
 {
     constexpr int T = 32 * P;
@@ -476,9 +484,10 @@ __device__ __forceinline__ void produce_bulk(const ConvArgs& a, unsigned char* s
     const size_t ch_bytes = (size_t)a.hw * SZ;
     const uint32_t smem_u32 = (uint32_t)__cvta_generic_to_shared(smem);
     const uint32_t ring = smem_u32 + 16 * kMaxStages;
-    const int S = a.stages;
+    const int S = a.stages / GR;            // stages of one group's ring
     const int items = a.n_tiles * a.n_rg;
     int kk = 0;
+    int kk_other = 0, turn = 0;             // (GR == 2) the other group's counter; whose item this is
 
     bool dep_ok = false;                    // has the predecessor kernel been waited for yet?
     for (int item = blockIdx.x; item < items; item += gridDim.x) {
@@ -493,7 +502,7 @@ __device__ __forceinline__ void produce_bulk(const ConvArgs& a, unsigned char* s
         const int* rowoff = a.rowoff + (size_t)rg * a.nch * a.ros;
 
         for (int k = 0; k < a.nch; ++k, ++kk) {
-            const int s = kk % S;
+            const int s = turn * S + kk % S;
             if (kk >= S) {
                 if (!mbar_wait(smem_u32 + 8 * kMaxStages + 8 * s, ((kk / S) - 1) & 1)) {
                     if (lane == 0) atomicExch(a.err, kErrEmptyWait);
@@ -533,11 +542,17 @@ __device__ __forceinline__ void produce_bulk(const ConvArgs& a, unsigned char* s
 
             }
         }
+        if constexpr (GR == 2) {            // the next item is the other group's
+            const int t = kk; kk = kk_other; kk_other = t;
+            turn ^= 1;
+        }
     }
 drain:
     // Do not leave while copies of this warp may still be landing: wait (bounded) for the last
     // fills of every stage.
-    for (int j = max(0, kk - S); j < kk; ++j) mbar_wait(smem_u32 + 8 * (j % S), (j / S) & 1);
+    for (int j = max(0, kk - S); j < kk; ++j) mbar_wait(smem_u32 + 8 * (turn * S + j % S), (j / S) & 1);
+    if constexpr (GR == 2)
+        for (int j = max(0, kk_other - S); j < kk_other; ++j) mbar_wait(smem_u32 + 8 * ((turn ^ 1) * S + j % S), (j / S) & 1);
 }
 
 template <typename XT, int G, int P, int RW, int NW, int MINB, int NPW>
@@ -698,10 +713,11 @@ struct KernelVariant {
     int is_f16, g, p, rw, nw, minb, npw;
     const void* fn;
     int mma;
+    int groups;     // consumer groups that take the items of a thread block in turn (1 or 2); nw counts all consumer warps
 };
 
 #define ALCS_VARIANT_P(XT, ISF16, G, P, RW, NW, MINB, NPW) \
-    {ISF16, G, P, RW, NW, MINB, NPW, (const void*)&spconv1x1_kernel<XT, G, P, RW, NW, MINB, NPW>, 0}
+    {ISF16, G, P, RW, NW, MINB, NPW, (const void*)&spconv1x1_kernel<XT, G, P, RW, NW, MINB, NPW>, 0, 1}
 #define ALCS_VARIANT(XT, ISF16, G, P, RW, NW, MINB) ALCS_VARIANT_P(XT, ISF16, G, P, RW, NW, MINB, 1)
 
 // Defined one per translation unit, concatenated by alcs_device.cu.

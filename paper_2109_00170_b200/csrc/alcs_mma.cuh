@@ -94,10 +94,16 @@ __device__ __forceinline__ uint32_t pack_half2(float lo, float hi)
     return *reinterpret_cast<const uint32_t*>(&h);
 }
 
-template <int G, int P, int RW, int NW, int NPW, int MINB>
+// GR = 1: all NW consumer warps work on the same item.  GR = 2: two groups of NW/2 warps take the
+// items of the thread block alternately, so that one group's multiply phase (shared-memory bound)
+// runs while the other group is in its epilogue (store bound) and the producers stream ahead for
+// both; each group has its own half of the ring's stages and barriers.
+template <int G, int P, int RW, int NW, int NPW, int MINB, int GR>
 __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_mma_kernel(const ConvArgs a)
 {
     static_assert(P == 4 || P == 8, "a lane stores runs of 4 or 8 pixels");
+    static_assert(GR == 1 || (GR == 2 && NW % 2 == 0), "one or two consumer groups");
+    constexpr int NWG = NW / GR;                      // consumer warps per group
     constexpr int T = 32 * P;
     constexpr int MT = 2 * P;
     constexpr int GP = G < 8 ? 8 : G;
@@ -117,7 +123,7 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_mma_kernel(co
     if (tid == 0) {
         for (int s = 0; s < S; ++s) {
             mbar_init(smem_u32 + 8 * s, a.bulk ? 1 : 32 * NPW);
-            mbar_init(smem_u32 + 8 * kMaxStages + 8 * s, NW);
+            mbar_init(smem_u32 + 8 * kMaxStages + 8 * s, NWG);
         }
     }
     __syncthreads();
@@ -126,14 +132,14 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_mma_kernel(co
     if (warp >= NW) {   // ---- producer warps ------------------------------------------------
         const int pw = warp - NW;
         if (a.bulk) {
-            produce_bulk<__half, G, P, kMmaXPad>(a, smem, lane, pw, NPW);
+            produce_bulk<__half, G, P, kMmaXPad, GR>(a, smem, lane, pw, NPW);
             return;
         }
         switch (a.ld_bytes) {
-            case 16: produce<__half, G, P, 16, kMmaXPad>(a, smem, lane, pw, NPW); break;
-            case 8: produce<__half, G, P, 8, kMmaXPad>(a, smem, lane, pw, NPW); break;
-            case 4: produce<__half, G, P, 4, kMmaXPad>(a, smem, lane, pw, NPW); break;
-            default: produce<__half, G, P, 2, kMmaXPad>(a, smem, lane, pw, NPW); break;
+            case 16: produce<__half, G, P, 16, kMmaXPad, GR>(a, smem, lane, pw, NPW); break;
+            case 8: produce<__half, G, P, 8, kMmaXPad, GR>(a, smem, lane, pw, NPW); break;
+            case 4: produce<__half, G, P, 4, kMmaXPad, GR>(a, smem, lane, pw, NPW); break;
+            default: produce<__half, G, P, 2, kMmaXPad, GR>(a, smem, lane, pw, NPW); break;
         }
         return;
     }
@@ -144,9 +150,13 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_mma_kernel(co
     const unsigned char* scratch = smem + scr_off;
     const int items = a.n_tiles * a.n_rg;
     const int gid = lane >> 2, tig = lane & 3;
+    const int grp = warp / NWG, wg = warp - grp * NWG;
     int kk = 0;
+    int turn = 0;
 
-    for (int item = blockIdx.x; item < items; item += gridDim.x) {
+    const int SG = S / GR;                  // stages of this group's half of the ring
+    for (int item = blockIdx.x; item < items; item += gridDim.x, turn ^= 1) {
+        if (GR == 2 && turn != grp) continue;       // the other group's item
         const int tile = item / a.n_rg;
         const int rg = item - tile * a.n_rg;
         const int q0 = tile * T;
@@ -155,7 +165,7 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_mma_kernel(co
         float2 bz[RW][NB];          // bias of the two channels this lane holds in an accumulator tile
 #pragma unroll
         for (int s = 0; s < RW; ++s) {
-            lrow[s] = s * NW + ((s & 1) ? NW - 1 - warp : warp);
+            lrow[s] = s * NWG + ((s & 1) ? NWG - 1 - wg : wg);
             rowid[s] = lrow[s] < a.rpg ? __ldg(a.rowmap + rg * a.rpg + lrow[s]) : -1;
 #pragma unroll
             for (int nb = 0; nb < NB; ++nb) {
@@ -178,8 +188,8 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_mma_kernel(co
                     for (int e = 0; e < 4; ++e) c[s][mt][nb][e] = 0.0f;
 
         for (int k = 0; k < a.nch; ++k, ++kk) {
-            const int st = kk % S;
-            if (!mbar_wait(smem_u32 + 8 * st, (kk / S) & 1)) {
+            const int st = grp * SG + kk % SG;
+            if (!mbar_wait(smem_u32 + 8 * st, (kk / SG) & 1)) {
                 if (lane == 0) atomicExch(a.err, kErrFullWait);
                 return;
             }
@@ -303,8 +313,8 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_mma_kernel(co
     }
 }
 
-#define ALCS_MMA_VARIANT(G, P, RW, NW, NPW, MINB) \
-    {1, G, P, RW, NW, MINB, NPW, (const void*)&spconv1x1_mma_kernel<G, P, RW, NW, NPW, MINB>, 1}
+#define ALCS_MMA_VARIANT(G, P, RW, NW, NPW, MINB, GR) \
+    {1, G, P, RW, NW, MINB, NPW, (const void*)&spconv1x1_mma_kernel<G, P, RW, NW, NPW, MINB, GR>, 1, GR}
 
 }  // namespace alcs
 

@@ -181,7 +181,7 @@ def test_every_kernel_variant(alcs, g, dtype):
             for stages in (2, 3, 4):
                 cfg = dict(pixels_per_lane=v["pixels_per_lane"], rows_per_warp=v["rows_per_warp"],
                            warps=v["warps"], min_blocks=v["min_blocks"], producer_warps=v["producer_warps"],
-                           math_mode=v["math_mode"], chunk_channels=kc,
+                           math_mode=v["math_mode"], consumer_groups=v["consumer_groups"], chunk_channels=kc,
                            stages=stages, row_groups=0)
                 try:
                     Y = run_gpu(alcs, W, M, X, b, True, g, cfg=cfg, packed=p)

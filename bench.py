@@ -464,7 +464,7 @@ def main():
     else:
         ach = stats[dom]["flops"] / (per_layer_ms[dom] * 1e-3) / 1e12
         roof = {"bound": "alu", "achieved": ach, "peak": fp32_tf, "unit": "TFLOP/s", "frac": ach / fp32_tf}
-    roof.update({"traffic": stored_traffic(d["layer"], d["cfg"]), "kernel": "spconv1x1_kernel", "layer": d["layer"],
+    roof.update({"traffic": stored_traffic(d["layer"], d["cfg"]), "kernel": "spconv1x1_mma_kernel" if d["cfg"].get("math_mode") == 2 else "spconv1x1_kernel", "layer": d["layer"],
                  "algorithmic_bytes": stats[dom]["bytes"], "algorithmic_flops": stats[dom]["flops"],
                  "peak_source": f"HBM {peak_src}; fp32 = {SM_COUNT} SMs x {FP32_LANES} lanes x 2 x {sm_max:.0f} MHz"})
     sum_roof = sum(r["t_roof_us"] for r in rows)

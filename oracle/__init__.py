@@ -1,9 +1,9 @@
-"""CPU oracle of the SIMD-structured sparse pointwise convolution and of its storage format.
+"""CPU oracle of the SIMD-structured sparse convolution (pointwise and general k x k) and of its storage format.
 
 TEST INFRASTRUCTURE ONLY.  Nothing in the product package imports this; only tests, the smoke
 check and the benchmark's CPU-baseline leg do.  It shares no code with the CUDA path.
 """
-from .conv import conv1x1, conv1x1_points, num_threads
+from .conv import conv1x1, conv1x1_points, conv2d, conv2d_points, num_threads
 from .storage import flatten, pack, unpack
 
-__all__ = ["conv1x1", "conv1x1_points", "num_threads", "pack", "unpack", "flatten"]
+__all__ = ["conv1x1", "conv1x1_points", "conv2d", "conv2d_points", "num_threads", "pack", "unpack", "flatten"]

@@ -1,5 +1,6 @@
 /*
- * CPU oracle for the SIMD-structured sparse pointwise convolution.
+ * CPU oracle for the SIMD-structured sparse convolution (pointwise first, general k x k at
+ * the end of the file).
  *
  * TEST INFRASTRUCTURE ONLY: the library under test never calls this file; only the tests,
  * the smoke check and the benchmark's CPU-baseline leg may.  It shares no code with the
@@ -170,6 +171,116 @@ int oracle_conv1x1_points(const void *W, const uint8_t *mask, int g, const void 
         }
         const double b = bias ? (double)bias[co] : 0.0;
         s += b;
+        if (relu && s < 0.0) s = 0.0;
+        out[k] = s;
+        if (mag) mag[k] = m + fabs(b);
+    }
+    return bad ? -1 : 0;
+}
+
+/* ------------------------------------------------------------------------------------------
+ * General k_h x k_w convolution: the same Section 3.2.2 formula with all three sums,
+ *
+ *     O(co, oh, ow) = sum_c sum_r sum_s Wm(co, c, r, s) * I(c, oh*stride - pad + r, ow*stride - pad + s),
+ *
+ * where I is read as zero outside the image.  The paper writes the stride-1, unpadded case
+ * (I(c, h+r, w+s)); stride and zero padding are what the ResNet / MobileNet layers add and
+ * reduce to the paper's formula at stride = 1, pad = 0.  The pruning pattern is the one of
+ * Section 3.2.1 for a general kernel: the parameters at the same location (c, r, s) of g
+ * adjacent filters form one group, so the block mask is [ceil(cout/g)][cin*kh*kw] over the
+ * columns of the flattened-filter matrix W*, column = (c*kh + r)*kw + s.
+ *
+ * As above: dense loops over the mask-applied weights, no zero skipping, double accumulation
+ * in ascending (c, r, s) order, then bias and ReLU.  W is [cout][cin][kh][kw], X is
+ * [n][cin][h][wd], Y and A are [n][cout][oh][ow] with oh = (h + 2*pad - kh)/stride + 1.
+ */
+static inline double conv2d_point(const void *W, const uint8_t *mask, int g, const void *X,
+                                  int is_f16, int cin, int cout, int h, int wd, int kh, int kw,
+                                  int stride, int pad, int in, int co, int oh, int ow, double *mag)
+{
+    const int K = cin * kh * kw;
+    double s = 0.0, m = 0.0;
+    for (int c = 0; c < cin; ++c)
+        for (int r = 0; r < kh; ++r)
+            for (int q = 0; q < kw; ++q) {
+#if ORACLE_MUTANT == 6            /* flipped kernel: true convolution instead of the paper's h+r, w+s */
+                const int ih = oh * stride - pad + (kh - 1 - r), iw = ow * stride - pad + (kw - 1 - q);
+#elif ORACLE_MUTANT == 7          /* taps transposed: r walks the width, s the height */
+                const int ih = oh * stride - pad + q, iw = ow * stride - pad + r;
+#elif ORACLE_MUTANT == 8          /* stride applied to the taps as well */
+                const int ih = (oh + r) * stride - pad, iw = (ow + q) * stride - pad;
+#elif ORACLE_MUTANT == 9          /* padding added instead of subtracted */
+                const int ih = oh * stride + pad + r, iw = ow * stride + pad + q;
+#else
+                const int ih = oh * stride - pad + r, iw = ow * stride - pad + q;
+#endif
+                if (ih < 0 || ih >= h || iw < 0 || iw >= wd) continue;   /* zero padding */
+                const int col = (c * kh + r) * kw + q;
+                const double wm = masked_weight(W, is_f16, mask, g, K, cout, co, col);
+                const size_t xi = (((size_t)in * cin + c) * (size_t)h + (size_t)ih) * (size_t)wd + (size_t)iw;
+                const double x = is_f16 ? ld_f16(X, xi) : ld_f32(X, xi);
+                s += wm * x;
+                m += fabs(wm) * fabs(x);
+            }
+    *mag = m;
+    return s;
+}
+
+int oracle_conv2d_out_size(int in, int k, int stride, int pad)
+{
+    if (stride < 1 || k < 1 || pad < 0 || in + 2 * pad < k) return -1;
+    return (in + 2 * pad - k) / stride + 1;
+}
+
+int oracle_conv2d(const void *W, const uint8_t *mask, int g, const void *X, const float *bias,
+                  int relu, int is_f16, int n, int cin, int cout, int h, int wd, int kh, int kw,
+                  int stride, int pad, double *Y, double *A)
+{
+    if (!W || !mask || !X || g < 1 || n < 0 || cin < 0 || cout < 0) return -1;
+    const int oh = oracle_conv2d_out_size(h, kh, stride, pad);
+    const int ow = oracle_conv2d_out_size(wd, kw, stride, pad);
+    if (oh < 0 || ow < 0) return -1;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int in = 0; in < n; ++in)
+        for (int co = 0; co < cout; ++co) {
+            const double b = bias ? (double)bias[co] : 0.0;
+            for (int y = 0; y < oh; ++y)
+                for (int x = 0; x < ow; ++x) {
+                    double m;
+                    double s = conv2d_point(W, mask, g, X, is_f16, cin, cout, h, wd, kh, kw, stride,
+                                            pad, in, co, y, x, &m) + b;
+                    if (relu && s < 0.0) s = 0.0;
+                    const size_t yi = (((size_t)in * cout + co) * (size_t)oh + (size_t)y) * (size_t)ow + (size_t)x;
+                    if (Y) Y[yi] = s;
+                    if (A) A[yi] = m + fabs(b);
+                }
+        }
+    return 0;
+}
+
+/* Selected outputs of the general convolution: idx[k] is a flat index into Y[n][cout][oh][ow]. */
+int oracle_conv2d_points(const void *W, const uint8_t *mask, int g, const void *X, const float *bias,
+                         int relu, int is_f16, int n, int cin, int cout, int h, int wd, int kh,
+                         int kw, int stride, int pad, const int64_t *idx, long n_idx, double *out,
+                         double *mag)
+{
+    if (!W || !mask || !X || !idx || !out || g < 1) return -1;
+    const int oh = oracle_conv2d_out_size(h, kh, stride, pad);
+    const int ow = oracle_conv2d_out_size(wd, kw, stride, pad);
+    if (oh < 0 || ow < 0) return -1;
+    int bad = 0;
+#pragma omp parallel for schedule(static)
+    for (long k = 0; k < n_idx; ++k) {
+        const int64_t f = idx[k];
+        if (f < 0 || f >= (int64_t)n * cout * oh * ow) { bad = 1; continue; }
+        const int x = (int)(f % ow);
+        const int y = (int)((f / ow) % oh);
+        const int co = (int)((f / ow / oh) % cout);
+        const int in = (int)(f / ow / oh / cout);
+        double m;
+        const double b = bias ? (double)bias[co] : 0.0;
+        double s = conv2d_point(W, mask, g, X, is_f16, cin, cout, h, wd, kh, kw, stride, pad, in,
+                                co, y, x, &m) + b;
         if (relu && s < 0.0) s = 0.0;
         out[k] = s;
         if (mag) mag[k] = m + fabs(b);

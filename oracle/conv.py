@@ -1,7 +1,8 @@
 """ctypes front end of the C oracle (oracle/alcs_oracle.c).  Test infrastructure only.
 
-The convolution definition it evaluates is the paper's Section 3.2.2 formula at
-k_h = k_w = 1 over mask-applied weights, in double precision, plus bias and ReLU.
+The convolution definition it evaluates is the paper's Section 3.2.2 formula over
+mask-applied weights, in double precision, plus bias and ReLU: conv1x1 at k_h = k_w = 1,
+conv2d for a general kernel with stride and zero padding.
 """
 from __future__ import annotations
 
@@ -24,6 +25,15 @@ def _lib(mutant: int = 0, build_dir: str | None = None):
     lib.oracle_conv1x1_points.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p,
                                           C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_long,
                                           C.c_void_p, C.c_long, C.c_void_p, C.c_void_p]
+    lib.oracle_conv2d.restype = C.c_int
+    lib.oracle_conv2d.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p,
+                                  C.c_int, C.c_int] + [C.c_int] * 9 + [C.c_void_p, C.c_void_p]
+    lib.oracle_conv2d_points.restype = C.c_int
+    lib.oracle_conv2d_points.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p,
+                                         C.c_int, C.c_int] + [C.c_int] * 9 + [
+                                             C.c_void_p, C.c_long, C.c_void_p, C.c_void_p]
+    lib.oracle_conv2d_out_size.restype = C.c_int
+    lib.oracle_conv2d_out_size.argtypes = [C.c_int] * 4
     lib.oracle_num_threads.restype = C.c_int
     lib.oracle_mutant.restype = C.c_int
     assert lib.oracle_mutant() == mutant
@@ -84,4 +94,60 @@ def conv1x1_points(W, mask, X, flat_idx, bias=None, relu=False, g=4):
         int(W.dtype == np.float16), n, cin, cout, hw, _ptr(idx), idx.size, _ptr(out), _ptr(mag))
     if rc != 0:
         raise RuntimeError(f"oracle_conv1x1_points failed: {rc}")
+    return out, mag
+
+
+def _prep2d(W, mask, X, bias, g, stride, pad):
+    if W.dtype not in (np.float32, np.float16) or X.dtype != W.dtype:
+        raise TypeError("W and X must both be float32 or both float16")
+    W = np.ascontiguousarray(W)
+    X = np.ascontiguousarray(X)
+    mask = np.ascontiguousarray(mask, dtype=np.uint8)
+    cout, cin, kh, kw = W.shape
+    n, cin2, h, wd = X.shape
+    rows = (cout + g - 1) // g
+    if cin2 != cin or mask.shape != (rows, cin * kh * kw):
+        raise ValueError("shape mismatch")
+    if bias is not None:
+        bias = np.ascontiguousarray(bias, dtype=np.float32)
+        if bias.shape != (cout,):
+            raise ValueError("bias shape")
+    oh = (h + 2 * pad - kh) // stride + 1
+    ow = (wd + 2 * pad - kw) // stride + 1
+    if stride < 1 or pad < 0 or h + 2 * pad < kh or wd + 2 * pad < kw:
+        raise ValueError("geometry")
+    return W, mask, X, bias, (n, cin, cout, h, wd, kh, kw, stride, pad), (oh, ow)
+
+
+def conv2d(W, mask, X, bias=None, relu=False, g=4, stride=1, pad=0, want_scale=False, mutant=0,
+           build_dir=None):
+    """Y[n,cout,oh,ow] (float64) of the general kernel: W [cout,cin,kh,kw], block mask
+    [ceil(cout/g), cin*kh*kw] over the flattened-filter columns (c*kh + r)*kw + s,
+    X [n,cin,h,w], zero padding `pad`, stride `stride`.
+
+    With want_scale also returns A = |bias| + sum |Wm||X| (float64, same shape).
+    """
+    W, mask, X, bias, geo, (oh, ow) = _prep2d(W, mask, X, bias, g, stride, pad)
+    n, cout = geo[0], geo[2]
+    Y = np.empty((n, cout, oh, ow), dtype=np.float64)
+    A = np.empty((n, cout, oh, ow), dtype=np.float64) if want_scale else None
+    rc = _lib(mutant, build_dir).oracle_conv2d(
+        _ptr(W), _ptr(mask), g, _ptr(X), _ptr(bias), int(bool(relu)),
+        int(W.dtype == np.float16), *geo, _ptr(Y), _ptr(A))
+    if rc != 0:
+        raise RuntimeError(f"oracle_conv2d failed: {rc}")
+    return (Y, A) if want_scale else Y
+
+
+def conv2d_points(W, mask, X, flat_idx, bias=None, relu=False, g=4, stride=1, pad=0):
+    """The same quantities at selected flat indices of Y[n,cout,oh,ow]; returns (values, scale)."""
+    W, mask, X, bias, geo, _ = _prep2d(W, mask, X, bias, g, stride, pad)
+    idx = np.ascontiguousarray(flat_idx, dtype=np.int64)
+    out = np.empty(idx.shape, dtype=np.float64)
+    mag = np.empty(idx.shape, dtype=np.float64)
+    rc = _lib().oracle_conv2d_points(
+        _ptr(W), _ptr(mask), g, _ptr(X), _ptr(bias), int(bool(relu)),
+        int(W.dtype == np.float16), *geo, _ptr(idx), idx.size, _ptr(out), _ptr(mag))
+    if rc != 0:
+        raise RuntimeError(f"oracle_conv2d_points failed: {rc}")
     return out, mag

@@ -1,5 +1,6 @@
 /*
- * alcs.h -- C ABI of the SIMD-structured sparse pointwise (1x1) convolution for NVIDIA B200.
+ * alcs.h -- C ABI of the SIMD-structured sparse convolution for NVIDIA B200: pointwise (1x1)
+ * layers first, the general k x k case (alcs_spconv2d) further down.
  *
  *   Y[n, cout, h*w] = W_sparse[cout, cin] x X[n, cin, h*w] + bias   (optionally ReLU)
  *
@@ -267,6 +268,47 @@ ALCS_API int alcs_spconv1x1_host(const alcs_packed* w, const void* x_host, void*
 #define ALCS_NOALLOC_SCRATCH_BYTES (16u << 20)
 ALCS_API int alcs_spconv1x1_noalloc(const alcs_packed* w, const void* x, void* y, int n, int h, int wd,
                                     const float* bias, unsigned flags, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * General k_h x k_w convolution (device), fp32.
+ *
+ * Operation: paper, Section 3.2.2, the convolution formula with all three sums,
+ *     O(co, oh, ow) = sum_c sum_r sum_s W(co, c, r, s) * I(c, oh*stride - pad + r, ow*stride - pad + s),
+ * I read as zero outside the image (the paper writes the stride-1, unpadded case), evaluated as
+ * W* x I* without materialising I*: W* stacks the flattened filters, so the packed matrix has
+ * cin*kh*kw columns and column (c*kh + r)*kw + s holds tap (r, s) of input channel c.  The pruning
+ * pattern is that of Section 3.2.1 for a general kernel: the parameters at one location (c, r, s)
+ * of g adjacent filters are kept or removed together.  Pack the weights with
+ *     alcs_pack(w [cout][cin*kh*kw], block_mask [ceil(cout/g)][cin*kh*kw], cout, cin*kh*kw, g, ALCS_F32, ...).
+ *
+ * alcs_spconv2d: x device [n][cin][h][wd], y device [n][cout][oh][ow] with
+ * oh = (h + 2*pad - kh)/stride + 1 (ow likewise), contiguous NCHW fp32, 4-byte aligned, not
+ * overlapping; bias device fp32 [cout] or NULL; flags = ALCS_RELU or 0.  Enqueues one kernel on
+ * cuda_stream.  The first call for a new geometry builds that geometry's launch schedule, allocates
+ * device memory owned by w for it and waits for its upload; later calls with the same geometry do
+ * neither.  n == 0 is a successful no-op.
+ * Errors: INVALID_ARG (null or misaligned or overlapping buffers, non-positive sizes, unknown
+ * flags), SHAPE (cin*kh*kw is not the packed column count, kernel larger than the padded image,
+ * more than 2^31-1 elements), UNSUPPORTED (fp16 weights, g outside {1,2,4,8,16}, stride > 2,
+ * kernels wider than 8*stride+1, or so many input channels that not even a one-row strip of all of
+ * them fits in shared memory), STATE, ALLOC, CUDA.
+ *
+ * alcs_spconv2d_plan reports the launch configuration alcs_spconv2d would use (host only).
+ * ------------------------------------------------------------------------------------------- */
+typedef struct {
+    int positions_per_lane;     /* output positions per lane (2, 4 or 8)                           */
+    int strip_rows;             /* output rows per work item                                        */
+    int row_groups;             /* work items that share one strip, each taking a subset of rows    */
+    int position_tiles;         /* tiles of 32*positions_per_lane positions per strip               */
+    int warps_per_tile;         /* warps that share one position tile and split its block rows      */
+    int smem_bytes;             /* dynamic shared memory per thread block                           */
+} alcs_conv2d_cfg;
+
+ALCS_API int alcs_spconv2d(const alcs_packed* w, const void* x, void* y, int n, int cin, int h, int wd,
+                           int kh, int kw, int stride, int pad, const float* bias, unsigned flags,
+                           void* cuda_stream);
+ALCS_API int alcs_spconv2d_plan(const alcs_packed* w, int n, int cin, int h, int wd, int kh, int kw,
+                                int stride, int pad, alcs_conv2d_cfg* out);
 
 /* ---------------------------------------------------------------------------------------------
  * Layer stack: a network's pointwise layers run back to back on one stream (paper, Section 3.3,

@@ -27,7 +27,7 @@ EXPORTS = ["alcs_strerror", "alcs_last_cuda_error", "alcs_version", "alcs_pack",
            "alcs_packed_upload", "alcs_packed_status", "alcs_packed_free", "alcs_variant_count", "alcs_variant_get",
            "alcs_spconv1x1", "alcs_spconv1x1_cfg",
            "alcs_spconv1x1_plan", "alcs_spconv1x1_tune", "alcs_spconv1x1_set_cfg", "alcs_spconv1x1_host_workspace",
-           "alcs_spconv1x1_host", "alcs_spconv1x1_noalloc", "alcs_stack_create", "alcs_stack_run", "alcs_stack_destroy"]
+           "alcs_spconv1x1_host", "alcs_spconv1x1_noalloc", "alcs_spconv2d", "alcs_spconv2d_plan", "alcs_stack_create", "alcs_stack_run", "alcs_stack_destroy"]
 
 
 class AlcsError(RuntimeError):
@@ -43,6 +43,14 @@ class LaunchCfg(C.Structure):
     _fields_ = [(k, C.c_int) for k in ("pixels_per_lane", "rows_per_warp", "warps",
                                        "chunk_channels", "stages", "row_groups", "min_blocks", "copy_mode",
                                        "producer_warps", "math_mode", "consumer_groups")]
+
+    def as_dict(self):
+        return {k: getattr(self, k) for k, _ in self._fields_}
+
+
+class Conv2dCfg(C.Structure):
+    _fields_ = [(k, C.c_int) for k in ("positions_per_lane", "strip_rows", "row_groups", "position_tiles",
+                                       "warps_per_tile", "smem_bytes")]
 
     def as_dict(self):
         return {k: getattr(self, k) for k, _ in self._fields_}
@@ -89,6 +97,8 @@ def lib():
     L.alcs_spconv1x1_host_workspace.restype = sz
     L.alcs_spconv1x1_host.argtypes = [vp, vp, vp, i, i, i, vp, u, vp, sz, vp]
     L.alcs_spconv1x1_noalloc.argtypes = [vp, vp, vp, i, i, i, vp, u, vp]
+    L.alcs_spconv2d.argtypes = [vp, vp, vp] + [i] * 8 + [vp, u, vp]
+    L.alcs_spconv2d_plan.argtypes = [vp] + [i] * 8 + [C.POINTER(Conv2dCfg)]
     L.alcs_stack_create.argtypes = [C.POINTER(Layer), i, u, C.POINTER(vp)]
     L.alcs_stack_run.argtypes = [vp, vp]
     L.alcs_stack_destroy.argtypes = [vp]
@@ -295,6 +305,22 @@ def alcs_spconv1x1_noalloc(w: Packed, x, y, n: int, h: int, wd: int, bias=None, 
     h*wd rows are not 16-byte multiples) has to fit ALCS_NOALLOC_SCRATCH_BYTES."""
     _check(lib().alcs_spconv1x1_noalloc(w.handle, _addr(x), _addr(y), n, h, wd, _addr(bias), flags, _stream(stream)),
            "alcs_spconv1x1_noalloc")
+
+
+def alcs_spconv2d(w: Packed, x, y, n: int, cin: int, h: int, wd: int, kh: int, kw: int, stride: int = 1,
+                  pad: int = 0, bias=None, flags: int = 0, stream=None):
+    """General k x k convolution: x [n,cin,h,wd], y [n,cout,oh,ow] fp32 device tensors; w packed from
+    the flattened filters [cout, cin*kh*kw]."""
+    _check(lib().alcs_spconv2d(w.handle, _addr(x), _addr(y), n, cin, h, wd, kh, kw, stride, pad, _addr(bias),
+                               flags, _stream(stream)), "alcs_spconv2d")
+
+
+def alcs_spconv2d_plan(w: Packed, n: int, cin: int, h: int, wd: int, kh: int, kw: int, stride: int = 1,
+                       pad: int = 0) -> dict:
+    out = Conv2dCfg()
+    _check(lib().alcs_spconv2d_plan(w.handle, n, cin, h, wd, kh, kw, stride, pad, C.byref(out)),
+           "alcs_spconv2d_plan")
+    return out.as_dict()
 
 
 class Stack:

@@ -1,0 +1,255 @@
+// Device code of the general k_h x k_w SIMD-structured sparse convolution for sm_100a.
+//
+// The paper's Section 3.2.2 views the convolution as W* x I*: W* stacks the flattened filters
+// (column = (c, r, s)), I* stacks the vectorised input patches, and the grouped-CSR format stores,
+// per group of g filters, the kept columns of W*.  The multiply loop is the same as for 1x1
+// kernels (zero the accumulators, walk the group's kept columns, multiply the column's g weights
+// with the input vector the column offset addresses); what changes is what a column addresses:
+// the input image of channel c shifted by the tap (r, s).  I* is never materialised.
+//
+//   work item    = (image, strip of TH output rows, row group)
+//   thread block = persistent; per item it first stages the input patch of ALL input channels
+//                  that the strip needs (halo and zero padding included) in shared memory, then
+//                  its warps multiply
+//   patch layout = per channel, stride x stride "parity planes": input pixel (ih, iw) of the
+//                  patch window lies in plane (ih % stride, iw % stride) at [ih / stride][iw / stride],
+//                  planes have PR rows of pitch WP words.  With that layout the address of the
+//                  input that output position (oh, ow) needs for column (c, r, s) is
+//                      coloff(c, r, s) + (oh * WP + ow),      coloff = c*CHW + plane(r,s)*PL + (r/stride)*WP + s/stride
+//                  for every stride: a per-column constant plus a per-position constant.  The
+//                  per-column constants are baked into the launch schedule as byte offsets.
+//   position     = j = oh_local * WP + ow, 0 <= j < TH*WP.  Positions with ow >= OW (the
+//                  (kw-1)/stride extra columns of the pitch) are computed and not stored.
+//   warp         = one tile of 32*P consecutive positions (lane owns j0 + lane + 32*t, so every
+//                  shared-memory load is 32 consecutive words) x one block row at a time; the
+//                  warps that share a position tile take the row group's rows from a shared
+//                  counter, longest rows first.  G*P fp32 accumulators per lane.
+//   weights      = pair records (two byte offsets of the NEXT pair, the 2*G values of this pair)
+//                  read straight from global memory with warp-uniform loads; each row is one
+//                  contiguous run, so the L1 prefetch a few hundred bytes ahead covers it.
+//
+// There are no cross-warp waits other than __syncthreads, so nothing here can spin.
+#ifndef ALCS_CONV2D_CUH_
+#define ALCS_CONV2D_CUH_
+
+#include "alcs_kernels.cuh"
+
+namespace alcs {
+
+struct Conv2dArgs {
+    const float* x;            // [n][cin][h][wd]
+    float* y;                  // [n][cout][oh][ow]
+    const float* bias;         // [cout] or nullptr
+    const unsigned char* rec;  // pair records, [row group][local row]
+    const int* slice;          // [n_rg + 1] start of each row group's records, 16-byte units
+    const int* rowoff;         // [n_rg][rpg] int4 {row start inside the slice (16-byte units), first two byte offsets, pairs}
+    const int* rowmap;         // [n_rg][rpg] block row of each local row, -1 = none
+    int rows, cin, cout;
+    int h, wd, oh, ow;
+    int kh, kw, pad;
+    int th;                    // output rows per strip
+    int n_strips, n_rg, rpg, n_img;
+    int wp, pr, pl, chw;       // plane pitch, plane rows, words per plane, words per channel
+    int npt, nrs;              // position tiles per strip, warps per position tile
+    int slack;                 // words after the patch that out-of-strip positions may read
+    int relu;
+};
+
+template <int P>
+__device__ __forceinline__ void load_x2d(const float* xs, int byte_off, float2 (&x)[P / 2])
+{
+    const float* p = reinterpret_cast<const float*>(reinterpret_cast<const unsigned char*>(xs) + byte_off);
+#pragma unroll
+    for (int t = 0; t < P / 2; ++t) x[t] = make_float2(p[64 * t], p[64 * t + 32]);
+}
+
+__device__ __forceinline__ void prefetch_l1(const void* p)
+{
+    asm volatile("prefetch.global.L1 [%0];\n" ::"l"(p));
+}
+
+// Multiply-accumulate one whole block row: `npairs` pair records starting at rp (global memory),
+// (oa0, oa1) = byte offsets of the first pair's columns.  Same two-register-set rotation as the
+// pointwise kernel: the record and the input vectors of pair i+1 are loaded while pair i is
+// multiplied.
+template <int G, int P>
+__device__ __forceinline__ void consume_row2d(float2 (&acc)[G][P / 2], const float* xs, const unsigned char* rp,
+                                              int npairs, int oa0, int oa1)
+{
+    constexpr int REC = record_bytes(G);
+    constexpr int AHEAD = 768;                      // bytes of records requested ahead of use
+    const unsigned char* re = rp + npairs * REC;
+    if constexpr (G <= 4) {
+        int ob0 = 0, ob1 = 0;
+        float wA0[G], wA1[G], wB0[G], wB1[G];
+        float2 xA0[P / 2], xA1[P / 2], xB0[P / 2], xB1[P / 2];
+        load_record<G>(rp, ob0, ob1, wA0, wA1);
+        load_x2d<P>(xs, oa0, xA0);
+        load_x2d<P>(xs, oa1, xA1);
+        while (true) {
+            if (rp + AHEAD < re) prefetch_l1(rp + AHEAD);
+            const bool moreB = rp + REC < re;
+            if (moreB) {
+                load_record<G>(rp + REC, oa0, oa1, wB0, wB1);
+                load_x2d<P>(xs, ob0, xB0);
+                load_x2d<P>(xs, ob1, xB1);
+            }
+            fma_block<G, P>(acc, wA0, xA0);
+            fma_block<G, P>(acc, wA1, xA1);
+            if (!moreB) break;
+            const bool moreA = rp + 2 * REC < re;
+            if (moreA) {
+                load_record<G>(rp + 2 * REC, ob0, ob1, wA0, wA1);
+                load_x2d<P>(xs, oa0, xA0);
+                load_x2d<P>(xs, oa1, xA1);
+            }
+            fma_block<G, P>(acc, wB0, xB0);
+            fma_block<G, P>(acc, wB1, xB1);
+            if (!moreA) break;
+            rp += 2 * REC;
+        }
+    } else {
+        // wide groups: the accumulators fill most of the register file; only the next pair's
+        // offsets are fetched ahead
+        while (true) {
+            if (rp + AHEAD < re) prefetch_l1(rp + AHEAD);
+            float2 x0[P / 2], x1[P / 2];
+            float w[G];
+            load_x2d<P>(xs, oa0, x0);
+            load_x2d<P>(xs, oa1, x1);
+            const int2 nx = *reinterpret_cast<const int2*>(rp);
+            load_w<G>(rp + 16, w);
+            fma_block<G, P>(acc, w, x0);
+            load_w<G>(rp + 16 + 4 * G, w);
+            fma_block<G, P>(acc, w, x1);
+            if (rp + REC >= re) break;
+            oa0 = nx.x;
+            oa1 = nx.y;
+            rp += REC;
+        }
+    }
+}
+
+// G = group size, P = positions per lane, ST = stride (1 or 2), NW = warps per thread block.
+template <int G, int P, int ST, int NW>
+__global__ void __launch_bounds__(NW * 32, 1) spconv2d_kernel(const Conv2dArgs a)
+{
+    extern __shared__ __align__(16) float patch[];     // [cin][ST*ST][pr][wp], then a.slack words
+    __shared__ int next_row[NW];                        // per position tile: next local row to take
+
+    const int tid = threadIdx.x;
+    const int lane = tid & 31;
+    const int warp = tid >> 5;
+    const int items = a.n_img * a.n_strips * a.n_rg;
+    const int patch_words = a.cin * a.chw;
+    const int positions = a.th * a.wp;
+
+    // the slack that positions past the last strip row, and the extra columns of the pitch, read
+    for (int i = tid; i < a.slack; i += NW * 32) patch[patch_words + i] = 0.0f;
+
+    const int pt = warp % a.npt;                        // position tile of this warp
+    const bool active = warp < a.npt * a.nrs;
+    const int jbase = pt * (32 * P) + lane;
+
+    for (int item = blockIdx.x; item < items; item += gridDim.x) {
+        const int rg = item % a.n_rg;
+        const int strip = (item / a.n_rg) % a.n_strips;
+        const int img = item / (a.n_rg * a.n_strips);
+        const int oh0 = strip * a.th;
+
+        __syncthreads();                                // everyone is done with the previous patch
+        if (tid < NW) next_row[tid] = 0;
+
+        // ---- stage the patch: one (channel, input row) per warp and pass, lanes along the row ----
+        {
+            const int ph_in = ST * a.pr, pw_in = ST * a.wp;
+            const int ih0 = oh0 * ST - a.pad;
+            const float* ximg = a.x + (size_t)img * a.cin * a.h * a.wd;
+            for (int idx = warp; idx < a.cin * ph_in; idx += NW) {
+                const int c = idx / ph_in;
+                const int rr = idx - c * ph_in;
+                const int ih = ih0 + rr;
+                const bool row_ok = ih >= 0 && ih < a.h;
+                const float* src = ximg + ((size_t)c * a.h + (row_ok ? ih : 0)) * a.wd;
+                float* dst = patch + c * a.chw + ((rr % ST) * ST) * a.pl + (rr / ST) * a.wp;
+                for (int cc = lane; cc < pw_in; cc += 32) {
+                    const int iw = cc - a.pad;
+                    const float v = (row_ok && iw >= 0 && iw < a.wd) ? __ldg(src + iw) : 0.0f;
+                    dst[(cc % ST) * a.pl + cc / ST] = v;
+                }
+            }
+        }
+        __syncthreads();
+
+        if (!active) continue;
+
+        // where this lane's positions go in Y (-1: not an output)
+        int yoff[P];
+#pragma unroll
+        for (int t = 0; t < P; ++t) {
+            const int j = jbase + 32 * t;
+            const int ol = j / a.wp;
+            const int ow = j - ol * a.wp;
+            yoff[t] = (j < positions && ow < a.ow && oh0 + ol < a.oh) ? (oh0 + ol) * a.ow + ow : -1;
+        }
+        // (positions past the end of the strip read on into the next channel or the slack: in
+        // bounds, finite, never stored)
+        const float* xs = patch + jbase;
+        const int* rowoff = a.rowoff + (size_t)rg * a.rpg * 4;
+        const unsigned char* recs = a.rec + (size_t)__ldg(a.slice + rg) * 16;
+        float* yimg = a.y + (size_t)img * a.cout * a.oh * a.ow;
+
+        while (true) {
+            int lr = 0;
+            if (lane == 0) lr = atomicAdd(&next_row[pt], 1);
+            lr = __shfl_sync(0xffffffffu, lr, 0);
+            if (lr >= a.rpg) break;
+            const int row = __ldg(a.rowmap + rg * a.rpg + lr);
+            if (row < 0) continue;
+            const int4 hd = __ldg(reinterpret_cast<const int4*>(rowoff) + lr);
+
+            float2 acc[G][P / 2];
+#pragma unroll
+            for (int j = 0; j < G; ++j)
+#pragma unroll
+                for (int e = 0; e < P / 2; ++e) acc[j][e] = make_float2(0.0f, 0.0f);
+
+            if (hd.w > 0) {
+                const unsigned char* rp = recs + (size_t)hd.x * 16;
+                const int row_bytes = hd.w * record_bytes(G);
+                prefetch_l1(rp);
+                if (row_bytes > 256) prefetch_l1(rp + 256);
+                if (row_bytes > 512) prefetch_l1(rp + 512);
+                consume_row2d<G, P>(acc, xs, rp, hd.w, hd.y, hd.z);
+            }
+
+#pragma unroll
+            for (int j = 0; j < G; ++j) {
+                const int co = row * G + j;
+                if (co >= a.cout) continue;
+                const float bv = a.bias ? __ldg(a.bias + co) : 0.0f;
+                float* yc = yimg + (size_t)co * a.oh * a.ow;
+#pragma unroll
+                for (int t = 0; t < P; ++t) {
+                    const float2 a2 = acc[j][t / 2];
+                    float v = ((t & 1) ? a2.y : a2.x) + bv;
+                    if (a.relu) v = fmaxf(v, 0.0f);
+                    if (yoff[t] >= 0) yc[yoff[t]] = v;
+                }
+            }
+        }
+    }
+}
+
+// Launch the compiled variant for (g, positions per lane, stride); defined in alcs_conv2d.cu.
+// Returns false if there is no such variant.  The first use of a variant raises its dynamic
+// shared-memory limit.
+constexpr int kConv2dWarps = 16;
+// dynamic shared memory a block may ask for: the 227 KB per-block limit minus the kernel's static part
+constexpr int kConv2dMaxDynSmem = 227 * 1024 - 256;
+bool conv2d_variant_exists(int g, int p, int stride);
+cudaError_t launch_conv2d(int g, int p, int stride, const Conv2dArgs& a, unsigned grid, size_t smem, cudaStream_t st);
+
+}  // namespace alcs
+
+#endif  // ALCS_CONV2D_CUH_

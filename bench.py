@@ -269,13 +269,108 @@ def measure_batch1(A, torch, dev, stream, steps, hbm_gbs, fp32_tf):
                      "nz_gflops": round(flops / cold_us / 1e3, 1), "frac": round(t_roof * 1e6 / cold_us, 4)}}
 
 
+def bench_conv2d(args):
+    """`--workload rn18_3x3_b32`: ResNet-18's 3x3 convolutions (stride 1 and 2, pad 1) through
+    alcs_spconv2d, one launch per layer on one stream; per-layer CUDA-event times, roofline as for
+    the pointwise layers (kept-block FLOPs at the fp32 peak against X, packed W and Y moved once)."""
+    import torch
+    import oracle
+    import paper_2109_00170_b200 as A
+    from alcs_workloads import make_bias2d, make_mask2d, make_weights2d, make_x2d, resnet18_3x3_stack
+    from dataclasses import replace
+    specs = resnet18_3x3_stack(32)
+    if args.layers:
+        specs = [specs[int(i)] for i in args.layers.split(",")]
+    hbm_gbs, peak_src, fp32_tf, _ = peaks()
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    A.lib()
+    stream = torch.cuda.current_stream()
+    L = []
+    for s in specs:
+        W, M, b = make_weights2d(s), make_mask2d(s), make_bias2d(s)
+        p = A.alcs_packed_upload(A.alcs_pack(W.reshape(s.cout, s.k), M, s.g), 0)
+        xd = torch.from_numpy(make_x2d(s)).to(dev)
+        yd = torch.empty((s.n, s.cout, s.oh, s.ow), device=dev)
+        nb = int(M.sum())
+        flops = 2.0 * nb * s.g * s.n * s.oh * s.ow
+        byts = nb * (s.g * 4 + 4) + (s.rows + 1) * 4 + 4 * (xd.numel() + yd.numel()) + 4 * s.cout
+        L.append(dict(spec=s, W=W, M=M, b=b, p=p, x=xd, y=yd, bd=torch.from_numpy(b).to(dev), nb=nb, flops=flops,
+                      bytes=byts, t_roof=max(flops / (fp32_tf * 1e12), byts / (hbm_gbs * 1e9)),
+                      bound="alu" if flops / (fp32_tf * 1e12) >= byts / (hbm_gbs * 1e9) else "hbm"))
+
+    def run_layer(l):
+        s = l["spec"]
+        A.alcs_spconv2d(l["p"], l["x"], l["y"], s.n, s.cin, s.h, s.w, s.kh, s.kw, s.stride, s.pad, l["bd"],
+                        A.ALCS_RELU if s.relu else 0, stream)
+
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)      # larger than L2
+    for _ in range(max(args.warmup, 3)):
+        for l in L:
+            run_layer(l)
+    torch.cuda.synchronize()
+    steps = min(args.steps, 50)
+    sampler = ClockSampler(0)
+    sampler.start()
+    t0 = time.time()
+    times = [[] for _ in L]
+    for _ in range(steps):
+        for i, l in enumerate(L):
+            flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            run_layer(l)
+            e1.record(stream)
+            e1.synchronize()
+            times[i].append(e0.elapsed_time(e1) * 1e3)
+    clocks = sampler.stop(t0, time.time())
+    rows, tot_us, tot_flops, tot_roof = [], 0.0, 0.0, 0.0
+    for l, ts in zip(L, times):
+        s, us = l["spec"], statistics.mean(ts)
+        tot_us += us; tot_flops += l["flops"]; tot_roof += l["t_roof"] * 1e6
+        rows.append({"layer": s.name, "sparsity": s.sparsity, "kept_blocks": l["nb"], "nz_mflop": round(l["flops"] / 1e6, 1),
+                     "mbytes": round(l["bytes"] / 1e6, 2), "t_roof_us": round(l["t_roof"] * 1e6, 2), "bound": l["bound"],
+                     "us": round(us, 2), "us_min": round(min(ts), 2), "nz_gflops": round(l["flops"] / us / 1e3, 1),
+                     "frac": round(l["t_roof"] * 1e6 / us, 4),
+                     "cfg": A.alcs_spconv2d_plan(l["p"], s.n, s.cin, s.h, s.w, s.kh, s.kw, s.stride, s.pad)})
+    dom = max(range(len(L)), key=lambda i: statistics.mean(times[i]))
+    dl, dus = L[dom], statistics.mean(times[dom])
+    if dl["bound"] == "alu":
+        roof = {"bound": "alu", "achieved": dl["flops"] / dus / 1e6, "peak": fp32_tf, "unit": "TFLOP/s"}
+    else:
+        roof = {"bound": "hbm", "achieved": dl["bytes"] / dus / 1e3, "peak": hbm_gbs, "unit": "GB/s"}
+    roof.update({"frac": roof["achieved"] / roof["peak"], "traffic": None, "kernel": "spconv2d_kernel",
+                 "layer": dl["spec"].name, "peak_source": f"HBM {peak_src}; fp32 = 148 SMs x 128 lanes x 2 x max SM clock"})
+    out = {"metric": "nonzero-GFLOP/s & % of roofline, SIMD-sparse 3x3 conv layers (ResNet-18), 1 B200, b=32",
+           "value": tot_flops / tot_us / 1e3, "unit": UNIT, "n_gpus": 1, "steps": steps, "warmup": max(args.warmup, 3),
+           "ms_per_step": tot_us / 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+           "data": "synthetic", "config": {"workload": "rn18_3x3_b32", "layers": len(L), "batch": 32, "g": 4,
+                                           "cache": "L2 flushed (256 MB written) before every timed launch"},
+           "roofline": roof, "stack_roofline": {"sum_t_roof_us": round(tot_roof, 1), "sum_layer_us": round(tot_us, 1),
+                                                "frac": round(tot_roof / tot_us, 4)},
+           "gpu_launches": steps * len(L), "clocks": clocks, "layers": rows}
+    if not args.no_cpu_baseline:
+        # the oracle as it stands on one image of every layer
+        t = nz = 0.0
+        for l in L:
+            s1 = replace(l["spec"], n=1)
+            X1 = make_x2d(s1)
+            c0 = time.perf_counter()
+            oracle.conv2d(l["W"], l["M"], X1, l["b"], s1.relu, s1.g, s1.stride, s1.pad)
+            t += time.perf_counter() - c0
+            nz += l["flops"] / l["spec"].n
+        out["cpu_baseline"] = {"value": nz / t / 1e9, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                               "sample": "1 of 32 images of every layer, one pass", "seconds": round(t, 2)}
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="alcs", choices=["alcs", "reference"])
-    ap.add_argument("--workload", default="mbv1_b64", choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default="mbv1_b64", choices=sorted(WORKLOADS) + ["rn18_3x3_b32"])
     ap.add_argument("--no-tune", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=3)
@@ -289,6 +384,10 @@ def main():
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "alcs" else args.warmup
     wl = args.workload
+    if wl == "rn18_3x3_b32":
+        if args.impl == "reference" or int(os.environ.get("WORLD_SIZE", "1")) > 1:
+            raise SystemExit("rn18_3x3_b32 is a single-GPU side workload of --impl alcs")
+        return bench_conv2d(args)
     specs = config_layers(WORKLOADS[wl])
     if args.layers:
         specs = [specs[int(i)] for i in args.layers.split(",")]

@@ -63,6 +63,12 @@ __device__ __forceinline__ void load_x2d(const float* xs, int byte_off, float2 (
     for (int t = 0; t < P / 2; ++t) x[t] = make_float2(p[64 * t], p[64 * t + 32]);
 }
 
+// 4-byte asynchronous copy global -> shared; src_bytes = 0 writes zero without reading src.
+__device__ __forceinline__ void cp_async_4_zfill(uint32_t dst, const void* src, int src_bytes)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+
 __device__ __forceinline__ void prefetch_l1(const void* p)
 {
     asm volatile("prefetch.global.L1 [%0];\n" ::"l"(p));
@@ -142,6 +148,7 @@ __global__ void __launch_bounds__(NW * 32, 1) spconv2d_kernel(const Conv2dArgs a
     const int warp = tid >> 5;
     const int items = a.n_img * a.n_strips * a.n_rg;
     const int patch_words = a.cin * a.chw;
+    const uint32_t patch_u32 = (uint32_t)__cvta_generic_to_shared(patch);
     const int positions = a.th * a.wp;
 
     // the slack that positions past the last strip row, and the extra columns of the pitch, read
@@ -171,13 +178,16 @@ __global__ void __launch_bounds__(NW * 32, 1) spconv2d_kernel(const Conv2dArgs a
                 const int ih = ih0 + rr;
                 const bool row_ok = ih >= 0 && ih < a.h;
                 const float* src = ximg + ((size_t)c * a.h + (row_ok ? ih : 0)) * a.wd;
-                float* dst = patch + c * a.chw + ((rr % ST) * ST) * a.pl + (rr / ST) * a.wp;
+                const uint32_t dst = patch_u32 + 4u * (uint32_t)(c * a.chw + ((rr % ST) * ST) * a.pl + (rr / ST) * a.wp);
+                // asynchronous 4-byte copies (zero-filled outside the image): all of a warp's loads are
+                // in flight at once instead of one round trip to L2 per pass
                 for (int cc = lane; cc < pw_in; cc += 32) {
                     const int iw = cc - a.pad;
-                    const float v = (row_ok && iw >= 0 && iw < a.wd) ? __ldg(src + iw) : 0.0f;
-                    dst[(cc % ST) * a.pl + cc / ST] = v;
+                    const bool ok = row_ok && iw >= 0 && iw < a.wd;
+                    cp_async_4_zfill(dst + 4u * (uint32_t)((cc % ST) * a.pl + cc / ST), ok ? src + iw : ximg, ok ? 4 : 0);
                 }
             }
+            cp_async_wait_all();
         }
         __syncthreads();
 

@@ -311,6 +311,61 @@ ALCS_API int alcs_spconv2d_plan(const alcs_packed* w, int n, int cin, int h, int
                                 int stride, int pad, alcs_conv2d_cfg* out);
 
 /* ---------------------------------------------------------------------------------------------
+ * Latency model and projection with bisection.
+ *
+ * Latency model: paper, Section 3.3.  The run time of layer l is a function of its number of
+ * non-zero parameters, T^(l)(W^(l)) = T^(||W^(l)||_0), approximated by linear interpolation over
+ * measured pairs (k_i, t_i), 0 = k_1 < ... < k_n = N^(l) (the paper measures 11 of them, at
+ * 0, 0.1 N, ..., N):  T^(s) = t_1 + sum_i delta_i alpha_i min(k_{i+1} - k_i, s - k_i) with
+ * delta_i = [s >= k_i] and alpha_i = (t_{i+1} - t_i) / (k_{i+1} - k_i); the network's run time is
+ * T(W) = tau + sum_l T^(l)(W^(l)).  Host only; all pointers are host memory.
+ * Errors: INVALID_ARG (null pointers, fewer than 2 knots, knots not strictly ascending).
+ * ------------------------------------------------------------------------------------------- */
+typedef struct {
+    int n_knots;                /* number of measured points, >= 2                               */
+    const int64_t* k;           /* [n_knots] non-zero parameter counts, strictly ascending        */
+    const double* t;            /* [n_knots] measured run time at each count (any unit)           */
+} alcs_latency_table;
+
+ALCS_API int alcs_layer_latency(const alcs_latency_table* tab, int64_t s, double* out);
+ALCS_API int alcs_network_latency(double tau, const alcs_latency_table* tabs, int n_layers, const int64_t* s,
+                                  double* out);
+
+/*
+ * alcs_project_bisection: paper, Section 3.4, Algorithm 1 ("Projection operation with bisection").
+ * The variable to project is given layer by layer: u_tilde[l] is a DEVICE pointer to a row-major
+ * fp32 matrix [cout[l]][cols[l]] (cols = cin*kh*kw, the flattened filters); the arrays u_tilde,
+ * cout, cols, tabs themselves are host memory.  Steps: (1) the groups are the g adjacent filters at
+ * one location (Section 3.2.1): group (r, c) of a layer = elements (r*g .. r*g+g-1, c); (2) all
+ * groups of all layers are ranked together by L2 norm, largest first -- the ranking key is the
+ * squared norm accumulated in fp32 in ascending filter order with separately rounded multiplies and
+ * adds, equal keys keep (layer, r, c) order; (3)-(14) N is bisected between 0 and the number of
+ * groups until the model latencies of the two ends of the bracket differ by at most eps, where the
+ * latency of "the top-N groups kept" uses ||W^(l)||_0 = g * (kept groups of layer l) in the model
+ * above; a bracket that can no longer shrink (N1 - N0 <= 1) also ends the loop, a case the paper's
+ * listing leaves open; (15) the (N0+N1)/2 best-ranked groups are kept.
+ * Outputs: mask_out, DEVICE, one byte per group, the layers one after the other, each
+ * [ceil(cout/g)][cols] -- the block_mask layout of alcs_pack; u_out (may be NULL), a host array of
+ * DEVICE pointers, u_out[l] (may be NULL) receives u_tilde[l] with the dropped groups set to +0;
+ * kept_per_layer (host, may be NULL) the number of kept groups per layer; *result (host, may be
+ * NULL).  The call allocates temporary device memory (about 18 bytes per group plus the sort's
+ * workspace), frees it before returning, and synchronises cuda_stream.
+ * Errors: INVALID_ARG, SHAPE (2^32 or more groups), UNSUPPORTED (more than 4096 layers), ALLOC, CUDA.
+ */
+typedef struct {
+    int64_t n_keep;             /* groups kept = (n0 + n1) / 2                                     */
+    int64_t n0, n1;             /* final bracket                                                   */
+    int64_t n_groups;           /* groups in total                                                 */
+    int iters;                  /* bisection steps taken                                           */
+    double latency;             /* model latency of the result                                     */
+} alcs_projection_result;
+
+ALCS_API int alcs_project_bisection(const float* const* u_tilde, const int* cout, const int* cols, int n_layers, int g,
+                                    const alcs_latency_table* tabs, double tau, double t_budget, double eps,
+                                    uint8_t* mask_out, float* const* u_out, int64_t* kept_per_layer,
+                                    alcs_projection_result* result, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Layer stack: a network's pointwise layers run back to back on one stream (paper, Section 3.3,
  * T(W) = tau + sum_l T_l(W_l): the network's run time is the sum over its layers).
  * ------------------------------------------------------------------------------------------- */

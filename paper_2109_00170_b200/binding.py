@@ -27,7 +27,8 @@ EXPORTS = ["alcs_strerror", "alcs_last_cuda_error", "alcs_version", "alcs_pack",
            "alcs_packed_upload", "alcs_packed_status", "alcs_packed_free", "alcs_variant_count", "alcs_variant_get",
            "alcs_spconv1x1", "alcs_spconv1x1_cfg",
            "alcs_spconv1x1_plan", "alcs_spconv1x1_tune", "alcs_spconv1x1_set_cfg", "alcs_spconv1x1_host_workspace",
-           "alcs_spconv1x1_host", "alcs_spconv1x1_noalloc", "alcs_spconv2d", "alcs_spconv2d_plan", "alcs_stack_create", "alcs_stack_run", "alcs_stack_destroy"]
+           "alcs_spconv1x1_host", "alcs_spconv1x1_noalloc", "alcs_spconv2d", "alcs_spconv2d_plan", "alcs_layer_latency", "alcs_network_latency",
+           "alcs_project_bisection", "alcs_stack_create", "alcs_stack_run", "alcs_stack_destroy"]
 
 
 class AlcsError(RuntimeError):
@@ -54,6 +55,15 @@ class Conv2dCfg(C.Structure):
 
     def as_dict(self):
         return {k: getattr(self, k) for k, _ in self._fields_}
+
+
+class LatencyTable(C.Structure):
+    _fields_ = [("n_knots", C.c_int), ("k", C.POINTER(C.c_int64)), ("t", C.POINTER(C.c_double))]
+
+
+class ProjectionResult(C.Structure):
+    _fields_ = [("n_keep", C.c_int64), ("n0", C.c_int64), ("n1", C.c_int64), ("n_groups", C.c_int64),
+                ("iters", C.c_int), ("latency", C.c_double)]
 
 
 class Layer(C.Structure):
@@ -99,6 +109,11 @@ def lib():
     L.alcs_spconv1x1_noalloc.argtypes = [vp, vp, vp, i, i, i, vp, u, vp]
     L.alcs_spconv2d.argtypes = [vp, vp, vp] + [i] * 8 + [vp, u, vp]
     L.alcs_spconv2d_plan.argtypes = [vp] + [i] * 8 + [C.POINTER(Conv2dCfg)]
+    L.alcs_layer_latency.argtypes = [C.POINTER(LatencyTable), C.c_int64, C.POINTER(C.c_double)]
+    L.alcs_network_latency.argtypes = [C.c_double, C.POINTER(LatencyTable), i, C.POINTER(C.c_int64), C.POINTER(C.c_double)]
+    L.alcs_project_bisection.argtypes = [C.POINTER(vp), ip, ip, i, i, C.POINTER(LatencyTable), C.c_double, C.c_double,
+                                         C.c_double, vp, C.POINTER(vp), C.POINTER(C.c_int64),
+                                         C.POINTER(ProjectionResult), vp]
     L.alcs_stack_create.argtypes = [C.POINTER(Layer), i, u, C.POINTER(vp)]
     L.alcs_stack_run.argtypes = [vp, vp]
     L.alcs_stack_destroy.argtypes = [vp]
@@ -321,6 +336,59 @@ def alcs_spconv2d_plan(w: Packed, n: int, cin: int, h: int, wd: int, kh: int, kw
     _check(lib().alcs_spconv2d_plan(w.handle, n, cin, h, wd, kh, kw, stride, pad, C.byref(out)),
            "alcs_spconv2d_plan")
     return out.as_dict()
+
+
+def _tables(tables):
+    """[(k, t), ...] -> (ctypes array of LatencyTable, keep-alive list)."""
+    arr = (LatencyTable * len(tables))()
+    keep = []
+    for j, (k, t) in enumerate(tables):
+        ka = np.ascontiguousarray(k, dtype=np.int64)
+        ta = np.ascontiguousarray(t, dtype=np.float64)
+        if ka.shape != ta.shape or ka.ndim != 1:
+            raise ValueError("latency table: k and t must be 1-D of equal length")
+        keep += [ka, ta]
+        arr[j].n_knots = ka.size
+        arr[j].k = ka.ctypes.data_as(C.POINTER(C.c_int64))
+        arr[j].t = ta.ctypes.data_as(C.POINTER(C.c_double))
+    return arr, keep
+
+
+def alcs_layer_latency(k, t, s: int) -> float:
+    arr, keep = _tables([(k, t)])
+    out = C.c_double()
+    _check(lib().alcs_layer_latency(arr, int(s), C.byref(out)), "alcs_layer_latency")
+    return out.value
+
+
+def alcs_network_latency(tau: float, tables, s) -> float:
+    arr, keep = _tables(tables)
+    sa = np.ascontiguousarray(s, dtype=np.int64)
+    out = C.c_double()
+    _check(lib().alcs_network_latency(float(tau), arr, len(tables), sa.ctypes.data_as(C.POINTER(C.c_int64)),
+                                      C.byref(out)), "alcs_network_latency")
+    return out.value
+
+
+def alcs_project_bisection(u_tilde, g: int, tables, tau: float, t_budget: float, eps: float, mask_out,
+                           u_out=None, stream=None) -> dict:
+    """u_tilde: list of fp32 device tensors [cout_l, cols_l]; mask_out: uint8 device tensor with one
+    byte per group, layer after layer; u_out: optional list of output tensors (entries may be None)."""
+    n = len(u_tilde)
+    ptrs = (C.c_void_p * n)(*[_addr(t) for t in u_tilde])
+    cout = (C.c_int * n)(*[int(t.shape[0]) for t in u_tilde])
+    cols = (C.c_int * n)(*[int(t.shape[1]) for t in u_tilde])
+    arr, keep = _tables(tables)
+    outs = None
+    if u_out is not None:
+        outs = (C.c_void_p * n)(*[_addr(t) for t in u_out])
+    kept = (C.c_int64 * n)()
+    res = ProjectionResult()
+    _check(lib().alcs_project_bisection(ptrs, cout, cols, n, g, arr, float(tau), float(t_budget), float(eps),
+                                        _addr(mask_out), outs, kept, C.byref(res), _stream(stream)),
+           "alcs_project_bisection")
+    return {"n_keep": res.n_keep, "n0": res.n0, "n1": res.n1, "n_groups": res.n_groups, "iters": res.iters,
+            "latency": res.latency, "kept_per_layer": list(kept)}
 
 
 class Stack:

@@ -269,6 +269,106 @@ def measure_batch1(A, torch, dev, stream, steps, hbm_gbs, fp32_tf):
                      "nz_gflops": round(flops / cold_us / 1e3, 1), "frac": round(t_roof * 1e6 / cold_us, 4)}}
 
 
+def bench_latency_model(args):
+    """`--workload latency_model`: the paper's Section 3.3 experiment on this GPU.  (1) For every layer
+    of the batch-64 MobileNetV1 pointwise stack, time the sparse kernel at 11 densities (0, 0.1, ..., 1
+    of the blocks kept): the (k_i, t_i) pairs of the interpolation.  (2) Draw random per-layer
+    densities, time the real layers, compare with the interpolated estimate.  (3) Project the stack's
+    weights onto a latency budget with alcs_project_bisection (Algorithm 1), pack the result, time it."""
+    import torch
+    from dataclasses import replace
+    import paper_2109_00170_b200 as A
+    from alcs_workloads import rng, uniform_block_mask
+    specs = config_layers(2)
+    if args.layers:
+        specs = [specs[int(i)] for i in args.layers.split(",")]
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    A.lib()
+    stream = torch.cuda.current_stream()
+    reps = 20
+    W = [make_weights(s) for s in specs]
+    bias = [torch.from_numpy(make_bias(s)).to(dev) for s in specs]
+    X = [torch.from_numpy(make_x(s)).to(dev) for s in specs]
+    Y = [torch.empty((s.n, s.cout, s.hw), device=dev) for s in specs]
+
+    def time_layer(i, mask):
+        s = specs[i]
+        p = A.alcs_packed_upload(A.alcs_pack(W[i], mask, s.g), 0)
+        run = lambda: A.alcs_spconv1x1(p, X[i], Y[i], s.n, s.h, s.w, bias[i], A.ALCS_RELU, stream)
+        for _ in range(3):
+            run()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            run()
+        e1.record(stream)
+        e1.synchronize()
+        A.alcs_packed_free(p)
+        return e0.elapsed_time(e1) * 1e3 / reps          # us
+
+    sampler = ClockSampler(0)
+    sampler.start()
+    t_start = time.time()
+    tables = []
+    for i, s in enumerate(specs):
+        blocks = s.rows * s.cin
+        k, t = [], []
+        for j in range(11):
+            m = uniform_block_mask(s.rows, s.cin, 1.0 - j / 10.0, s.seed + 50 + j)
+            k.append(int(m.sum()) * s.g)
+            t.append(time_layer(i, m))
+        tables.append((k, t))
+    # (2) random density settings, real against estimated
+    trials, errs, rows = 20, [], []
+    for tr in range(trials):
+        u = rng.uniform01_f64(BASE_TRIAL_SEED + tr, 3, len(specs))
+        real, nz = 0.0, []
+        for i, s in enumerate(specs):
+            m = uniform_block_mask(s.rows, s.cin, float(0.05 + 0.9 * u[i]), s.seed + 500 + tr)
+            nz.append(int(m.sum()) * s.g)
+            real += time_layer(i, m)
+        est = A.alcs_network_latency(0.0, tables, nz)
+        errs.append(abs(est - real) / real)
+        rows.append({"real_us": round(real, 1), "estimated_us": round(est, 1)})
+    # (3) projection of the stack's weights onto 50 % of the dense latency
+    dense_t = A.alcs_network_latency(0.0, tables, [k[-1] for k, _ in tables])
+    empty_t = A.alcs_network_latency(0.0, tables, [0] * len(specs))
+    budget = empty_t + 0.5 * (dense_t - empty_t)
+    eps = 0.002 * (dense_t - empty_t)
+    ud = [torch.from_numpy(w).to(dev) for w in W]
+    total = sum(s.rows * s.cin for s in specs)
+    mask_d = torch.empty((total,), dtype=torch.uint8, device=dev)
+    A.alcs_project_bisection(ud, specs[0].g, tables, 0.0, budget, eps, mask_d, None, stream)      # warm-up
+    c0 = time.perf_counter()
+    pr = A.alcs_project_bisection(ud, specs[0].g, tables, 0.0, budget, eps, mask_d, None, stream)
+    proj_ms = (time.perf_counter() - c0) * 1e3
+    mask_h = mask_d.cpu().numpy()
+    real, off = 0.0, 0
+    for i, s in enumerate(specs):
+        m = mask_h[off:off + s.rows * s.cin].reshape(s.rows, s.cin)
+        off += s.rows * s.cin
+        real += time_layer(i, m)
+    clocks = sampler.stop(t_start, time.time())
+    out = {"metric": "latency model: relative error of the interpolated stack latency; projection with bisection",
+           "value": statistics.mean(errs), "unit": "mean |estimated - real| / real", "n_gpus": 1, "steps": trials,
+           "warmup": 3, "higher_is_better": False, "dtype": "f32", "data": "synthetic",
+           "config": {"workload": "latency_model", "stack": "mbv1_b64", "layers": len(specs), "knots": 11,
+                      "runs_per_point": reps, "launch_cfgs": "planner defaults (no per-mask tuning)"},
+           "estimation": {"trials": trials, "mean_rel_err": statistics.mean(errs), "max_rel_err": max(errs), "pairs": rows},
+           "tables_us": [{"layer": s.name, "t": [round(x, 2) for x in t]} for s, (_, t) in zip(specs, tables)],
+           "projection": {"groups": pr["n_groups"], "kept": pr["n_keep"], "iters": pr["iters"], "call_ms": round(proj_ms, 3),
+                          "budget_us": round(budget, 1), "model_latency_us": round(pr["latency"], 1),
+                          "measured_us": round(real, 1), "dense_model_us": round(dense_t, 1),
+                          "kept_fraction_per_layer": [round(kp / (s.rows * s.cin), 3)
+                                                      for kp, s in zip(pr["kept_per_layer"], specs)]},
+           "clocks": clocks}
+    print(json.dumps(out))
+
+
+BASE_TRIAL_SEED = 2109001
+
+
 def bench_conv2d(args):
     """`--workload rn18_3x3_b32`: ResNet-18's 3x3 convolutions (stride 1 and 2, pad 1) through
     alcs_spconv2d, one launch per layer on one stream; per-layer CUDA-event times, roofline as for
@@ -370,7 +470,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="alcs", choices=["alcs", "reference"])
-    ap.add_argument("--workload", default="mbv1_b64", choices=sorted(WORKLOADS) + ["rn18_3x3_b32"])
+    ap.add_argument("--workload", default="mbv1_b64", choices=sorted(WORKLOADS) + ["rn18_3x3_b32", "latency_model"])
     ap.add_argument("--no-tune", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=3)
@@ -384,10 +484,10 @@ def main():
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "alcs" else args.warmup
     wl = args.workload
-    if wl == "rn18_3x3_b32":
+    if wl in ("rn18_3x3_b32", "latency_model"):
         if args.impl == "reference" or int(os.environ.get("WORLD_SIZE", "1")) > 1:
-            raise SystemExit("rn18_3x3_b32 is a single-GPU side workload of --impl alcs")
-        return bench_conv2d(args)
+            raise SystemExit(f"{wl} is a single-GPU side workload of --impl alcs")
+        return bench_conv2d(args) if wl == "rn18_3x3_b32" else bench_latency_model(args)
     specs = config_layers(WORKLOADS[wl])
     if args.layers:
         specs = [specs[int(i)] for i in args.layers.split(",")]

@@ -302,11 +302,19 @@ typedef struct {
     int position_tiles;         /* tiles of 32*positions_per_lane positions per strip               */
     int warps_per_tile;         /* warps that share one position tile and split its block rows      */
     int smem_bytes;             /* dynamic shared memory per thread block                           */
+    int chunk_channels;         /* input channels staged at a time (cin: all at once)               */
 } alcs_conv2d_cfg;
 
 ALCS_API int alcs_spconv2d(const alcs_packed* w, const void* x, void* y, int n, int cin, int h, int wd,
                            int kh, int kw, int stride, int pad, const float* bias, unsigned flags,
                            void* cuda_stream);
+/* Same, with parts of the launch configuration fixed (tests, tuning): non-zero positions_per_lane,
+ * strip_rows, chunk_channels and row_groups of *cfg are taken as given (row_groups only when all
+ * channels are staged at once), the rest is chosen; UNSUPPORTED if nothing fits.  cfg == NULL
+ * behaves like alcs_spconv2d. */
+ALCS_API int alcs_spconv2d_cfg(const alcs_packed* w, const void* x, void* y, int n, int cin, int h, int wd,
+                               int kh, int kw, int stride, int pad, const float* bias, unsigned flags,
+                               const alcs_conv2d_cfg* cfg, void* cuda_stream);
 ALCS_API int alcs_spconv2d_plan(const alcs_packed* w, int n, int cin, int h, int wd, int kh, int kw,
                                 int stride, int pad, alcs_conv2d_cfg* out);
 

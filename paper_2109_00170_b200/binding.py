@@ -27,7 +27,7 @@ EXPORTS = ["alcs_strerror", "alcs_last_cuda_error", "alcs_version", "alcs_pack",
            "alcs_packed_upload", "alcs_packed_status", "alcs_packed_free", "alcs_variant_count", "alcs_variant_get",
            "alcs_spconv1x1", "alcs_spconv1x1_cfg",
            "alcs_spconv1x1_plan", "alcs_spconv1x1_tune", "alcs_spconv1x1_set_cfg", "alcs_spconv1x1_host_workspace",
-           "alcs_spconv1x1_host", "alcs_spconv1x1_noalloc", "alcs_spconv2d", "alcs_spconv2d_plan", "alcs_layer_latency", "alcs_network_latency",
+           "alcs_spconv1x1_host", "alcs_spconv1x1_noalloc", "alcs_spconv2d", "alcs_spconv2d_cfg", "alcs_spconv2d_plan", "alcs_layer_latency", "alcs_network_latency",
            "alcs_project_bisection", "alcs_stack_create", "alcs_stack_run", "alcs_stack_destroy"]
 
 
@@ -51,7 +51,7 @@ class LaunchCfg(C.Structure):
 
 class Conv2dCfg(C.Structure):
     _fields_ = [(k, C.c_int) for k in ("positions_per_lane", "strip_rows", "row_groups", "position_tiles",
-                                       "warps_per_tile", "smem_bytes")]
+                                       "warps_per_tile", "smem_bytes", "chunk_channels")]
 
     def as_dict(self):
         return {k: getattr(self, k) for k, _ in self._fields_}
@@ -108,6 +108,7 @@ def lib():
     L.alcs_spconv1x1_host.argtypes = [vp, vp, vp, i, i, i, vp, u, vp, sz, vp]
     L.alcs_spconv1x1_noalloc.argtypes = [vp, vp, vp, i, i, i, vp, u, vp]
     L.alcs_spconv2d.argtypes = [vp, vp, vp] + [i] * 8 + [vp, u, vp]
+    L.alcs_spconv2d_cfg.argtypes = [vp, vp, vp] + [i] * 8 + [vp, u, C.POINTER(Conv2dCfg), vp]
     L.alcs_spconv2d_plan.argtypes = [vp] + [i] * 8 + [C.POINTER(Conv2dCfg)]
     L.alcs_layer_latency.argtypes = [C.POINTER(LatencyTable), C.c_int64, C.POINTER(C.c_double)]
     L.alcs_network_latency.argtypes = [C.c_double, C.POINTER(LatencyTable), i, C.POINTER(C.c_int64), C.POINTER(C.c_double)]
@@ -323,11 +324,16 @@ def alcs_spconv1x1_noalloc(w: Packed, x, y, n: int, h: int, wd: int, bias=None, 
 
 
 def alcs_spconv2d(w: Packed, x, y, n: int, cin: int, h: int, wd: int, kh: int, kw: int, stride: int = 1,
-                  pad: int = 0, bias=None, flags: int = 0, stream=None):
+                  pad: int = 0, bias=None, flags: int = 0, stream=None, cfg=None):
     """General k x k convolution: x [n,cin,h,wd], y [n,cout,oh,ow] fp32 device tensors; w packed from
-    the flattened filters [cout, cin*kh*kw]."""
-    _check(lib().alcs_spconv2d(w.handle, _addr(x), _addr(y), n, cin, h, wd, kh, kw, stride, pad, _addr(bias),
-                               flags, _stream(stream)), "alcs_spconv2d")
+    the flattened filters [cout, cin*kh*kw].  cfg: optional dict of alcs_conv2d_cfg fields to fix."""
+    if cfg is None:
+        _check(lib().alcs_spconv2d(w.handle, _addr(x), _addr(y), n, cin, h, wd, kh, kw, stride, pad, _addr(bias),
+                                   flags, _stream(stream)), "alcs_spconv2d")
+    else:
+        c = Conv2dCfg(**{k: int(v) for k, v in cfg.items()})
+        _check(lib().alcs_spconv2d_cfg(w.handle, _addr(x), _addr(y), n, cin, h, wd, kh, kw, stride, pad, _addr(bias),
+                                       flags, C.byref(c), _stream(stream)), "alcs_spconv2d_cfg")
 
 
 def alcs_spconv2d_plan(w: Packed, n: int, cin: int, h: int, wd: int, kh: int, kw: int, stride: int = 1,

@@ -9,11 +9,13 @@ namespace {
 
 struct Conv2dVariant {
     int g, p, st;
-    const void* fn;
-    bool ready;
+    const void* fn[2];      // [0] all channels in one chunk, [1] chunked
+    bool ready[2];
 };
 
-#define ALCS_C2D(G, P, ST) {G, P, ST, (const void*)&spconv2d_kernel<G, P, ST, kConv2dWarps>, false}
+#define ALCS_C2D(G, P, ST)                                                              \
+    {G, P, ST, {(const void*)&spconv2d_kernel<G, P, ST, kConv2dWarps, false>,           \
+                (const void*)&spconv2d_kernel<G, P, ST, kConv2dWarps, true>}, {false, false}}
 #define ALCS_C2D_G(G) ALCS_C2D(G, 2, 1), ALCS_C2D(G, 4, 1), ALCS_C2D(G, 8, 1), ALCS_C2D(G, 2, 2), ALCS_C2D(G, 4, 2), ALCS_C2D(G, 8, 2)
 
 // (g = 16 with 8 positions per lane would need 128 accumulator registers: left out)
@@ -36,17 +38,18 @@ cudaError_t launch_conv2d(int g, int p, int stride, const Conv2dArgs& a, unsigne
 {
     Conv2dVariant* v = find(g, p, stride);
     if (!v) return cudaErrorInvalidValue;
+    const int ch = a.nch > 1 ? 1 : 0;
     {
         std::lock_guard<std::mutex> lk(g_c2d_mu);
-        if (!v->ready) {
-            cudaError_t e = cudaFuncSetAttribute(v->fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kConv2dMaxDynSmem);
+        if (!v->ready[ch]) {
+            cudaError_t e = cudaFuncSetAttribute(v->fn[ch], cudaFuncAttributeMaxDynamicSharedMemorySize, kConv2dMaxDynSmem);
             if (e != cudaSuccess) return e;
-            v->ready = true;
+            v->ready[ch] = true;
         }
     }
     Conv2dArgs args = a;
     void* params[] = {&args};
-    return cudaLaunchKernel(v->fn, dim3(grid), dim3(kConv2dWarps * 32), params, smem, st);
+    return cudaLaunchKernel(v->fn[ch], dim3(grid), dim3(kConv2dWarps * 32), params, smem, st);
 }
 
 }  // namespace alcs

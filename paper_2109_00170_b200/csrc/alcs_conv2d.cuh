@@ -8,9 +8,9 @@
 // the input image of channel c shifted by the tap (r, s).  I* is never materialised.
 //
 //   work item    = (image, strip of TH output rows, row group)
-//   thread block = persistent; per item it first stages the input patch of ALL input channels
-//                  that the strip needs (halo and zero padding included) in shared memory, then
-//                  its warps multiply
+//   thread block = persistent; per item it stages the input patch that the strip needs (halo and
+//                  zero padding included) in shared memory -- all input channels at once where
+//                  they fit, else chunk of channels after chunk -- and its warps multiply
 //   patch layout = per channel, stride x stride "parity planes": input pixel (ih, iw) of the
 //                  patch window lies in plane (ih % stride, iw % stride) at [ih / stride][iw / stride],
 //                  planes have PR rows of pitch WP words.  With that layout the address of the
@@ -24,9 +24,9 @@
 //                  shared-memory load is 32 consecutive words) x one block row at a time; the
 //                  warps that share a position tile take the row group's rows from a shared
 //                  counter, longest rows first.  G*P fp32 accumulators per lane.
-//   weights      = pair records (two byte offsets of the NEXT pair, the 2*G values of this pair)
-//                  read straight from global memory with warp-uniform loads; each row is one
-//                  contiguous run, so the L1 prefetch a few hundred bytes ahead covers it.
+//   weights      = pair records (two byte offsets of the NEXT pair, the 2*G values of this pair);
+//                  each row is one contiguous run in global memory, which its warp streams
+//                  through a private shared-memory double buffer with cp.async.
 //
 // There are no cross-warp waits other than __syncthreads, so nothing here can spin.
 #ifndef ALCS_CONV2D_CUH_
@@ -51,7 +51,9 @@ struct Conv2dArgs {
     int n_strips, n_rg, rpg, n_img;
     int wp, pr, pl, chw;       // plane pitch, plane rows, words per plane, words per channel
     int npt, nrs;              // position tiles per strip, warps per position tile
+    int kc, nch;               // input channels per chunk, number of chunks
     int slack;                 // words after the patch that out-of-strip positions may read
+    int off_wbuf;              // byte offset of the warps' record buffers in shared memory (16-byte aligned)
     int relu;
 };
 
@@ -69,22 +71,21 @@ __device__ __forceinline__ void cp_async_4_zfill(uint32_t dst, const void* src, 
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
 }
 
-__device__ __forceinline__ void prefetch_l1(const void* p)
-{
-    asm volatile("prefetch.global.L1 [%0];\n" ::"l"(p));
-}
+// Records of one warp travel through a private shared-memory double buffer: rec_batch(g) records
+// (600 to 800 bytes) per half, copied with 16-byte cp.async, so the hot loop reads them as
+// shared-memory broadcasts (as the pointwise kernel does) instead of waiting for L2.
+__host__ __device__ constexpr int rec_batch(int g) { return g <= 4 ? 16 : g == 8 ? 8 : 4; }
+__host__ __device__ constexpr int rec_buffer_bytes(int g) { return 2 * rec_batch(g) * record_bytes(g); }
 
-// Multiply-accumulate one whole block row: `npairs` pair records starting at rp (global memory),
-// (oa0, oa1) = byte offsets of the first pair's columns.  Same two-register-set rotation as the
-// pointwise kernel: the record and the input vectors of pair i+1 are loaded while pair i is
-// multiplied.
+// Multiply-accumulate `n` pair records that lie in shared memory at rp; (oa0, oa1) = byte offsets of
+// the first pair's columns on entry and of the pair after the last one on return.  Same
+// two-register-set rotation as the pointwise kernel: the record and the input vectors of pair i+1
+// are loaded while pair i is multiplied.
 template <int G, int P>
-__device__ __forceinline__ void consume_row2d(float2 (&acc)[G][P / 2], const float* xs, const unsigned char* rp,
-                                              int npairs, int oa0, int oa1)
+__device__ __forceinline__ void consume_batch2d(float2 (&acc)[G][P / 2], const float* xs, const unsigned char* rp, int n,
+                                                int& oa0, int& oa1)
 {
     constexpr int REC = record_bytes(G);
-    constexpr int AHEAD = 768;                      // bytes of records requested ahead of use
-    const unsigned char* re = rp + npairs * REC;
     if constexpr (G <= 4) {
         int ob0 = 0, ob1 = 0;
         float wA0[G], wA1[G], wB0[G], wB1[G];
@@ -92,9 +93,9 @@ __device__ __forceinline__ void consume_row2d(float2 (&acc)[G][P / 2], const flo
         load_record<G>(rp, ob0, ob1, wA0, wA1);
         load_x2d<P>(xs, oa0, xA0);
         load_x2d<P>(xs, oa1, xA1);
+        int left = n;                       // pairs not yet multiplied, A is loaded
         while (true) {
-            if (rp + AHEAD < re) prefetch_l1(rp + AHEAD);
-            const bool moreB = rp + REC < re;
+            const bool moreB = left > 1;
             if (moreB) {
                 load_record<G>(rp + REC, oa0, oa1, wB0, wB1);
                 load_x2d<P>(xs, ob0, xB0);
@@ -102,8 +103,8 @@ __device__ __forceinline__ void consume_row2d(float2 (&acc)[G][P / 2], const flo
             }
             fma_block<G, P>(acc, wA0, xA0);
             fma_block<G, P>(acc, wA1, xA1);
-            if (!moreB) break;
-            const bool moreA = rp + 2 * REC < re;
+            if (!moreB) { oa0 = ob0; oa1 = ob1; break; }      // A was the last: its header names the next pair
+            const bool moreA = left > 2;
             if (moreA) {
                 load_record<G>(rp + 2 * REC, ob0, ob1, wA0, wA1);
                 load_x2d<P>(xs, oa0, xA0);
@@ -111,14 +112,14 @@ __device__ __forceinline__ void consume_row2d(float2 (&acc)[G][P / 2], const flo
             }
             fma_block<G, P>(acc, wB0, xB0);
             fma_block<G, P>(acc, wB1, xB1);
-            if (!moreA) break;
+            if (!moreA) break;                                // B was the last: (oa0, oa1) came from its header
             rp += 2 * REC;
+            left -= 2;
         }
     } else {
         // wide groups: the accumulators fill most of the register file; only the next pair's
         // offsets are fetched ahead
-        while (true) {
-            if (rp + AHEAD < re) prefetch_l1(rp + AHEAD);
+        for (int i = 0; i < n; ++i, rp += REC) {
             float2 x0[P / 2], x1[P / 2];
             float w[G];
             load_x2d<P>(xs, oa0, x0);
@@ -128,26 +129,64 @@ __device__ __forceinline__ void consume_row2d(float2 (&acc)[G][P / 2], const flo
             fma_block<G, P>(acc, w, x0);
             load_w<G>(rp + 16 + 4 * G, w);
             fma_block<G, P>(acc, w, x1);
-            if (rp + REC >= re) break;
             oa0 = nx.x;
             oa1 = nx.y;
-            rp += REC;
         }
     }
 }
 
-// G = group size, P = positions per lane, ST = stride (1 or 2), NW = warps per thread block.
-template <int G, int P, int ST, int NW>
+// Multiply-accumulate one whole block row (or its segment inside a channel chunk): `npairs` pair
+// records starting at rp in GLOBAL memory, streamed through this warp's double buffer `wbuf`.
+template <int G, int P>
+__device__ __forceinline__ void consume_row2d(float2 (&acc)[G][P / 2], const float* xs, const unsigned char* rp,
+                                              int npairs, int oa0, int oa1, unsigned char* wbuf, int lane)
+{
+    constexpr int REC = record_bytes(G);
+    constexpr int kRecBatch = rec_batch(G);
+    constexpr int HALF = kRecBatch * REC;
+    const uint32_t wbuf_u32 = (uint32_t)__cvta_generic_to_shared(wbuf);
+    const int nb = (npairs + kRecBatch - 1) / kRecBatch;
+    auto fetch = [&](int b) {
+        const int bytes = min(kRecBatch, npairs - b * kRecBatch) * REC;
+        const unsigned char* src = rp + (size_t)b * HALF;
+        const uint32_t dst = wbuf_u32 + (b & 1) * HALF;
+        for (int o = lane * 16; o < bytes; o += 512) cp_async_16(dst + o, src + o);
+        asm volatile("cp.async.commit_group;\n" ::: "memory");
+    };
+    fetch(0);
+    for (int b = 0; b < nb; ++b) {
+        if (b + 1 < nb) {
+            fetch(b + 1);
+            asm volatile("cp.async.wait_group 1;\n" ::: "memory");
+        } else {
+            asm volatile("cp.async.wait_group 0;\n" ::: "memory");
+        }
+        __syncwarp();
+        consume_batch2d<G, P>(acc, xs, wbuf + (b & 1) * HALF, min(kRecBatch, npairs - b * kRecBatch), oa0, oa1);
+        __syncwarp();           // every lane has read this half before the fetch after next refills it
+    }
+}
+
+// G = group size, P = positions per lane, ST = stride (1 or 2), NW = warps per thread block,
+// CHUNKED = which of the two ways through a work item this instance takes.
+//
+// Two ways through a work item.  With all input channels in one chunk (nch == 1) the warps that
+// share a position tile take block rows from a shared counter, one row at a time.  With the
+// channels split into nch chunks (patches too large for shared memory otherwise) every warp owns
+// ONE block row of the row group for the whole item, keeps its accumulators across the chunks, and
+// the block walks stage -> multiply -> stage -> ... ; the schedule then holds one segment per
+// (row group, chunk, row) with chunk-local offsets.
+template <int G, int P, int ST, int NW, bool CHUNKED>
 __global__ void __launch_bounds__(NW * 32, 1) spconv2d_kernel(const Conv2dArgs a)
 {
-    extern __shared__ __align__(16) float patch[];     // [cin][ST*ST][pr][wp], then a.slack words
+    extern __shared__ __align__(16) float patch[];     // [kc][ST*ST][pr][wp], a.slack words, then the warps' record buffers
     __shared__ int next_row[NW];                        // per position tile: next local row to take
 
     const int tid = threadIdx.x;
     const int lane = tid & 31;
     const int warp = tid >> 5;
     const int items = a.n_img * a.n_strips * a.n_rg;
-    const int patch_words = a.cin * a.chw;
+    const int patch_words = a.kc * a.chw;
     const uint32_t patch_u32 = (uint32_t)__cvta_generic_to_shared(patch);
     const int positions = a.th * a.wp;
 
@@ -155,43 +194,20 @@ __global__ void __launch_bounds__(NW * 32, 1) spconv2d_kernel(const Conv2dArgs a
     for (int i = tid; i < a.slack; i += NW * 32) patch[patch_words + i] = 0.0f;
 
     const int pt = warp % a.npt;                        // position tile of this warp
+    const int rs = warp / a.npt;                        // its slot among the warps of that tile
     const bool active = warp < a.npt * a.nrs;
     const int jbase = pt * (32 * P) + lane;
+    unsigned char* wbuf = reinterpret_cast<unsigned char*>(patch) + a.off_wbuf + warp * rec_buffer_bytes(G);
+    const float* xs = patch + jbase;                    // (positions past the end of the strip read on into
+                                                        //  the next channel or the slack: in bounds, never stored)
 
     for (int item = blockIdx.x; item < items; item += gridDim.x) {
         const int rg = item % a.n_rg;
         const int strip = (item / a.n_rg) % a.n_strips;
         const int img = item / (a.n_rg * a.n_strips);
         const int oh0 = strip * a.th;
-
-        __syncthreads();                                // everyone is done with the previous patch
-        if (tid < NW) next_row[tid] = 0;
-
-        // ---- stage the patch: one (channel, input row) per warp and pass, lanes along the row ----
-        {
-            const int ph_in = ST * a.pr, pw_in = ST * a.wp;
-            const int ih0 = oh0 * ST - a.pad;
-            const float* ximg = a.x + (size_t)img * a.cin * a.h * a.wd;
-            for (int idx = warp; idx < a.cin * ph_in; idx += NW) {
-                const int c = idx / ph_in;
-                const int rr = idx - c * ph_in;
-                const int ih = ih0 + rr;
-                const bool row_ok = ih >= 0 && ih < a.h;
-                const float* src = ximg + ((size_t)c * a.h + (row_ok ? ih : 0)) * a.wd;
-                const uint32_t dst = patch_u32 + 4u * (uint32_t)(c * a.chw + ((rr % ST) * ST) * a.pl + (rr / ST) * a.wp);
-                // asynchronous 4-byte copies (zero-filled outside the image): all of a warp's loads are
-                // in flight at once instead of one round trip to L2 per pass
-                for (int cc = lane; cc < pw_in; cc += 32) {
-                    const int iw = cc - a.pad;
-                    const bool ok = row_ok && iw >= 0 && iw < a.wd;
-                    cp_async_4_zfill(dst + 4u * (uint32_t)((cc % ST) * a.pl + cc / ST), ok ? src + iw : ximg, ok ? 4 : 0);
-                }
-            }
-            cp_async_wait_all();
-        }
-        __syncthreads();
-
-        if (!active) continue;
+        const float* ximg = a.x + (size_t)img * a.cin * a.h * a.wd;
+        float* yimg = a.y + (size_t)img * a.cout * a.oh * a.ow;
 
         // where this lane's positions go in Y (-1: not an output)
         int yoff[P];
@@ -202,37 +218,30 @@ __global__ void __launch_bounds__(NW * 32, 1) spconv2d_kernel(const Conv2dArgs a
             const int ow = j - ol * a.wp;
             yoff[t] = (j < positions && ow < a.ow && oh0 + ol < a.oh) ? (oh0 + ol) * a.ow + ow : -1;
         }
-        // (positions past the end of the strip read on into the next channel or the slack: in
-        // bounds, finite, never stored)
-        const float* xs = patch + jbase;
-        const int* rowoff = a.rowoff + (size_t)rg * a.rpg * 4;
-        const unsigned char* recs = a.rec + (size_t)__ldg(a.slice + rg) * 16;
-        float* yimg = a.y + (size_t)img * a.cout * a.oh * a.ow;
 
-        while (true) {
-            int lr = 0;
-            if (lane == 0) lr = atomicAdd(&next_row[pt], 1);
-            lr = __shfl_sync(0xffffffffu, lr, 0);
-            if (lr >= a.rpg) break;
-            const int row = __ldg(a.rowmap + rg * a.rpg + lr);
-            if (row < 0) continue;
-            const int4 hd = __ldg(reinterpret_cast<const int4*>(rowoff) + lr);
-
-            float2 acc[G][P / 2];
-#pragma unroll
-            for (int j = 0; j < G; ++j)
-#pragma unroll
-                for (int e = 0; e < P / 2; ++e) acc[j][e] = make_float2(0.0f, 0.0f);
-
-            if (hd.w > 0) {
-                const unsigned char* rp = recs + (size_t)hd.x * 16;
-                const int row_bytes = hd.w * record_bytes(G);
-                prefetch_l1(rp);
-                if (row_bytes > 256) prefetch_l1(rp + 256);
-                if (row_bytes > 512) prefetch_l1(rp + 512);
-                consume_row2d<G, P>(acc, xs, rp, hd.w, hd.y, hd.z);
+        // stage channels [c0, c0 + nc) of the strip's input window: one (channel, input row) per warp
+        // and pass, lanes along the row, asynchronous 4-byte copies (zero-filled outside the image)
+        // so that all of a warp's loads are in flight at once
+        auto stage = [&](int c0, int nc) {
+            const int ph_in = ST * a.pr, pw_in = ST * a.wp;
+            const int ih0 = oh0 * ST - a.pad;
+            for (int idx = warp; idx < nc * ph_in; idx += NW) {
+                const int c = idx / ph_in;
+                const int rr = idx - c * ph_in;
+                const int ih = ih0 + rr;
+                const bool row_ok = ih >= 0 && ih < a.h;
+                const float* src = ximg + ((size_t)(c0 + c) * a.h + (row_ok ? ih : 0)) * a.wd;
+                const uint32_t dst = patch_u32 + 4u * (uint32_t)(c * a.chw + ((rr % ST) * ST) * a.pl + (rr / ST) * a.wp);
+                for (int cc = lane; cc < pw_in; cc += 32) {
+                    const int iw = cc - a.pad;
+                    const bool ok = row_ok && iw >= 0 && iw < a.wd;
+                    cp_async_4_zfill(dst + 4u * (uint32_t)((cc % ST) * a.pl + cc / ST), ok ? src + iw : ximg, ok ? 4 : 0);
+                }
             }
+            cp_async_wait_all();
+        };
 
+        auto epilogue = [&](int row, float2 (&acc)[G][P / 2]) {
 #pragma unroll
             for (int j = 0; j < G; ++j) {
                 const int co = row * G + j;
@@ -247,6 +256,55 @@ __global__ void __launch_bounds__(NW * 32, 1) spconv2d_kernel(const Conv2dArgs a
                     if (yoff[t] >= 0) yc[yoff[t]] = v;
                 }
             }
+        };
+
+        if constexpr (!CHUNKED) {
+            __syncthreads();                            // everyone is done with the previous patch
+            if (tid < NW) next_row[tid] = 0;
+            stage(0, a.cin);
+            __syncthreads();
+            if (!active) continue;
+            const int4* rowoff = reinterpret_cast<const int4*>(a.rowoff) + (size_t)rg * a.rpg;
+            const unsigned char* recs = a.rec + (size_t)__ldg(a.slice + rg) * 16;
+            while (true) {
+                int lr = 0;
+                if (lane == 0) lr = atomicAdd(&next_row[pt], 1);
+                lr = __shfl_sync(0xffffffffu, lr, 0);
+                if (lr >= a.rpg) break;
+                const int row = __ldg(a.rowmap + rg * a.rpg + lr);
+                if (row < 0) continue;
+                const int4 hd = __ldg(rowoff + lr);
+                float2 acc[G][P / 2];
+#pragma unroll
+                for (int j = 0; j < G; ++j)
+#pragma unroll
+                    for (int e = 0; e < P / 2; ++e) acc[j][e] = make_float2(0.0f, 0.0f);
+                if (hd.w > 0) {
+                    const unsigned char* rp = recs + (size_t)hd.x * 16;
+                    consume_row2d<G, P>(acc, xs, rp, hd.w, hd.y, hd.z, wbuf, lane);
+                }
+                epilogue(row, acc);
+            }
+        } else {
+            // one block row per warp, accumulators kept across the channel chunks
+            const int row = (active && rs < a.rpg) ? __ldg(a.rowmap + rg * a.rpg + rs) : -1;
+            float2 acc[G][P / 2];
+#pragma unroll
+            for (int j = 0; j < G; ++j)
+#pragma unroll
+                for (int e = 0; e < P / 2; ++e) acc[j][e] = make_float2(0.0f, 0.0f);
+            for (int k = 0; k < a.nch; ++k) {
+                __syncthreads();                        // everyone is done with the previous chunk
+                stage(k * a.kc, min(a.kc, a.cin - k * a.kc));
+                __syncthreads();
+                if (row < 0) continue;
+                const int4 hd = __ldg(reinterpret_cast<const int4*>(a.rowoff) + ((size_t)rg * a.nch + k) * a.rpg + rs);
+                if (hd.w > 0) {
+                    const unsigned char* rp = a.rec + ((size_t)__ldg(a.slice + rg * a.nch + k) + hd.x) * 16;
+                    consume_row2d<G, P>(acc, xs, rp, hd.w, hd.y, hd.z, wbuf, lane);
+                }
+            }
+            if (row >= 0) epilogue(row, acc);
         }
     }
 }

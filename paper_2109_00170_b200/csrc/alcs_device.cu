@@ -1023,6 +1023,7 @@ struct Conv2dPlan {
     int n_strips = 0, n_rg = 0;
     int npt = 0, nrs = 0;
     int wp = 0, pr = 0, pl = 0, chw = 0, slack = 0;
+    int kc = 0, nch = 0;     // input channels per chunk, chunks
     size_t smem = 0;
     double cost = 0;    // model estimate, cycles per SM
 };
@@ -1031,7 +1032,8 @@ struct Conv2dPlan {
 // the patch is staged once (about 16 words per cycle per SM from L2) and every kept block costs
 // G*P*32 FMAs per position tile at the rate the shared-memory-bound hot loop sustains; items are
 // dealt to one persistent thread block per SM.
-int plan_conv2d(const alcs_packed* w, const Conv2dGeom& g, int sms, int smem_max, Conv2dPlan* out)
+int plan_conv2d(const alcs_packed* w, const Conv2dGeom& g, int sms, int smem_max, Conv2dPlan* out,
+                const alcs_conv2d_cfg* force = nullptr)
 {
     const int NW = alcs::kConv2dWarps;
     const int wp = g.ow + (g.kw - 1) / g.st;
@@ -1040,39 +1042,53 @@ int plan_conv2d(const alcs_packed* w, const Conv2dGeom& g, int sms, int smem_max
     best.cost = 1e300;
     for (int p = 8; p >= 2; p /= 2) {
         if (!alcs::conv2d_variant_exists(w->g, p, g.st)) continue;
+        if (force && force->positions_per_lane && force->positions_per_lane != p) continue;
         // sustained fraction of the fp32 peak in the hot loop: per pair of blocks 2P X wavefronts
         // plus 3 of records against 16P/8 cycles of FMA issue
         const double rate = 128.0 * 0.6 * (2.0 * p / (2.0 * p + 3.0)) / (16.0 / 19.0);
         for (int th = 1; th <= g.oh; ++th) {
+            if (force && force->strip_rows && force->strip_rows != th) continue;
             const int positions = th * wp;
             const int npt = (positions + 32 * p - 1) / (32 * p);
             if (npt > NW) break;
             const int pr = th + halo;
             const long long chw = (long long)g.st * g.st * pr * wp;
             const int slack = npt * 32 * p - positions + 8;
-            const long long smem = ((long long)g.cin * chw + slack) * 4;
-            if (smem > smem_max) break;
             const int nrs = NW / npt;
             const int n_strips = (g.oh + th - 1) / th;
             const long long base_items = (long long)g.n * n_strips;
-            const int rg_max = std::max(1, std::min(w->rows / std::max(1, nrs), 32));
-            for (int n_rg = 1; n_rg <= rg_max; ++n_rg) {
-                const long long items = base_items * n_rg;
-                const long long rounds = (items + sms - 1) / sms;
-                const double stage = (double)g.cin * chw / 16.0;
-                const double blocks_item = (double)w->nb / n_rg;
-                const double fma = blocks_item * npt * (double)(w->g * p * 32);
-                // warps that share a position tile split its rows; idle warps (NW not a multiple of
-                // npt) and a short row list (fewer rows than warps) leave lanes unused
-                const int rpg = (w->rows + n_rg - 1) / n_rg;
-                const double use = (double)(npt * std::min(nrs, rpg)) / NW;
-                const double compute = fma / (rate * use);
-                const double cost = rounds * (stage + compute + 3000.0);
-                if (cost < best.cost) {
-                    best.p = p; best.th = th; best.n_strips = n_strips; best.n_rg = n_rg;
-                    best.npt = npt; best.nrs = nrs; best.wp = wp; best.pr = pr; best.pl = pr * wp;
-                    best.chw = (int)chw; best.slack = slack; best.smem = (size_t)smem; best.cost = cost;
+            // channels per chunk: all of them if the patch fits, else halves, quarters, ...
+            for (int nch = 1; nch <= g.cin; nch *= 2) {
+                const int kc = (force && force->chunk_channels) ? std::min(force->chunk_channels, g.cin) : (g.cin + nch - 1) / nch;
+                const int nch_real = (g.cin + kc - 1) / kc;
+                const long long smem = (((long long)kc * chw + slack) * 4 + 15) / 16 * 16 + (long long)NW * alcs::rec_buffer_bytes(w->g);
+                if (smem > smem_max) { if (force && force->chunk_channels) break; continue; }
+                // one chunk: warps take rows from a counter, any number of row groups; several chunks:
+                // one row per warp, so the row groups are fixed by the warps per position tile
+                const int rg_fixed = (w->rows + nrs - 1) / nrs;
+                const int rg_lo = nch_real == 1 ? 1 : rg_fixed;
+                const int rg_hi = nch_real == 1 ? std::max(1, std::min(w->rows, 32)) : rg_fixed;
+                for (int n_rg = rg_lo; n_rg <= rg_hi; ++n_rg) {
+                    if (force && force->row_groups && nch_real == 1 && force->row_groups != n_rg) continue;
+                    const long long items = base_items * n_rg;
+                    const long long rounds = (items + sms - 1) / sms;
+                    const double stage = (double)g.cin * chw / 16.0 + 1500.0 * nch_real;
+                    const double blocks_item = (double)w->nb / n_rg;
+                    const double fma = blocks_item * npt * (double)(w->g * p * 32);
+                    // warps that share a position tile split its rows; idle warps (NW not a multiple of
+                    // npt) and a short row list (fewer rows than warps) leave lanes unused
+                    const int rpg = (w->rows + n_rg - 1) / n_rg;
+                    const double use = (double)(npt * std::min(nrs, rpg)) / NW;
+                    const double compute = fma / (rate * use);
+                    const double cost = rounds * (stage + compute + 3000.0);
+                    if (cost < best.cost) {
+                        best.p = p; best.th = th; best.n_strips = n_strips; best.n_rg = n_rg;
+                        best.npt = npt; best.nrs = nrs; best.wp = wp; best.pr = pr; best.pl = pr * wp;
+                        best.chw = (int)chw; best.slack = slack; best.smem = (size_t)smem; best.cost = cost;
+                        best.kc = kc; best.nch = nch_real;
+                    }
                 }
+                break;      // the largest chunk that fits is the one to use for this (p, th)
             }
         }
     }
@@ -1085,28 +1101,30 @@ int plan_conv2d(const alcs_packed* w, const Conv2dGeom& g, int sms, int smem_max
 // offset of that column's (channel, tap) inside the shared-memory patch.
 Schedule* get_schedule2d(const alcs_packed* w, const Conv2dGeom& g, const Conv2dPlan& p)
 {
-    const std::array<int, 7> key = {p.n_rg, p.chw, p.pl, p.wp, g.st, g.kh, g.kw};
+    const std::array<int, 8> key = {p.n_rg, p.chw, p.pl, p.wp, g.st, g.kh, g.kw, p.kc};
     std::lock_guard<std::mutex> lk(w->mu);
     auto it = w->sched2d.find(key);
     if (it != w->sched2d.end()) return &it->second;
     try {
         Schedule& sc = w->sched2d[key];
-        alcs::build_schedule(*w, w->cin, p.n_rg, true, sc);
         const int taps = g.kh * g.kw;
+        alcs::build_schedule(*w, p.kc * taps, p.n_rg, true, sc);      // chunk = kc channels = kc*taps columns
         auto coloff = [&](int col) {
             const int c = col / taps, tap = col - c * taps;
             const int r = tap / g.kw, s = tap - r * g.kw;
             return 4 * (c * p.chw + ((r % g.st) * g.st + (s % g.st)) * p.pl + (r / g.st) * p.wp + s / g.st);
         };
         const int REC = alcs::record_bytes(w->g);
-        for (int rg = 0; rg < sc.n_rg; ++rg)
+        // (columns inside a chunk are chunk-local, and a chunk starts at a channel boundary, so the
+        //  same formula gives the offset inside the staged chunk)
+        for (int rgk = 0; rgk < sc.n_rg * sc.nch; ++rgk)
             for (int t = 0; t < sc.rpg; ++t) {
-                int* hd = &sc.h_rowoff[((size_t)rg * sc.nch) * sc.ros + 4 * t];
+                int* hd = &sc.h_rowoff[(size_t)rgk * sc.ros + 4 * t];
                 const int npairs = hd[3];
                 if (npairs == 0) continue;
                 hd[1] = coloff(hd[1]);
                 hd[2] = coloff(hd[2]);
-                unsigned char* base = &sc.h_rec[((size_t)sc.h_slice[(size_t)rg * sc.nch] + hd[0]) * 16];
+                unsigned char* base = &sc.h_rec[((size_t)sc.h_slice[rgk] + hd[0]) * 16];
                 for (int q = 0; q < npairs; ++q) {
                     int hdr[2];
                     std::memcpy(hdr, base + (size_t)q * REC, 8);
@@ -1164,12 +1182,13 @@ extern "C" ALCS_API int alcs_spconv2d_plan(const alcs_packed* w, int n, int cin,
     if (rc) return rc;
     out->positions_per_lane = p.p; out->strip_rows = p.th; out->row_groups = p.n_rg;
     out->position_tiles = p.npt; out->warps_per_tile = p.nrs; out->smem_bytes = (int)p.smem;
+    out->chunk_channels = p.kc;
     return ALCS_OK;
 }
 
-extern "C" ALCS_API int alcs_spconv2d(const alcs_packed* w, const void* x, void* y, int n, int cin, int h, int wd,
-                                      int kh, int kw, int stride, int pad, const float* bias, unsigned flags,
-                                      void* cuda_stream)
+extern "C" ALCS_API int alcs_spconv2d_cfg(const alcs_packed* w, const void* x, void* y, int n, int cin, int h, int wd,
+                                          int kh, int kw, int stride, int pad, const float* bias, unsigned flags,
+                                          const alcs_conv2d_cfg* cfg, void* cuda_stream)
 {
     Conv2dGeom g;
     int rc = check_conv2d_args(w, x, y, n, cin, h, wd, kh, kw, stride, pad, flags, &g);
@@ -1182,7 +1201,7 @@ extern "C" ALCS_API int alcs_spconv2d(const alcs_packed* w, const void* x, void*
     rc = device_info(w->device, &di);
     if (rc) return rc;
     Conv2dPlan p;
-    rc = plan_conv2d(w, g, di.sms, std::min(alcs::kConv2dMaxDynSmem, di.smem_optin - 256), &p);
+    rc = plan_conv2d(w, g, di.sms, std::min(alcs::kConv2dMaxDynSmem, di.smem_optin - 256), &p, cfg);
     if (rc) return rc;
     Schedule* sc = get_schedule2d(w, g, p);
     if (!sc) return ALCS_ERR_ALLOC;
@@ -1197,10 +1216,20 @@ extern "C" ALCS_API int alcs_spconv2d(const alcs_packed* w, const void* x, void*
     a.h = h; a.wd = wd; a.oh = g.oh; a.ow = g.ow; a.kh = kh; a.kw = kw; a.pad = pad;
     a.th = p.th; a.n_strips = p.n_strips; a.n_rg = sc->n_rg; a.rpg = sc->rpg; a.n_img = n;
     a.wp = p.wp; a.pr = p.pr; a.pl = p.pl; a.chw = p.chw; a.npt = p.npt; a.nrs = p.nrs; a.slack = p.slack;
+    a.kc = p.kc; a.nch = sc->nch;
+    a.off_wbuf = (int)(((size_t)p.kc * p.chw + p.slack) * 4 + 15) / 16 * 16;
+    if (sc->nch != p.nch || (sc->nch > 1 && sc->rpg > p.nrs)) return ALCS_ERR_STATE;      // (cannot happen: plan and schedule agree)
     a.relu = (flags & ALCS_RELU) ? 1 : 0;
     const long long items = (long long)n * p.n_strips * sc->n_rg;
     if (items > 0x7fffffffll) return ALCS_ERR_SHAPE;
     const unsigned grid = (unsigned)std::min<long long>(items, di.sms);
     ALCS_CUDA(alcs::launch_conv2d(w->g, p.p, stride, a, grid, p.smem, st));
     return ALCS_OK;
+}
+
+extern "C" ALCS_API int alcs_spconv2d(const alcs_packed* w, const void* x, void* y, int n, int cin, int h, int wd,
+                                      int kh, int kw, int stride, int pad, const float* bias, unsigned flags,
+                                      void* cuda_stream)
+{
+    return alcs_spconv2d_cfg(w, x, y, n, cin, h, wd, kh, kw, stride, pad, bias, flags, nullptr, cuda_stream);
 }

@@ -101,8 +101,9 @@ struct alcs_packed {
     // by (kc, n_rg), built on demand; the tensor-core flavour of a schedule is stored under -kc
     mutable std::map<std::pair<int, int>, alcs::Schedule> sched;
     // schedules of the general k x k convolution, by {row groups, words per channel, words per parity
-    // plane, plane pitch, stride, kh, kw}: the column offsets baked into them depend on the geometry
-    mutable std::map<std::array<int, 7>, alcs::Schedule> sched2d;
+    // plane, plane pitch, stride, kh, kw, channels per chunk}: the column offsets baked into them depend
+    // on the geometry
+    mutable std::map<std::array<int, 8>, alcs::Schedule> sched2d;
     std::map<alcs::ShapeKey, alcs_launch_cfg> tuned;   // filled by alcs_spconv1x1_tune
     mutable std::map<alcs::ShapeKey, alcs::Plan> plan_cache;   // resolved plans, by shape
     mutable std::mutex mu;                                      // guards plan_cache and sched

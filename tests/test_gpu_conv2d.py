@@ -13,7 +13,7 @@ from gpu_util import assert_parity
 pytestmark = pytest.mark.gpu
 
 
-def _run(alcs, W, M, X, b, relu, g, stride, pad):
+def _run(alcs, W, M, X, b, relu, g, stride, pad, cfg=None):
     import torch
     dev = torch.device("cuda:0")
     cout, cin, kh, kw = W.shape
@@ -27,7 +27,7 @@ def _run(alcs, W, M, X, b, relu, g, stride, pad):
     for _ in range(2):      # second call: schedule already resident
         yd.fill_(float("nan"))
         alcs.alcs_spconv2d(p, xd, yd, n, cin, h, wd, kh, kw, stride, pad, bd, alcs.ALCS_RELU if relu else 0,
-                           torch.cuda.current_stream())
+                           torch.cuda.current_stream(), cfg)
         torch.cuda.synchronize()
     return yd.cpu().numpy()
 
@@ -70,6 +70,19 @@ def test_conv2d_matches_oracle(alcs, geom, relu):
     W, M, X, b = _case(500 + cin + kh, n, cin, cout, h, w, kh, kw, g)
     Y = _run(alcs, W, M, X, b, relu, g, stride, pad)
     Yref, A = oracle.conv2d(W, M, X, b, relu, g, stride, pad, want_scale=True)
+    assert_parity(Y, Yref, A, "f32")
+
+
+@pytest.mark.parametrize("cfg", [dict(chunk_channels=8), dict(chunk_channels=5, positions_per_lane=4),
+                                 dict(chunk_channels=16, strip_rows=3), dict(chunk_channels=1, positions_per_lane=2),
+                                 dict(strip_rows=2, row_groups=2), dict(positions_per_lane=2, strip_rows=5)])
+@pytest.mark.parametrize("stride", [1, 2])
+def test_conv2d_forced_configurations(alcs, cfg, stride):
+    """Channel chunks (one block row per warp, accumulators kept across chunks, a ragged last chunk),
+    several row groups, short strips: every path of the kernel against the oracle."""
+    W, M, X, b = _case(91, 2, 24, 40, 18, 19, 3, 3, 4)
+    Y = _run(alcs, W, M, X, b, True, 4, stride, 1, cfg)
+    Yref, A = oracle.conv2d(W, M, X, b, True, 4, stride, 1, want_scale=True)
     assert_parity(Y, Yref, A, "f32")
 
 

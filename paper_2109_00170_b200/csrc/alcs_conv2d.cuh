@@ -32,6 +32,8 @@
 #ifndef ALCS_CONV2D_CUH_
 #define ALCS_CONV2D_CUH_
 
+#include <utility>
+
 #include "alcs_kernels.cuh"
 
 namespace alcs {
@@ -57,12 +59,59 @@ struct Conv2dArgs {
     int relu;
 };
 
-template <int P>
-__device__ __forceinline__ void load_x2d(const float* xs, int byte_off, float2 (&x)[P / 2])
+// Shared-memory loads by 32-bit shared-space address (no generic-pointer arithmetic in the hot loop).
+// The P positions a lane owns of the input row a column addresses: xs = shared address of the
+// lane's first position, byte_off = the column's offset; positions are 32 words apart.
+template <int OFF>
+__device__ __forceinline__ float lds_off(uint32_t p)
 {
-    const float* p = reinterpret_cast<const float*>(reinterpret_cast<const unsigned char*>(xs) + byte_off);
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1 + %2];\n" : "=f"(v) : "r"(p), "n"(OFF));
+    return v;
+}
+template <int P, int... T>
+__device__ __forceinline__ void load_x2d_seq(uint32_t p, float2 (&x)[P / 2], std::integer_sequence<int, T...>)
+{
+    ((x[T].x = lds_off<256 * T>(p), x[T].y = lds_off<256 * T + 128>(p)), ...);
+}
+template <int P>
+__device__ __forceinline__ void load_x2d(uint32_t xs, int byte_off, float2 (&x)[P / 2])
+{
+    load_x2d_seq<P>(xs + (uint32_t)byte_off, x, std::make_integer_sequence<int, P / 2>{});
+}
+
+__device__ __forceinline__ float4 lds_v4(uint32_t addr)
+{
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];\n" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+    return v;
+}
+
+// One pair record from shared memory by shared-space address (same layout as load_record).
+template <int G>
+__device__ __forceinline__ void load_record_s(uint32_t p, int& c0, int& c1, float (&w0)[G], float (&w1)[G])
+{
+    const float4 h = lds_v4(p);
+    c0 = __float_as_int(h.x);
+    c1 = __float_as_int(h.y);
+    if constexpr (G == 1) {
+        w0[0] = h.z;
+        w1[0] = h.w;
+    } else if constexpr (G == 2) {
+        const float4 v = lds_v4(p + 16);
+        w0[0] = v.x; w0[1] = v.y; w1[0] = v.z; w1[1] = v.w;
+    } else {
 #pragma unroll
-    for (int t = 0; t < P / 2; ++t) x[t] = make_float2(p[64 * t], p[64 * t + 32]);
+        for (int i = 0; i < G / 4; ++i) {
+            const float4 v = lds_v4(p + 16 + 16 * i);
+            w0[4 * i] = v.x; w0[4 * i + 1] = v.y; w0[4 * i + 2] = v.z; w0[4 * i + 3] = v.w;
+        }
+#pragma unroll
+        for (int i = 0; i < G / 4; ++i) {
+            const float4 v = lds_v4(p + 16 + 4 * G + 16 * i);
+            w1[4 * i] = v.x; w1[4 * i + 1] = v.y; w1[4 * i + 2] = v.z; w1[4 * i + 3] = v.w;
+        }
+    }
 }
 
 // 4-byte asynchronous copy global -> shared; src_bytes = 0 writes zero without reading src.
@@ -82,7 +131,7 @@ __host__ __device__ constexpr int rec_buffer_bytes(int g) { return 2 * rec_batch
 // two-register-set rotation as the pointwise kernel: the record and the input vectors of pair i+1
 // are loaded while pair i is multiplied.
 template <int G, int P>
-__device__ __forceinline__ void consume_batch2d(float2 (&acc)[G][P / 2], const float* xs, const unsigned char* rp, int n,
+__device__ __forceinline__ void consume_batch2d(float2 (&acc)[G][P / 2], uint32_t xs, uint32_t rp, int n,
                                                 int& oa0, int& oa1)
 {
     constexpr int REC = record_bytes(G);
@@ -90,14 +139,14 @@ __device__ __forceinline__ void consume_batch2d(float2 (&acc)[G][P / 2], const f
         int ob0 = 0, ob1 = 0;
         float wA0[G], wA1[G], wB0[G], wB1[G];
         float2 xA0[P / 2], xA1[P / 2], xB0[P / 2], xB1[P / 2];
-        load_record<G>(rp, ob0, ob1, wA0, wA1);
+        load_record_s<G>(rp, ob0, ob1, wA0, wA1);
         load_x2d<P>(xs, oa0, xA0);
         load_x2d<P>(xs, oa1, xA1);
         int left = n;                       // pairs not yet multiplied, A is loaded
         while (true) {
             const bool moreB = left > 1;
             if (moreB) {
-                load_record<G>(rp + REC, oa0, oa1, wB0, wB1);
+                load_record_s<G>(rp + REC, oa0, oa1, wB0, wB1);
                 load_x2d<P>(xs, ob0, xB0);
                 load_x2d<P>(xs, ob1, xB1);
             }
@@ -106,7 +155,7 @@ __device__ __forceinline__ void consume_batch2d(float2 (&acc)[G][P / 2], const f
             if (!moreB) { oa0 = ob0; oa1 = ob1; break; }      // A was the last: its header names the next pair
             const bool moreA = left > 2;
             if (moreA) {
-                load_record<G>(rp + 2 * REC, ob0, ob1, wA0, wA1);
+                load_record_s<G>(rp + 2 * REC, ob0, ob1, wA0, wA1);
                 load_x2d<P>(xs, oa0, xA0);
                 load_x2d<P>(xs, oa1, xA1);
             }
@@ -124,13 +173,21 @@ __device__ __forceinline__ void consume_batch2d(float2 (&acc)[G][P / 2], const f
             float w[G];
             load_x2d<P>(xs, oa0, x0);
             load_x2d<P>(xs, oa1, x1);
-            const int2 nx = *reinterpret_cast<const int2*>(rp);
-            load_w<G>(rp + 16, w);
+            const float4 nx = lds_v4(rp);
+#pragma unroll
+            for (int q = 0; q < G / 4; ++q) {
+                const float4 v = lds_v4(rp + 16 + 16 * q);
+                w[4 * q] = v.x; w[4 * q + 1] = v.y; w[4 * q + 2] = v.z; w[4 * q + 3] = v.w;
+            }
             fma_block<G, P>(acc, w, x0);
-            load_w<G>(rp + 16 + 4 * G, w);
+#pragma unroll
+            for (int q = 0; q < G / 4; ++q) {
+                const float4 v = lds_v4(rp + 16 + 4 * G + 16 * q);
+                w[4 * q] = v.x; w[4 * q + 1] = v.y; w[4 * q + 2] = v.z; w[4 * q + 3] = v.w;
+            }
             fma_block<G, P>(acc, w, x1);
-            oa0 = nx.x;
-            oa1 = nx.y;
+            oa0 = __float_as_int(nx.x);
+            oa1 = __float_as_int(nx.y);
         }
     }
 }
@@ -138,13 +195,12 @@ __device__ __forceinline__ void consume_batch2d(float2 (&acc)[G][P / 2], const f
 // Multiply-accumulate one whole block row (or its segment inside a channel chunk): `npairs` pair
 // records starting at rp in GLOBAL memory, streamed through this warp's double buffer `wbuf`.
 template <int G, int P>
-__device__ __forceinline__ void consume_row2d(float2 (&acc)[G][P / 2], const float* xs, const unsigned char* rp,
-                                              int npairs, int oa0, int oa1, unsigned char* wbuf, int lane)
+__device__ __forceinline__ void consume_row2d(float2 (&acc)[G][P / 2], uint32_t xs, const unsigned char* rp,
+                                              int npairs, int oa0, int oa1, uint32_t wbuf_u32, int lane)
 {
     constexpr int REC = record_bytes(G);
     constexpr int kRecBatch = rec_batch(G);
     constexpr int HALF = kRecBatch * REC;
-    const uint32_t wbuf_u32 = (uint32_t)__cvta_generic_to_shared(wbuf);
     const int nb = (npairs + kRecBatch - 1) / kRecBatch;
     auto fetch = [&](int b) {
         const int bytes = min(kRecBatch, npairs - b * kRecBatch) * REC;
@@ -162,7 +218,7 @@ __device__ __forceinline__ void consume_row2d(float2 (&acc)[G][P / 2], const flo
             asm volatile("cp.async.wait_group 0;\n" ::: "memory");
         }
         __syncwarp();
-        consume_batch2d<G, P>(acc, xs, wbuf + (b & 1) * HALF, min(kRecBatch, npairs - b * kRecBatch), oa0, oa1);
+        consume_batch2d<G, P>(acc, xs, wbuf_u32 + (b & 1) * HALF, min(kRecBatch, npairs - b * kRecBatch), oa0, oa1);
         __syncwarp();           // every lane has read this half before the fetch after next refills it
     }
 }
@@ -197,8 +253,8 @@ __global__ void __launch_bounds__(NW * 32, 1) spconv2d_kernel(const Conv2dArgs a
     const int rs = warp / a.npt;                        // its slot among the warps of that tile
     const bool active = warp < a.npt * a.nrs;
     const int jbase = pt * (32 * P) + lane;
-    unsigned char* wbuf = reinterpret_cast<unsigned char*>(patch) + a.off_wbuf + warp * rec_buffer_bytes(G);
-    const float* xs = patch + jbase;                    // (positions past the end of the strip read on into
+    const uint32_t wbuf = patch_u32 + a.off_wbuf + warp * rec_buffer_bytes(G);
+    const uint32_t xs = patch_u32 + 4u * jbase;                    // (positions past the end of the strip read on into
                                                         //  the next channel or the slack: in bounds, never stored)
 
     for (int item = blockIdx.x; item < items; item += gridDim.x) {

@@ -303,13 +303,14 @@ typedef struct {
     int warps_per_tile;         /* warps that share one position tile and split its block rows      */
     int smem_bytes;             /* dynamic shared memory per thread block                           */
     int chunk_channels;         /* input channels staged at a time (cin: all at once)               */
+    int images_per_item;        /* whole images per work item (1, 2 or 4; > 1 only for small images) */
 } alcs_conv2d_cfg;
 
 ALCS_API int alcs_spconv2d(const alcs_packed* w, const void* x, void* y, int n, int cin, int h, int wd,
                            int kh, int kw, int stride, int pad, const float* bias, unsigned flags,
                            void* cuda_stream);
 /* Same, with parts of the launch configuration fixed (tests, tuning): non-zero positions_per_lane,
- * strip_rows, chunk_channels and row_groups of *cfg are taken as given (row_groups only when all
+ * strip_rows, chunk_channels, images_per_item and row_groups of *cfg are taken as given (row_groups only when all
  * channels are staged at once), the rest is chosen; UNSUPPORTED if nothing fits.  cfg == NULL
  * behaves like alcs_spconv2d. */
 ALCS_API int alcs_spconv2d_cfg(const alcs_packed* w, const void* x, void* y, int n, int cin, int h, int wd,

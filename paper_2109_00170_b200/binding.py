@@ -51,7 +51,7 @@ class LaunchCfg(C.Structure):
 
 class Conv2dCfg(C.Structure):
     _fields_ = [(k, C.c_int) for k in ("positions_per_lane", "strip_rows", "row_groups", "position_tiles",
-                                       "warps_per_tile", "smem_bytes", "chunk_channels")]
+                                       "warps_per_tile", "smem_bytes", "chunk_channels", "images_per_item")]
 
     def as_dict(self):
         return {k: getattr(self, k) for k, _ in self._fields_}

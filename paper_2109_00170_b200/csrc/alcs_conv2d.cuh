@@ -7,7 +7,8 @@
 // with the input vector the column offset addresses); what changes is what a column addresses:
 // the input image of channel c shifted by the tap (r, s).  I* is never materialised.
 //
-//   work item    = (image, strip of TH output rows, row group)
+//   work item    = (image, strip of TH output rows, row group); for images of at most 64 output
+//                  positions, (2 or 4 whole images, row group)
 //   thread block = persistent; per item it stages the input patch that the strip needs (halo and
 //                  zero padding included) in shared memory -- all input channels at once where
 //                  they fit, else chunk of channels after chunk -- and its warps multiply
@@ -51,7 +52,9 @@ struct Conv2dArgs {
     int kh, kw, pad;
     int th;                    // output rows per strip
     int n_strips, n_rg, rpg, n_img;
-    int wp, pr, pl, chw;       // plane pitch, plane rows, words per plane, words per channel
+    int wp, pr, pl, chw;       // plane pitch, plane rows, words per plane, words per channel and image
+    int chs;                   // words per channel of the staged patch = images per item * chw
+    int n_igrp;                // groups of NI images = work items per (strip, row group)
     int npt, nrs;              // position tiles per strip, warps per position tile
     int kc, nch;               // input channels per chunk, number of chunks
     int slack;                 // words after the patch that out-of-strip positions may read
@@ -69,15 +72,22 @@ __device__ __forceinline__ float lds_off(uint32_t p)
     asm volatile("ld.shared.f32 %0, [%1 + %2];\n" : "=f"(v) : "r"(p), "n"(OFF));
     return v;
 }
-template <int P, int... T>
-__device__ __forceinline__ void load_x2d_seq(uint32_t p, float2 (&x)[P / 2], std::integer_sequence<int, T...>)
+// Position t of a lane (t < P) belongs to image t / M of the work item's NI images, M = P / NI, and is
+// position lane + 32 * (t % M) inside it: which image and which immediate offset are compile-time
+// facts, so a column costs NI address additions and P loads.
+template <int P, int NI, int... T>
+__device__ __forceinline__ void load_x2d_seq(const uint32_t (&p)[NI], float2 (&x)[P / 2], std::integer_sequence<int, T...>)
 {
-    ((x[T].x = lds_off<256 * T>(p), x[T].y = lds_off<256 * T + 128>(p)), ...);
+    constexpr int M = P / NI;
+    ((x[T].x = lds_off<128 * ((2 * T) % M)>(p[(2 * T) / M]), x[T].y = lds_off<128 * ((2 * T + 1) % M)>(p[(2 * T + 1) / M])), ...);
 }
-template <int P>
-__device__ __forceinline__ void load_x2d(uint32_t xs, int byte_off, float2 (&x)[P / 2])
+template <int P, int NI>
+__device__ __forceinline__ void load_x2d(const uint32_t (&xs)[NI], int byte_off, float2 (&x)[P / 2])
 {
-    load_x2d_seq<P>(xs + (uint32_t)byte_off, x, std::make_integer_sequence<int, P / 2>{});
+    uint32_t p[NI];
+#pragma unroll
+    for (int i = 0; i < NI; ++i) p[i] = xs[i] + (uint32_t)byte_off;
+    load_x2d_seq<P, NI>(p, x, std::make_integer_sequence<int, P / 2>{});
 }
 
 __device__ __forceinline__ float4 lds_v4(uint32_t addr)
@@ -130,8 +140,8 @@ __host__ __device__ constexpr int rec_buffer_bytes(int g) { return 2 * rec_batch
 // the first pair's columns on entry and of the pair after the last one on return.  Same
 // two-register-set rotation as the pointwise kernel: the record and the input vectors of pair i+1
 // are loaded while pair i is multiplied.
-template <int G, int P>
-__device__ __forceinline__ void consume_batch2d(float2 (&acc)[G][P / 2], uint32_t xs, uint32_t rp, int n,
+template <int G, int P, int NI>
+__device__ __forceinline__ void consume_batch2d(float2 (&acc)[G][P / 2], const uint32_t (&xs)[NI], uint32_t rp, int n,
                                                 int& oa0, int& oa1)
 {
     constexpr int REC = record_bytes(G);
@@ -140,15 +150,15 @@ __device__ __forceinline__ void consume_batch2d(float2 (&acc)[G][P / 2], uint32_
         float wA0[G], wA1[G], wB0[G], wB1[G];
         float2 xA0[P / 2], xA1[P / 2], xB0[P / 2], xB1[P / 2];
         load_record_s<G>(rp, ob0, ob1, wA0, wA1);
-        load_x2d<P>(xs, oa0, xA0);
-        load_x2d<P>(xs, oa1, xA1);
+        load_x2d<P, NI>(xs, oa0, xA0);
+        load_x2d<P, NI>(xs, oa1, xA1);
         int left = n;                       // pairs not yet multiplied, A is loaded
         while (true) {
             const bool moreB = left > 1;
             if (moreB) {
                 load_record_s<G>(rp + REC, oa0, oa1, wB0, wB1);
-                load_x2d<P>(xs, ob0, xB0);
-                load_x2d<P>(xs, ob1, xB1);
+                load_x2d<P, NI>(xs, ob0, xB0);
+                load_x2d<P, NI>(xs, ob1, xB1);
             }
             fma_block<G, P>(acc, wA0, xA0);
             fma_block<G, P>(acc, wA1, xA1);
@@ -156,8 +166,8 @@ __device__ __forceinline__ void consume_batch2d(float2 (&acc)[G][P / 2], uint32_
             const bool moreA = left > 2;
             if (moreA) {
                 load_record_s<G>(rp + 2 * REC, ob0, ob1, wA0, wA1);
-                load_x2d<P>(xs, oa0, xA0);
-                load_x2d<P>(xs, oa1, xA1);
+                load_x2d<P, NI>(xs, oa0, xA0);
+                load_x2d<P, NI>(xs, oa1, xA1);
             }
             fma_block<G, P>(acc, wB0, xB0);
             fma_block<G, P>(acc, wB1, xB1);
@@ -171,8 +181,8 @@ __device__ __forceinline__ void consume_batch2d(float2 (&acc)[G][P / 2], uint32_
         for (int i = 0; i < n; ++i, rp += REC) {
             float2 x0[P / 2], x1[P / 2];
             float w[G];
-            load_x2d<P>(xs, oa0, x0);
-            load_x2d<P>(xs, oa1, x1);
+            load_x2d<P, NI>(xs, oa0, x0);
+            load_x2d<P, NI>(xs, oa1, x1);
             const float4 nx = lds_v4(rp);
 #pragma unroll
             for (int q = 0; q < G / 4; ++q) {
@@ -194,8 +204,8 @@ __device__ __forceinline__ void consume_batch2d(float2 (&acc)[G][P / 2], uint32_
 
 // Multiply-accumulate one whole block row (or its segment inside a channel chunk): `npairs` pair
 // records starting at rp in GLOBAL memory, streamed through this warp's double buffer `wbuf`.
-template <int G, int P>
-__device__ __forceinline__ void consume_row2d(float2 (&acc)[G][P / 2], uint32_t xs, const unsigned char* rp,
+template <int G, int P, int NI>
+__device__ __forceinline__ void consume_row2d(float2 (&acc)[G][P / 2], const uint32_t (&xs)[NI], const unsigned char* rp,
                                               int npairs, int oa0, int oa1, uint32_t wbuf_u32, int lane)
 {
     constexpr int REC = record_bytes(G);
@@ -218,13 +228,15 @@ __device__ __forceinline__ void consume_row2d(float2 (&acc)[G][P / 2], uint32_t 
             asm volatile("cp.async.wait_group 0;\n" ::: "memory");
         }
         __syncwarp();
-        consume_batch2d<G, P>(acc, xs, wbuf_u32 + (b & 1) * HALF, min(kRecBatch, npairs - b * kRecBatch), oa0, oa1);
+        consume_batch2d<G, P, NI>(acc, xs, wbuf_u32 + (b & 1) * HALF, min(kRecBatch, npairs - b * kRecBatch), oa0, oa1);
         __syncwarp();           // every lane has read this half before the fetch after next refills it
     }
 }
 
 // G = group size, P = positions per lane, ST = stride (1 or 2), NW = warps per thread block,
-// CHUNKED = which of the two ways through a work item this instance takes.
+// CHUNKED = which of the two ways through a work item this instance takes, NI = images per work item
+// (small images: NI > 1 puts NI whole images, each padded to 32 * P / NI positions, into one position
+// tile, so that a lane still owns P positions).
 //
 // Two ways through a work item.  With all input channels in one chunk (nch == 1) the warps that
 // share a position tile take block rows from a shared counter, one row at a time.  With the
@@ -232,7 +244,7 @@ __device__ __forceinline__ void consume_row2d(float2 (&acc)[G][P / 2], uint32_t 
 // ONE block row of the row group for the whole item, keeps its accumulators across the chunks, and
 // the block walks stage -> multiply -> stage -> ... ; the schedule then holds one segment per
 // (row group, chunk, row) with chunk-local offsets.
-template <int G, int P, int ST, int NW, bool CHUNKED>
+template <int G, int P, int ST, int NW, bool CHUNKED, int NI>
 __global__ void __launch_bounds__(NW * 32, 1) spconv2d_kernel(const Conv2dArgs a)
 {
     extern __shared__ __align__(16) float patch[];     // [kc][ST*ST][pr][wp], a.slack words, then the warps' record buffers
@@ -241,8 +253,9 @@ __global__ void __launch_bounds__(NW * 32, 1) spconv2d_kernel(const Conv2dArgs a
     const int tid = threadIdx.x;
     const int lane = tid & 31;
     const int warp = tid >> 5;
-    const int items = a.n_img * a.n_strips * a.n_rg;
-    const int patch_words = a.kc * a.chw;
+    constexpr int M = P / NI;                           // positions per lane and image
+    const int items = a.n_igrp * a.n_strips * a.n_rg;
+    const int patch_words = a.kc * a.chs;
     const uint32_t patch_u32 = (uint32_t)__cvta_generic_to_shared(patch);
     const int positions = a.th * a.wp;
 
@@ -254,13 +267,16 @@ __global__ void __launch_bounds__(NW * 32, 1) spconv2d_kernel(const Conv2dArgs a
     const bool active = warp < a.npt * a.nrs;
     const int jbase = pt * (32 * P) + lane;
     const uint32_t wbuf = patch_u32 + a.off_wbuf + warp * rec_buffer_bytes(G);
-    const uint32_t xs = patch_u32 + 4u * jbase;                    // (positions past the end of the strip read on into
-                                                        //  the next channel or the slack: in bounds, never stored)
+    // shared address of the lane's first position of each image (positions past the end of a strip
+    // or image read on into the next image, channel or the slack: in bounds, never stored)
+    uint32_t xs[NI];
+#pragma unroll
+    for (int i = 0; i < NI; ++i) xs[i] = patch_u32 + 4u * (uint32_t)(NI == 1 ? jbase : i * a.chw + lane);
 
     for (int item = blockIdx.x; item < items; item += gridDim.x) {
         const int rg = item % a.n_rg;
         const int strip = (item / a.n_rg) % a.n_strips;
-        const int img = item / (a.n_rg * a.n_strips);
+        const int img = item / (a.n_rg * a.n_strips) * NI;      // first image of the item
         const int oh0 = strip * a.th;
         const float* ximg = a.x + (size_t)img * a.cin * a.h * a.wd;
         float* yimg = a.y + (size_t)img * a.cout * a.oh * a.ow;
@@ -269,10 +285,11 @@ __global__ void __launch_bounds__(NW * 32, 1) spconv2d_kernel(const Conv2dArgs a
         int yoff[P];
 #pragma unroll
         for (int t = 0; t < P; ++t) {
-            const int j = jbase + 32 * t;
+            const int j = NI == 1 ? jbase + 32 * t : lane + 32 * (t % M);
             const int ol = j / a.wp;
             const int ow = j - ol * a.wp;
-            yoff[t] = (j < positions && ow < a.ow && oh0 + ol < a.oh) ? (oh0 + ol) * a.ow + ow : -1;
+            const bool ok = j < positions && ow < a.ow && oh0 + ol < a.oh && img + t / M < a.n_img;
+            yoff[t] = ok ? (NI == 1 ? 0 : (t / M) * a.cout * a.oh * a.ow) + (oh0 + ol) * a.ow + ow : -1;
         }
 
         // stage channels [c0, c0 + nc) of the strip's input window: one (channel, input row) per warp
@@ -281,17 +298,42 @@ __global__ void __launch_bounds__(NW * 32, 1) spconv2d_kernel(const Conv2dArgs a
         auto stage = [&](int c0, int nc) {
             const int ph_in = ST * a.pr, pw_in = ST * a.wp;
             const int ih0 = oh0 * ST - a.pad;
-            for (int idx = warp; idx < nc * ph_in; idx += NW) {
-                const int c = idx / ph_in;
-                const int rr = idx - c * ph_in;
-                const int ih = ih0 + rr;
-                const bool row_ok = ih >= 0 && ih < a.h;
-                const float* src = ximg + ((size_t)(c0 + c) * a.h + (row_ok ? ih : 0)) * a.wd;
-                const uint32_t dst = patch_u32 + 4u * (uint32_t)(c * a.chw + ((rr % ST) * ST) * a.pl + (rr / ST) * a.wp);
-                for (int cc = lane; cc < pw_in; cc += 32) {
-                    const int iw = cc - a.pad;
-                    const bool ok = row_ok && iw >= 0 && iw < a.wd;
-                    cp_async_4_zfill(dst + 4u * (uint32_t)((cc % ST) * a.pl + cc / ST), ok ? src + iw : ximg, ok ? 4 : 0);
+            if (pw_in > 16) {
+                // wide rows: one (channel, image, input row) per warp and pass, lanes along the row
+                for (int idx = warp; idx < nc * NI * ph_in; idx += NW) {
+                    const int c = idx / (NI * ph_in);
+                    const int rem = idx - c * (NI * ph_in);
+                    const int il = rem / ph_in;                     // image of the item
+                    const int rr = rem - il * ph_in;
+                    if (NI > 1 && img + il >= a.n_img) continue;    // (its slots keep stale values: never stored)
+                    const int ih = ih0 + rr;
+                    const bool row_ok = ih >= 0 && ih < a.h;
+                    const float* src = ximg + (((size_t)il * a.cin + c0 + c) * a.h + (row_ok ? ih : 0)) * a.wd;
+                    const uint32_t dst = patch_u32 + 4u * (uint32_t)(c * a.chs + il * a.chw + ((rr % ST) * ST) * a.pl + (rr / ST) * a.wp);
+                    for (int cc = lane; cc < pw_in; cc += 32) {
+                        const int iw = cc - a.pad;
+                        const bool ok = row_ok && iw >= 0 && iw < a.wd;
+                        cp_async_4_zfill(dst + 4u * (uint32_t)((cc % ST) * a.pl + cc / ST), ok ? src + iw : ximg, ok ? 4 : 0);
+                    }
+                }
+            } else {
+                // narrow rows (small images): one (channel, image) window per warp and pass, lanes over
+                // all of its rows and columns, so that most lanes have an element to copy
+                const int win = ph_in * pw_in;
+                for (int idx = warp; idx < nc * NI; idx += NW) {
+                    const int c = idx / NI;
+                    const int il = idx - c * NI;
+                    if (NI > 1 && img + il >= a.n_img) continue;
+                    const float* src = ximg + ((size_t)il * a.cin + c0 + c) * a.h * a.wd;
+                    const uint32_t dst = patch_u32 + 4u * (uint32_t)(c * a.chs + il * a.chw);
+                    for (int e = lane; e < win; e += 32) {
+                        const int rr = e / pw_in;
+                        const int cc = e - rr * pw_in;
+                        const int ih = ih0 + rr, iw = cc - a.pad;
+                        const bool ok = ih >= 0 && ih < a.h && iw >= 0 && iw < a.wd;
+                        cp_async_4_zfill(dst + 4u * (uint32_t)(((rr % ST) * ST + cc % ST) * a.pl + (rr / ST) * a.wp + cc / ST),
+                                         ok ? src + ih * a.wd + iw : ximg, ok ? 4 : 0);
+                    }
                 }
             }
             cp_async_wait_all();
@@ -337,7 +379,7 @@ __global__ void __launch_bounds__(NW * 32, 1) spconv2d_kernel(const Conv2dArgs a
                     for (int e = 0; e < P / 2; ++e) acc[j][e] = make_float2(0.0f, 0.0f);
                 if (hd.w > 0) {
                     const unsigned char* rp = recs + (size_t)hd.x * 16;
-                    consume_row2d<G, P>(acc, xs, rp, hd.w, hd.y, hd.z, wbuf, lane);
+                    consume_row2d<G, P, NI>(acc, xs, rp, hd.w, hd.y, hd.z, wbuf, lane);
                 }
                 epilogue(row, acc);
             }
@@ -357,7 +399,7 @@ __global__ void __launch_bounds__(NW * 32, 1) spconv2d_kernel(const Conv2dArgs a
                 const int4 hd = __ldg(reinterpret_cast<const int4*>(a.rowoff) + ((size_t)rg * a.nch + k) * a.rpg + rs);
                 if (hd.w > 0) {
                     const unsigned char* rp = a.rec + ((size_t)__ldg(a.slice + rg * a.nch + k) + hd.x) * 16;
-                    consume_row2d<G, P>(acc, xs, rp, hd.w, hd.y, hd.z, wbuf, lane);
+                    consume_row2d<G, P, NI>(acc, xs, rp, hd.w, hd.y, hd.z, wbuf, lane);
                 }
             }
             if (row >= 0) epilogue(row, acc);
@@ -371,8 +413,8 @@ __global__ void __launch_bounds__(NW * 32, 1) spconv2d_kernel(const Conv2dArgs a
 constexpr int kConv2dWarps = 16;
 // dynamic shared memory a block may ask for: the 227 KB per-block limit minus the kernel's static part
 constexpr int kConv2dMaxDynSmem = 227 * 1024 - 256;
-bool conv2d_variant_exists(int g, int p, int stride);
-cudaError_t launch_conv2d(int g, int p, int stride, const Conv2dArgs& a, unsigned grid, size_t smem, cudaStream_t st);
+bool conv2d_variant_exists(int g, int p, int stride, int ni);
+cudaError_t launch_conv2d(int g, int p, int stride, int ni, const Conv2dArgs& a, unsigned grid, size_t smem, cudaStream_t st);
 
 }  // namespace alcs
 

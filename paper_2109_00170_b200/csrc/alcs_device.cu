@@ -1024,6 +1024,7 @@ struct Conv2dPlan {
     int npt = 0, nrs = 0;
     int wp = 0, pr = 0, pl = 0, chw = 0, slack = 0;
     int kc = 0, nch = 0;     // input channels per chunk, chunks
+    int ni = 1;              // images per work item
     size_t smem = 0;
     double cost = 0;    // model estimate, cycles per SM
 };
@@ -1040,8 +1041,10 @@ int plan_conv2d(const alcs_packed* w, const Conv2dGeom& g, int sms, int smem_max
     const int halo = (g.kh - 1) / g.st;
     Conv2dPlan best;
     best.cost = 1e300;
+    for (int ni = 1; ni <= 4; ni *= 2)
     for (int p = 8; p >= 2; p /= 2) {
-        if (!alcs::conv2d_variant_exists(w->g, p, g.st)) continue;
+        if (!alcs::conv2d_variant_exists(w->g, p, g.st, ni)) continue;
+        if (force && force->images_per_item && force->images_per_item != ni) continue;
         if (force && force->positions_per_lane && force->positions_per_lane != p) continue;
         // sustained fraction of the fp32 peak in the hot loop: per pair of blocks 2P X wavefronts
         // plus 3 of records against 16P/8 cycles of FMA issue
@@ -1049,19 +1052,21 @@ int plan_conv2d(const alcs_packed* w, const Conv2dGeom& g, int sms, int smem_max
         for (int th = 1; th <= g.oh; ++th) {
             if (force && force->strip_rows && force->strip_rows != th) continue;
             const int positions = th * wp;
-            const int npt = (positions + 32 * p - 1) / (32 * p);
+            // several images per item: whole images only, each within its 32 * p / ni position slots
+            if (ni > 1 && (th != g.oh || positions > 32 * p / ni)) continue;
+            const int npt = ni > 1 ? 1 : (positions + 32 * p - 1) / (32 * p);
             if (npt > NW) break;
             const int pr = th + halo;
             const long long chw = (long long)g.st * g.st * pr * wp;
-            const int slack = npt * 32 * p - positions + 8;
+            const int slack = (ni > 1 ? 32 * p / ni : npt * 32 * p) - positions + 8;
             const int nrs = NW / npt;
             const int n_strips = (g.oh + th - 1) / th;
-            const long long base_items = (long long)g.n * n_strips;
+            const long long base_items = (long long)((g.n + ni - 1) / ni) * n_strips;
             // channels per chunk: all of them if the patch fits, else halves, quarters, ...
             for (int nch = 1; nch <= g.cin; nch *= 2) {
                 const int kc = (force && force->chunk_channels) ? std::min(force->chunk_channels, g.cin) : (g.cin + nch - 1) / nch;
                 const int nch_real = (g.cin + kc - 1) / kc;
-                const long long smem = (((long long)kc * chw + slack) * 4 + 15) / 16 * 16 + (long long)NW * alcs::rec_buffer_bytes(w->g);
+                const long long smem = (((long long)kc * chw * ni + slack) * 4 + 15) / 16 * 16 + (long long)NW * alcs::rec_buffer_bytes(w->g);
                 if (smem > smem_max) { if (force && force->chunk_channels) break; continue; }
                 // one chunk: warps take rows from a counter, any number of row groups; several chunks:
                 // one row per warp, so the row groups are fixed by the warps per position tile
@@ -1072,7 +1077,7 @@ int plan_conv2d(const alcs_packed* w, const Conv2dGeom& g, int sms, int smem_max
                     if (force && force->row_groups && nch_real == 1 && force->row_groups != n_rg) continue;
                     const long long items = base_items * n_rg;
                     const long long rounds = (items + sms - 1) / sms;
-                    const double stage = (double)g.cin * chw / 16.0 + 1500.0 * nch_real;
+                    const double stage = (double)g.cin * chw * ni / 16.0 + 1500.0 * nch_real;
                     const double blocks_item = (double)w->nb / n_rg;
                     const double fma = blocks_item * npt * (double)(w->g * p * 32);
                     // warps that share a position tile split its rows; idle warps (NW not a multiple of
@@ -1085,7 +1090,7 @@ int plan_conv2d(const alcs_packed* w, const Conv2dGeom& g, int sms, int smem_max
                         best.p = p; best.th = th; best.n_strips = n_strips; best.n_rg = n_rg;
                         best.npt = npt; best.nrs = nrs; best.wp = wp; best.pr = pr; best.pl = pr * wp;
                         best.chw = (int)chw; best.slack = slack; best.smem = (size_t)smem; best.cost = cost;
-                        best.kc = kc; best.nch = nch_real;
+                        best.kc = kc; best.nch = nch_real; best.ni = ni;
                     }
                 }
                 break;      // the largest chunk that fits is the one to use for this (p, th)
@@ -1101,7 +1106,8 @@ int plan_conv2d(const alcs_packed* w, const Conv2dGeom& g, int sms, int smem_max
 // offset of that column's (channel, tap) inside the shared-memory patch.
 Schedule* get_schedule2d(const alcs_packed* w, const Conv2dGeom& g, const Conv2dPlan& p)
 {
-    const std::array<int, 8> key = {p.n_rg, p.chw, p.pl, p.wp, g.st, g.kh, g.kw, p.kc};
+    const int chs = p.chw * p.ni;      // words per channel of the staged patch
+    const std::array<int, 8> key = {p.n_rg, chs, p.pl, p.wp, g.st, g.kh, g.kw, p.kc};
     std::lock_guard<std::mutex> lk(w->mu);
     auto it = w->sched2d.find(key);
     if (it != w->sched2d.end()) return &it->second;
@@ -1112,7 +1118,7 @@ Schedule* get_schedule2d(const alcs_packed* w, const Conv2dGeom& g, const Conv2d
         auto coloff = [&](int col) {
             const int c = col / taps, tap = col - c * taps;
             const int r = tap / g.kw, s = tap - r * g.kw;
-            return 4 * (c * p.chw + ((r % g.st) * g.st + (s % g.st)) * p.pl + (r / g.st) * p.wp + s / g.st);
+            return 4 * (c * chs + ((r % g.st) * g.st + (s % g.st)) * p.pl + (r / g.st) * p.wp + s / g.st);
         };
         const int REC = alcs::record_bytes(w->g);
         // (columns inside a chunk are chunk-local, and a chunk starts at a channel boundary, so the
@@ -1182,7 +1188,7 @@ extern "C" ALCS_API int alcs_spconv2d_plan(const alcs_packed* w, int n, int cin,
     if (rc) return rc;
     out->positions_per_lane = p.p; out->strip_rows = p.th; out->row_groups = p.n_rg;
     out->position_tiles = p.npt; out->warps_per_tile = p.nrs; out->smem_bytes = (int)p.smem;
-    out->chunk_channels = p.kc;
+    out->chunk_channels = p.kc; out->images_per_item = p.ni;
     return ALCS_OK;
 }
 
@@ -1217,13 +1223,14 @@ extern "C" ALCS_API int alcs_spconv2d_cfg(const alcs_packed* w, const void* x, v
     a.th = p.th; a.n_strips = p.n_strips; a.n_rg = sc->n_rg; a.rpg = sc->rpg; a.n_img = n;
     a.wp = p.wp; a.pr = p.pr; a.pl = p.pl; a.chw = p.chw; a.npt = p.npt; a.nrs = p.nrs; a.slack = p.slack;
     a.kc = p.kc; a.nch = sc->nch;
-    a.off_wbuf = (int)(((size_t)p.kc * p.chw + p.slack) * 4 + 15) / 16 * 16;
+    a.chs = p.chw * p.ni; a.n_igrp = (n + p.ni - 1) / p.ni;
+    a.off_wbuf = (int)(((size_t)p.kc * a.chs + p.slack) * 4 + 15) / 16 * 16;
     if (sc->nch != p.nch || (sc->nch > 1 && sc->rpg > p.nrs)) return ALCS_ERR_STATE;      // (cannot happen: plan and schedule agree)
     a.relu = (flags & ALCS_RELU) ? 1 : 0;
-    const long long items = (long long)n * p.n_strips * sc->n_rg;
+    const long long items = (long long)a.n_igrp * p.n_strips * sc->n_rg;
     if (items > 0x7fffffffll) return ALCS_ERR_SHAPE;
     const unsigned grid = (unsigned)std::min<long long>(items, di.sms);
-    ALCS_CUDA(alcs::launch_conv2d(w->g, p.p, stride, a, grid, p.smem, st));
+    ALCS_CUDA(alcs::launch_conv2d(w->g, p.p, stride, p.ni, a, grid, p.smem, st));
     return ALCS_OK;
 }
 

@@ -58,6 +58,7 @@ GEOMS = [  # n, cin, cout, h, w, kh, kw, stride, pad, g
     (2, 32, 32, 7, 7, 3, 3, 1, 1, 16),
     (2, 32, 17, 7, 7, 3, 3, 1, 1, 1),        # unstructured
     (4, 20, 24, 12, 40, 1, 1, 1, 0, 4),      # 1x1 through the general path
+    (3, 32, 16, 15, 14, 1, 1, 2, 0, 4),      # strided 1x1 (projection shortcuts of ResNets)
     (1, 5, 8, 33, 65, 3, 2, 1, 1, 4),        # even kernel width, wide image
     (1, 64, 64, 28, 28, 3, 3, 2, 1, 4),
 ]
@@ -84,6 +85,17 @@ def test_conv2d_forced_configurations(alcs, cfg, stride):
     Y = _run(alcs, W, M, X, b, True, 4, stride, 1, cfg)
     Yref, A = oracle.conv2d(W, M, X, b, True, 4, stride, 1, want_scale=True)
     assert_parity(Y, Yref, A, "f32")
+
+
+@pytest.mark.parametrize("stride", [1, 2])
+def test_conv2d_several_images_per_item(alcs, stride):
+    """Small images: 2 or 4 whole images share one position tile (odd batch: the last item is short),
+    with all channels at once and with channel chunks."""
+    W, M, X, b = _case(93, 7, 20, 24, 7 * stride, 7 * stride, 3, 3, 4)
+    Yref, A = oracle.conv2d(W, M, X, b, True, 4, stride, 1, want_scale=True)
+    for cfg in (dict(images_per_item=4), dict(images_per_item=2, positions_per_lane=4),
+                dict(images_per_item=4, chunk_channels=8), dict(images_per_item=2, chunk_channels=7)):
+        assert_parity(_run(alcs, W, M, X, b, True, 4, stride, 1, cfg), Yref, A, "f32")
 
 
 @pytest.mark.parametrize("stride", [1, 2])

@@ -1030,7 +1030,7 @@ struct Conv2dPlan {
 };
 
 // Choose positions per lane, strip height and row-group count by a small cost model: per work item
-// the patch is staged once (about 16 words per cycle per SM from L2) and every kept block costs
+// the patch is staged once (element-wise copies, about 2 words per cycle per SM) and every kept block costs
 // G*P*32 FMAs per position tile at the rate the shared-memory-bound hot loop sustains; items are
 // dealt to one persistent thread block per SM.
 int plan_conv2d(const alcs_packed* w, const Conv2dGeom& g, int sms, int smem_max, Conv2dPlan* out,
@@ -1077,7 +1077,8 @@ int plan_conv2d(const alcs_packed* w, const Conv2dGeom& g, int sms, int smem_max
                     if (force && force->row_groups && nch_real == 1 && force->row_groups != n_rg) continue;
                     const long long items = base_items * n_rg;
                     const long long rounds = (items + sms - 1) / sms;
-                    const double stage = (double)g.cin * chw * ni / 16.0 + 1500.0 * nch_real;
+                    // (measured: the 4-byte staging copies sustain about 2 words per cycle and SM)
+                    const double stage = (double)g.cin * chw * ni / 2.0 + 1500.0 * nch_real;
                     const double blocks_item = (double)w->nb / n_rg;
                     const double fma = blocks_item * npt * (double)(w->g * p * 32);
                     // warps that share a position tile split its rows; idle warps (NW not a multiple of

@@ -299,21 +299,47 @@ __global__ void __launch_bounds__(NW * 32, 1) spconv2d_kernel(const Conv2dArgs a
             const int ph_in = ST * a.pr, pw_in = ST * a.wp;
             const int ih0 = oh0 * ST - a.pad;
             if (pw_in > 16) {
-                // wide rows: one (channel, image, input row) per warp and pass, lanes along the row
-                for (int idx = warp; idx < nc * NI * ph_in; idx += NW) {
-                    const int c = idx / (NI * ph_in);
-                    const int rem = idx - c * (NI * ph_in);
-                    const int il = rem / ph_in;                     // image of the item
-                    const int rr = rem - il * ph_in;
-                    if (NI > 1 && img + il >= a.n_img) continue;    // (its slots keep stale values: never stored)
-                    const int ih = ih0 + rr;
-                    const bool row_ok = ih >= 0 && ih < a.h;
-                    const float* src = ximg + (((size_t)il * a.cin + c0 + c) * a.h + (row_ok ? ih : 0)) * a.wd;
-                    const uint32_t dst = patch_u32 + 4u * (uint32_t)(c * a.chs + il * a.chw + ((rr % ST) * ST) * a.pl + (rr / ST) * a.wp);
-                    for (int cc = lane; cc < pw_in; cc += 32) {
-                        const int iw = cc - a.pad;
-                        const bool ok = row_ok && iw >= 0 && iw < a.wd;
-                        cp_async_4_zfill(dst + 4u * (uint32_t)((cc % ST) * a.pl + cc / ST), ok ? src + iw : ximg, ok ? 4 : 0);
+                // wide rows: one (channel, image, input row) per warp and pass, lanes along the row.  What
+                // depends only on the column (source column, destination offset, inside the image or not)
+                // is worked out once per call; the row index advances without divisions.
+                constexpr int kPass = 4;                            // columns per lane handled from registers
+                int col_src[kPass];
+                uint32_t col_dst[kPass];
+                bool col_in[kPass], col_ok[kPass];
+#pragma unroll
+                for (int k = 0; k < kPass; ++k) {
+                    const int cc = lane + 32 * k;
+                    col_in[k] = cc < pw_in;
+                    col_src[k] = cc - a.pad;
+                    col_ok[k] = col_in[k] && col_src[k] >= 0 && col_src[k] < a.wd;
+                    col_dst[k] = 4u * (uint32_t)((cc % ST) * a.pl + cc / ST);
+                }
+                const int total = nc * NI * ph_in;
+                int c = warp / (NI * ph_in);
+                int il = (warp - c * (NI * ph_in)) / ph_in;
+                int rr = warp - (c * NI + il) * ph_in;
+                for (int idx = warp; idx < total; idx += NW) {
+                    if (NI == 1 || img + il < a.n_img) {            // (a missing image's slots keep stale values: never stored)
+                        const int ih = ih0 + rr;
+                        const bool row_ok = ih >= 0 && ih < a.h;
+                        const float* src = ximg + (((size_t)il * a.cin + c0 + c) * a.h + (row_ok ? ih : 0)) * a.wd;
+                        const uint32_t dst = patch_u32 + 4u * (uint32_t)(c * a.chs + il * a.chw + ((rr % ST) * ST) * a.pl + (rr / ST) * a.wp);
+#pragma unroll
+                        for (int k = 0; k < kPass; ++k) {
+                            if (!col_in[k]) continue;
+                            const bool ok = row_ok && col_ok[k];
+                            cp_async_4_zfill(dst + col_dst[k], ok ? src + col_src[k] : ximg, ok ? 4 : 0);
+                        }
+                        for (int cc = lane + 32 * kPass; cc < pw_in; cc += 32) {      // images wider than 128 columns
+                            const int iw = cc - a.pad;
+                            const bool ok = row_ok && iw >= 0 && iw < a.wd;
+                            cp_async_4_zfill(dst + 4u * (uint32_t)((cc % ST) * a.pl + cc / ST), ok ? src + iw : ximg, ok ? 4 : 0);
+                        }
+                    }
+                    rr += NW;
+                    while (rr >= ph_in) {
+                        rr -= ph_in;
+                        if (++il == NI) { il = 0; ++c; }
                     }
                 }
             } else {

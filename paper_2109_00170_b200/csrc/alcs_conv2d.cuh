@@ -202,6 +202,43 @@ __device__ __forceinline__ void consume_batch2d(float2 (&acc)[G][P / 2], const u
     }
 }
 
+// A FULL batch of rec_batch(G) (an even number of) pair records: the same rotation without any loop
+// test, fully unrolled, so that the only branches left in the steady state are the batch loop's.
+template <int G, int P, int NI>
+__device__ __forceinline__ void consume_full_batch2d(float2 (&acc)[G][P / 2], const uint32_t (&xs)[NI], uint32_t rp,
+                                                     int& oa0, int& oa1)
+{
+    constexpr int REC = record_bytes(G);
+    constexpr int N = rec_batch(G);
+    static_assert(N % 2 == 0, "the unrolled rotation handles the records two by two");
+    if constexpr (G <= 4) {
+        int ob0 = 0, ob1 = 0;
+        float wA0[G], wA1[G], wB0[G], wB1[G];
+        float2 xA0[P / 2], xA1[P / 2], xB0[P / 2], xB1[P / 2];
+        load_record_s<G>(rp, ob0, ob1, wA0, wA1);
+        load_x2d<P, NI>(xs, oa0, xA0);
+        load_x2d<P, NI>(xs, oa1, xA1);
+#pragma unroll
+        for (int i = 0; i < N / 2; ++i) {
+            load_record_s<G>(rp + (2 * i + 1) * REC, oa0, oa1, wB0, wB1);
+            load_x2d<P, NI>(xs, ob0, xB0);
+            load_x2d<P, NI>(xs, ob1, xB1);
+            fma_block<G, P>(acc, wA0, xA0);
+            fma_block<G, P>(acc, wA1, xA1);
+            if (i + 1 < N / 2) {
+                load_record_s<G>(rp + (2 * i + 2) * REC, ob0, ob1, wA0, wA1);
+                load_x2d<P, NI>(xs, oa0, xA0);
+                load_x2d<P, NI>(xs, oa1, xA1);
+            }
+            fma_block<G, P>(acc, wB0, xB0);
+            fma_block<G, P>(acc, wB1, xB1);
+        }
+        // (oa0, oa1) now hold the header of the last record: the columns of the pair after the batch
+    } else {
+        consume_batch2d<G, P, NI>(acc, xs, rp, N, oa0, oa1);
+    }
+}
+
 // Multiply-accumulate one whole block row (or its segment inside a channel chunk): `npairs` pair
 // records starting at rp in GLOBAL memory, streamed through this warp's double buffer `wbuf`.
 template <int G, int P, int NI>
@@ -228,7 +265,9 @@ __device__ __forceinline__ void consume_row2d(float2 (&acc)[G][P / 2], const uin
             asm volatile("cp.async.wait_group 0;\n" ::: "memory");
         }
         __syncwarp();
-        consume_batch2d<G, P, NI>(acc, xs, wbuf_u32 + (b & 1) * HALF, min(kRecBatch, npairs - b * kRecBatch), oa0, oa1);
+        const int nrec = min(kRecBatch, npairs - b * kRecBatch);
+        if (nrec == kRecBatch) consume_full_batch2d<G, P, NI>(acc, xs, wbuf_u32 + (b & 1) * HALF, oa0, oa1);
+        else consume_batch2d<G, P, NI>(acc, xs, wbuf_u32 + (b & 1) * HALF, nrec, oa0, oa1);
         __syncwarp();           // every lane has read this half before the fetch after next refills it
     }
 }

@@ -117,6 +117,10 @@ float half_bits_to_float(uint16_t h);
 void build_schedule(const alcs_packed& p, int kc, int n_rg, bool with_records, Schedule& out);
 void build_schedule_mma(const alcs_packed& p, int kc, int n_rg, bool with_records, Schedule& out);
 inline std::pair<int, int> sched_key(int kc, int n_rg, int mma) { return std::make_pair(mma ? -kc : kc, n_rg); }
+// Device-side helpers implemented in alcs_device.cu, for the library's other translation units.
+int device_limits(int device, int* sms, int* smem_optin);                 // SM count, opt-in shared memory per block
+int schedule_upload(const alcs_packed* w, Schedule* sc, void* cuda_stream); // copy a schedule to w's device (once)
+int require_current_device(const alcs_packed* w);                          // ALCS_OK if w is uploaded and its device is current
 // bytes of one step record of the tensor-core flavour
 constexpr int step_record_bytes(int g) { return 32 + 32 * (g < 8 ? 8 : g); }
 

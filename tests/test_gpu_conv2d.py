@@ -147,6 +147,18 @@ def test_conv2d_resnet18_layers_sampled(alcs):
         assert np.isfinite(Y).all() and np.all(d <= 1e-5 * m + 1e-300), s.name
 
 
+def test_conv2d_resnet18_layers_full_batch_sampled(alcs):
+    """The same layers at the benchmark's batch (32), i.e. in the launch configurations the benchmark
+    times (several images per item, channel chunks, small strips): sampled points against the oracle."""
+    for s in resnet18_3x3_stack(batch=32):
+        W, M, X, b = make_weights2d(s), make_mask2d(s), make_x2d(s), make_bias2d(s)
+        Y = _run(alcs, W, M, X, b, True, s.g, s.stride, s.pad)
+        idx = np.concatenate([rng.permutation(s.seed, 10, Y.size)[:6000], np.arange(Y.size - 200, Y.size), np.arange(200)])
+        v, m = oracle.conv2d_points(W, M, X, idx, b, True, s.g, s.stride, s.pad)
+        d = np.abs(Y.reshape(-1)[idx].astype(np.float64) - v)
+        assert np.isfinite(Y).all() and np.all(d <= 1e-5 * m + 1e-300), s.name
+
+
 def test_conv2d_errors(alcs):
     import torch
     W, M, X, b = _case(79, 1, 4, 8, 6, 6, 3, 3, 4)

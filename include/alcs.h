@@ -165,7 +165,12 @@ ALCS_API void alcs_packed_free(alcs_packed* p);
  *   math_mode         1 = fp32 FMA on the CUDA cores; 2 = tensor cores (fp16 weights and activations
  *                     only): 16 kept blocks of a block row times the 16 input rows they select is a
  *                     dense 16 x g by 16 x pixels contraction, run as warp-level MMA with fp32
- *                     accumulation
+ *                     accumulation; 3 = the small-problem kernel (fp32 only, meant for batch 1): no
+ *                     staging of X, a thread block is one (block row, image, pixel tile) and its `warps`
+ *                     (1..16) warps share the row's kept columns, reading the canonical storage format and
+ *                     the input vectors straight from global memory; partial sums are added in a fixed
+ *                     order.  Only pixels_per_lane (2, 4, 8; g * pixels_per_lane <= 32) and warps apply;
+ *                     the device copy of the storage format is made on its first use with a packed matrix
  *   consumer_groups   1 = all consumer warps work on one work item at a time; 2 = two halves of the
  *                     consumer warps take the thread block's work items alternately (tensor-core
  *                     kernels only), so that one half multiplies while the other half stores

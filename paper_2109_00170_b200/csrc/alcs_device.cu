@@ -10,6 +10,7 @@
 #include <new>
 #include <vector>
 
+#include "alcs_gather.h"
 #include "alcs_internal.h"
 #include "alcs_kernels.cuh"
 
@@ -222,6 +223,29 @@ int occupancy_of(const VariantInfo& vi, size_t smem)
     return occ;
 }
 
+// The small-problem kernel as a plan.  Its cost estimate is a latency model: a warp issues the loads of
+// a few blocks at a time and waits about one L2 round trip for each batch; the arithmetic term makes it
+// lose against the staged kernels as soon as there is enough work to keep the SMs busy.
+bool gather_plan(const alcs_packed* w, int n, int hw, int p, int ks, int sms, Plan* out)
+{
+    if (w->dt != ALCS_F32) return false;
+    if (!alcs::gather_config_ok(w->g, p, ks, false)) return false;
+    const long long tiles = (hw + 32 * p - 1) / (32 * p);
+    const long long blocks = (long long)w->rows * n * tiles;
+    if (blocks > (1ll << 22)) return false;
+    Plan pl;
+    pl.variant = -1; pl.gather = 1; pl.gp = p; pl.gks = ks;
+    const double per_row = w->rows ? (double)w->nb / w->rows : 0.0;
+    const double batches = std::ceil(per_row / ks / 4.0);
+    const double resident = std::max(1.0, std::floor(2048.0 / (ks * 32)));          // thread blocks per SM
+    const double rounds = std::ceil((double)blocks / (sms * resident));
+    const double latency = rounds * (batches * 900.0 + 2500.0);
+    const double alu = (double)w->nb * w->g * n * tiles * 32.0 * p / (sms * 128.0 * 0.25);
+    pl.cost = std::max(latency, alu) / 1.9e9;
+    *out = pl;
+    return true;
+}
+
 // Enumerate every valid launch configuration for this shape, cheapest (by the model) first.
 int enumerate_plans(const alcs_packed* w, long long q, int hw, std::vector<Plan>& out)
 {
@@ -290,12 +314,26 @@ int enumerate_plans(const alcs_packed* w, long long q, int hw, std::vector<Plan>
             }
         }
     }
+    if (hw > 0 && q / hw <= 64) {       // small batches only: one thread block per (block row, image, pixel tile)
+        for (int p = 8; p >= 2; p /= 2)
+            for (int ks = 4; ks <= 16; ks *= 2) {
+                Plan g;
+                if (gather_plan(w, (int)(q / hw), hw, p, ks, di.sms, &g)) out.push_back(g);
+            }
+    }
     std::stable_sort(out.begin(), out.end(), [](const Plan& a, const Plan& b) { return a.cost < b.cost; });
     return out.empty() ? ALCS_ERR_UNSUPPORTED : ALCS_OK;
 }
 
 void plan_to_cfg(const Plan& p, alcs_launch_cfg* c)
 {
+    if (p.gather) {
+        std::memset(c, 0, sizeof *c);
+        c->pixels_per_lane = p.gp;
+        c->warps = p.gks;
+        c->math_mode = 3;
+        return;
+    }
     const KernelVariant& v = g_variants[p.variant].v;
     c->pixels_per_lane = v.p;
     c->rows_per_warp = v.rw;
@@ -317,7 +355,21 @@ int cfg_to_plan(const alcs_packed* w, long long q, int hw, const alcs_launch_cfg
     int rc = enumerate_plans(w, q, hw, all);
     if (rc) return rc;
     if (!c) { *out = all[0]; return ALCS_OK; }
+    if (c->math_mode == 3) {        // the small-problem kernel, with the given (or the best-ranked) shape
+        for (const Plan& p : all)
+            if (p.gather && (!c->pixels_per_lane || c->pixels_per_lane == p.gp) && (!c->warps || c->warps == p.gks)) {
+                *out = p;
+                return ALCS_OK;
+            }
+        DeviceInfo di;
+        rc = device_info(w->device, &di);
+        if (rc) return rc;
+        if (hw > 0 && c->pixels_per_lane && c->warps &&
+            gather_plan(w, (int)(q / hw), hw, c->pixels_per_lane, c->warps, di.sms, out)) return ALCS_OK;
+        return ALCS_ERR_UNSUPPORTED;
+    }
     auto variant_ok = [&](const Plan& p) {
+        if (p.gather) return false;
         const KernelVariant& v = g_variants[p.variant].v;
         if (c->pixels_per_lane && c->pixels_per_lane != v.p) return false;
         if (c->rows_per_warp && c->rows_per_warp != v.rw) return false;
@@ -426,9 +478,55 @@ int check_conv_args(const alcs_packed* w, const void* x, const void* y, int n, i
     return ALCS_OK;
 }
 
+// Device copy of the canonical storage format (row_ptr, col_idx, vals) for the small-problem kernel:
+// made the first time that kernel is used with w (allocates, and waits for the copy), kept until w is freed.
+int ensure_canonical_on_device(const alcs_packed* w, cudaStream_t st)
+{
+    std::lock_guard<std::mutex> lk(w->mu);
+    if (w->d_row_ptr) return ALCS_OK;
+    int32_t *rp = nullptr, *ci = nullptr;
+    void* va = nullptr;
+    cudaError_t e = cudaMalloc(&rp, w->row_ptr.size() * 4);
+    if (e == cudaSuccess) e = cudaMalloc(&ci, std::max<size_t>(w->col_idx.size() * 4, 16));
+    if (e == cudaSuccess) e = cudaMalloc(&va, std::max<size_t>(w->vals.size(), 16));
+    if (e == cudaSuccess) e = cudaMemcpyAsync(rp, w->row_ptr.data(), w->row_ptr.size() * 4, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && !w->col_idx.empty())
+        e = cudaMemcpyAsync(ci, w->col_idx.data(), w->col_idx.size() * 4, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && !w->vals.empty()) e = cudaMemcpyAsync(va, w->vals.data(), w->vals.size(), cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) {
+        alcs::set_cuda_error_text(cudaGetErrorString(e));
+        cudaFree(rp); cudaFree(ci); cudaFree(va);
+        (void)cudaGetLastError();
+        return e == cudaErrorMemoryAllocation ? ALCS_ERR_ALLOC : ALCS_ERR_CUDA;
+    }
+    w->d_col_idx = ci; w->d_vals = va;
+    w->d_row_ptr = rp;
+    return ALCS_OK;
+}
+
+// Launch the small-problem kernel; the canonical arrays must be on the device.
+int launch_gather_plan(const alcs_packed* w, const Plan& p, const void* x, void* y, int n, int h, int wd,
+                       const float* bias, unsigned flags, cudaStream_t st)
+{
+    alcs::GatherArgs a;
+    a.x = static_cast<const float*>(x); a.y = static_cast<float*>(y); a.bias = bias;
+    a.row_ptr = w->d_row_ptr; a.col_idx = w->d_col_idx; a.vals = static_cast<const float*>(w->d_vals);
+    a.rows = w->rows; a.cin = w->cin; a.cout = w->cout; a.hw = h * wd; a.n = n;
+    a.tiles = (a.hw + 32 * p.gp - 1) / (32 * p.gp);
+    a.relu = (flags & ALCS_RELU) ? 1 : 0;
+    a.vec = (p.gp >= 4 && a.hw % 4 == 0 && (uintptr_t)x % 16 == 0) ? 1 : 0;
+    ALCS_CUDA(alcs::launch_gather(w->g, p.gp, p.gks, a, st));
+    return ALCS_OK;
+}
+
 int launch_plan(const alcs_packed* w, const Plan& p, const void* x, void* y, int n, int h, int wd,
                 const float* bias, unsigned flags, cudaStream_t st)
 {
+    if (p.gather) {
+        const int rc = ensure_canonical_on_device(w, st);
+        return rc ? rc : launch_gather_plan(w, p, x, y, n, h, wd, bias, flags, st);
+    }
     const KernelVariant& v = g_variants[p.variant].v;
     Schedule* sc = get_schedule(w, p.kc, p.n_rg, true, v.mma);
     if (!sc) return ALCS_ERR_ALLOC;
@@ -621,6 +719,7 @@ ALCS_API void alcs_packed_free(alcs_packed* p)
             for (auto& kv : p->sched2d) free_schedule_device(kv.second);
             cudaFree(p->d_err);
             cudaFree(p->d_xpad);
+            cudaFree(p->d_row_ptr); cudaFree(p->d_col_idx); cudaFree(p->d_vals);
             cudaSetDevice(prev);
         }
         (void)cudaGetLastError();
@@ -759,7 +858,9 @@ ALCS_API int alcs_spconv1x1_tune(alcs_packed* w, const void* x, void* y, int n, 
     }
     {   // release the device copies of the schedules that did not win
         std::lock_guard<std::mutex> lk(w->mu);
-        auto key_of = [&](const Plan& pl) { return alcs::sched_key(pl.kc, pl.n_rg, g_variants[pl.variant].v.mma); };
+        auto key_of = [&](const Plan& pl) {      // (the small-problem kernel uses no schedule: a key that matches none)
+            return pl.gather ? std::make_pair(0, 0) : alcs::sched_key(pl.kc, pl.n_rg, g_variants[pl.variant].v.mma);
+        };
         for (auto& kv : w->sched)
             if (kv.second.uploaded && kv.first != key_of(all[best_i])) {
                 bool used = false;
@@ -845,7 +946,9 @@ ALCS_API int alcs_stack_create(const alcs_layer* layers, int n_layers, unsigned 
         int rc = check_conv_args(L.w, L.x, L.y, L.n, L.h, L.wd, L.flags, &it.q);
         if (!rc) rc = check_device(L.w);
         if (!rc && it.q > 0) rc = resolve_plan(L.w, L.n, L.h, L.wd, L.flags, it.q, nullptr, &it.plan);
-        if (!rc && it.q > 0) {   // the schedule must be resident before any launch is captured
+        if (!rc && it.q > 0 && it.plan.gather) {
+            rc = ensure_canonical_on_device(L.w, nullptr);
+        } else if (!rc && it.q > 0) {   // the schedule must be resident before any launch is captured
             Schedule* sc = get_schedule(L.w, it.plan.kc, it.plan.n_rg, true, g_variants[it.plan.variant].v.mma);
             rc = sc ? upload_schedule(L.w, sc, nullptr) : ALCS_ERR_ALLOC;
             const int elt = (int)L.w->elt();
@@ -963,6 +1066,10 @@ extern "C" ALCS_API int alcs_spconv1x1_noalloc(const alcs_packed* w, const void*
         auto it = w->plan_cache.find(alcs::ShapeKey{n, h, wd, flags});
         if (it == w->plan_cache.end()) return ALCS_ERR_STATE;
         plan = it->second;
+        if (plan.gather) {      // the small-problem kernel: needs only its resident copy of the storage format
+            if (!w->d_row_ptr) return ALCS_ERR_STATE;
+            return launch_gather_plan(w, plan, x, y, n, h, wd, bias, flags, st);
+        }
         auto si = w->sched.find(alcs::sched_key(plan.kc, plan.n_rg, g_variants[plan.variant].v.mma));
         if (si == w->sched.end() || !si->second.uploaded) return ALCS_ERR_STATE;
         sc = &si->second;

@@ -1,0 +1,30 @@
+// Launcher of the small-problem (direct gather) kernel of the sparse pointwise convolution.
+// Internal to libalcs.
+#ifndef ALCS_GATHER_H_
+#define ALCS_GATHER_H_
+
+#include <cuda_runtime.h>
+
+namespace alcs {
+
+struct GatherArgs {
+    const float* x;           // [n][cin][hw]
+    float* y;                 // [n][cout][hw]
+    const float* bias;        // [cout] or nullptr
+    const int* row_ptr;       // the canonical storage format, on the device
+    const int* col_idx;
+    const float* vals;
+    int rows, cin, cout, hw, n;
+    int tiles;                // pixel tiles of 32 * P per image
+    int relu;
+    int vec;                  // 1: rows of x are 16-byte aligned multiples of 4 pixels
+};
+
+// g in {1,2,4,8,16}, p = pixels per lane in {2,4,8}, ks = warps per thread block (1..16) that share one
+// block row's columns.
+bool gather_config_ok(int g, int p, int ks, bool vec);
+cudaError_t launch_gather(int g, int p, int ks, const GatherArgs& a, cudaStream_t st);
+
+}  // namespace alcs
+
+#endif  // ALCS_GATHER_H_

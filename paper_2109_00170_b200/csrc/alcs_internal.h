@@ -69,6 +69,9 @@ struct Plan {
     int occ = 1;           // resident thread blocks per SM
     size_t smem = 0;
     double cost = 0;       // model estimate, seconds
+    // the small-problem kernel (no staging, reads the canonical format): variant is -1, and
+    int gather = 0;        // 1 selects it,
+    int gp = 0, gks = 0;   // pixels per lane and warps per thread block (shares of one block row's columns)
 };
 
 // Key of the plan cache: the problem shape plus the requested configuration (all zero = automatic).
@@ -97,6 +100,10 @@ struct alcs_packed {
     int device = -1;
     int* d_err = nullptr;             // device error word written by a kernel whose bounded wait ran out
     mutable void* d_xpad = nullptr;   // scratch: X repacked to 16-byte aligned rows (grown on demand)
+    // device copy of row_ptr / col_idx / vals for the small-problem kernel (made on first use)
+    mutable int32_t* d_row_ptr = nullptr;
+    mutable int32_t* d_col_idx = nullptr;
+    mutable void* d_vals = nullptr;
     mutable size_t xpad_bytes = 0;
     // by (kc, n_rg), built on demand; the tensor-core flavour of a schedule is stored under -kc
     mutable std::map<std::pair<int, int>, alcs::Schedule> sched;

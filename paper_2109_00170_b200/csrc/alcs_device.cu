@@ -314,7 +314,7 @@ int enumerate_plans(const alcs_packed* w, long long q, int hw, std::vector<Plan>
             }
         }
     }
-    if (hw > 0 && q / hw <= 64) {       // small batches only: one thread block per (block row, image, pixel tile)
+    if (hw > 0 && q / hw <= 8) {        // small batches only: one thread block per (block row, image, pixel tile)
         for (int p = 8; p >= 2; p /= 2)
             for (int ks = 4; ks <= 16; ks *= 2) {
                 Plan g;

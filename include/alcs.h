@@ -264,8 +264,11 @@ ALCS_API int alcs_spconv1x1_host(const alcs_packed* w, const void* x_host, void*
  *     part of the library image (every GPU that loads the library holds it until the process exits).
  *     A problem that needs more, n*cin*round_up(h*wd to 16 bytes)*element size, is rejected with
  *     ALCS_ERR_TOO_LARGE; inputs with 16-byte-multiple rows need no scratch and have no size limit.
- * The first call on each device looks up the address of that array (with that device current); make
- * that first call before any stream capture begins.  All calls share the one array and it keeps
+ * The address of that array is looked up per device at set-up time, by alcs_packed_upload (which
+ * runs with that device current); loading the library's device code on a GPU -- which is when the
+ * driver backs the array there -- therefore also happens during set-up, not inside the phase that
+ * may not allocate.  Should that look-up have failed, the first alcs_spconv1x1_noalloc call on the
+ * device repeats it; make that first call before any stream capture begins.  All calls share the one array and it keeps
  * what the previous call left there: every call rewrites the part it uses, padding included, but two
  * calls that overlap on the GPU (different streams) race on it -- keep them on one stream or order
  * them with events.  Arguments, results and error codes are otherwise those of alcs_spconv1x1.
@@ -400,6 +403,11 @@ typedef struct {
  * the stack) and fixes each layer's launch configuration.  With ALCS_STACK_GRAPH the first
  * alcs_stack_run captures the launches into a CUDA graph on that stream and later runs replay it.
  * alcs_stack_run enqueues all layers in order on cuda_stream without synchronising.
+ * Layers whose input rows are not a multiple of 16 bytes long are repacked into scratch memory that
+ * the STACK owns (allocated by alcs_stack_create with the layers' device current, sized for its
+ * largest such layer, released by alcs_stack_destroy): nothing a captured graph refers to is freed
+ * or moved by later alcs_spconv1x1 calls with the same packed matrices, at any batch size.  Two runs
+ * of the same stack must not overlap on the GPU (they share that scratch and the outputs).
  */
 ALCS_API int alcs_stack_create(const alcs_layer* layers, int n_layers, unsigned stack_flags,
                       alcs_stack** out);

@@ -20,12 +20,12 @@ namespace {
 struct Conv2dVariant {
     int g, p, st, ni;
     const void* fn[2];      // [0] all channels in one chunk, [1] chunked
-    bool ready[2];
+    bool ready[2][64];      // by device: the shared-memory attribute is set per device
 };
 
 #define ALCS_C2D_N(G, P, ST, NI)                                                            \
     {G, P, ST, NI, {(const void*)&spconv2d_kernel<G, P, ST, kConv2dWarps, false, NI>,       \
-                    (const void*)&spconv2d_kernel<G, P, ST, kConv2dWarps, true, NI>}, {false, false}}
+                    (const void*)&spconv2d_kernel<G, P, ST, kConv2dWarps, true, NI>}, {}}
 #define ALCS_C2D(G, P, ST) ALCS_C2D_N(G, P, ST, 1)
 #define ALCS_C2D_G(G)                                                                                      \
     ALCS_C2D(G, 2, 1), ALCS_C2D(G, 4, 1), ALCS_C2D(G, 8, 1), ALCS_C2D(G, 2, 2), ALCS_C2D(G, 4, 2), ALCS_C2D(G, 8, 2), \
@@ -55,11 +55,15 @@ cudaError_t launch_conv2d(int g, int p, int stride, int ni, const Conv2dArgs& a,
     if (!v) return cudaErrorInvalidValue;
     const int ch = a.nch > 1 ? 1 : 0;
     {
+        int dev = -1;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
         std::lock_guard<std::mutex> lk(g_c2d_mu);
-        if (!v->ready[ch]) {
-            cudaError_t e = cudaFuncSetAttribute(v->fn[ch], cudaFuncAttributeMaxDynamicSharedMemorySize, kConv2dMaxDynSmem);
+        if (!v->ready[ch][dev]) {
+            e = cudaFuncSetAttribute(v->fn[ch], cudaFuncAttributeMaxDynamicSharedMemorySize, kConv2dMaxDynSmem);
             if (e != cudaSuccess) return e;
-            v->ready[ch] = true;
+            v->ready[ch][dev] = true;
         }
     }
     Conv2dArgs args = a;

@@ -38,12 +38,14 @@ constexpr int kMaxSmem = 227 * 1024;
 struct VariantInfo {
     KernelVariant v;
     int regs = 0;
-    bool ready = false;
+    bool ready[64] = {};    // per device: the dynamic shared-memory attribute is a per-device setting
 };
 
 struct DeviceInfo {
     int sms = 0;
     int smem_optin = 0;
+    double sm_hz = 0;       // maximum SM clock
+    double hbm_bps = 0;     // nominal DRAM bandwidth (bus width x memory clock x 2), bytes per second
     bool ok = false;
 };
 
@@ -72,22 +74,33 @@ int device_info(int dev, DeviceInfo* out)
     if (!g_dev[dev].ok) {
         ALCS_CUDA(cudaDeviceGetAttribute(&g_dev[dev].sms, cudaDevAttrMultiProcessorCount, dev));
         ALCS_CUDA(cudaDeviceGetAttribute(&g_dev[dev].smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+        int khz = 0, mem_khz = 0, bus_bits = 0;
+        ALCS_CUDA(cudaDeviceGetAttribute(&khz, cudaDevAttrClockRate, dev));
+        ALCS_CUDA(cudaDeviceGetAttribute(&mem_khz, cudaDevAttrMemoryClockRate, dev));
+        ALCS_CUDA(cudaDeviceGetAttribute(&bus_bits, cudaDevAttrGlobalMemoryBusWidth, dev));
+        g_dev[dev].sm_hz = khz > 0 ? khz * 1e3 : 1.9e9;
+        // the cost models only rank configurations, so the nominal figure (about 80 % of which a
+        // streaming kernel reaches) is good enough
+        const double nominal = 2.0 * mem_khz * 1e3 * (bus_bits / 8.0);
+        g_dev[dev].hbm_bps = nominal > 0 ? 0.8 * nominal : 6.0e12;
         g_dev[dev].ok = true;
     }
     *out = g_dev[dev];
     return ALCS_OK;
 }
 
-// Make a variant launchable with large dynamic shared memory (once per process).
-int prepare_variant(VariantInfo& vi)
+// Make a variant launchable with large dynamic shared memory on the current device `dev` (once per
+// device: the attribute belongs to the function as loaded on that device).
+int prepare_variant(VariantInfo& vi, int dev)
 {
+    if (dev < 0 || dev >= 64) return ALCS_ERR_INVALID_ARG;
     std::lock_guard<std::mutex> lk(g_mu);
-    if (vi.ready) return ALCS_OK;
+    if (vi.ready[dev]) return ALCS_OK;
     ALCS_CUDA(cudaFuncSetAttribute(vi.v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
     cudaFuncAttributes fa;
     ALCS_CUDA(cudaFuncGetAttributes(&fa, vi.v.fn));
     vi.regs = fa.numRegs;
-    vi.ready = true;
+    vi.ready[dev] = true;
     return ALCS_OK;
 }
 
@@ -173,8 +186,9 @@ void free_schedule_device(Schedule& sc)
 // are modelled per SM: FMA issue slots, shared-memory wavefronts and bytes arriving from L2;
 // plus the HBM floor and the quantisation of work items over the persistent thread blocks.
 double model_cost(const alcs_packed* w, const KernelVariant& v, const Schedule& sc, long long q,
-                  int sms, int occ)
+                  const DeviceInfo& di, int occ)
 {
+    const int sms = di.sms;
     const int elt = (int)w->elt();
     const int T = 32 * v.p;
     const long long n_tiles = (q + T - 1) / T;
@@ -193,9 +207,9 @@ double model_cost(const alcs_packed* w, const KernelVariant& v, const Schedule& 
         const double warps = (double)v.nw * occ;
         const double hide = std::min(1.0, 0.4 + warps / 20.0);
         const double item_cycles = (std::max(std::max(issue, lsu) / hide, l2b) + 2500.0) * (v.groups == 2 && rounds > 1 ? 0.7 : 1.0);
-        const double t_sm = (double)rounds * occ * item_cycles / 1.9e9;
+        const double t_sm = (double)rounds * occ * item_cycles / di.sm_hz;
         const double bytes = (double)q * (w->cin + w->cout) * elt;
-        return std::max(t_sm, bytes / 6.0e12);
+        return std::max(t_sm, bytes / di.hbm_bps);
     }
     const int vg = (v.p * elt >= 16) ? 16 / elt : v.p;
     const int ng = v.p / vg;
@@ -208,9 +222,9 @@ double model_cost(const alcs_packed* w, const KernelVariant& v, const Schedule& 
     const double warps = (double)v.nw * occ;
     const double hide = std::min(1.0, 0.5 + warps / 30.0);
     const double item_cycles = std::max(std::max(fma_issue, lsu), l2) / hide + 1500.0;
-    const double t_sm = (double)rounds * occ * item_cycles / 1.9e9;
+    const double t_sm = (double)rounds * occ * item_cycles / di.sm_hz;
     const double bytes = (double)q * (w->cin + w->cout) * elt;
-    return std::max(t_sm, bytes / 6.0e12);
+    return std::max(t_sm, bytes / di.hbm_bps);
 }
 
 int occupancy_of(const VariantInfo& vi, size_t smem)
@@ -226,8 +240,9 @@ int occupancy_of(const VariantInfo& vi, size_t smem)
 // The small-problem kernel as a plan.  Its cost estimate is a latency model: a warp issues the loads of
 // a few blocks at a time and waits about one L2 round trip for each batch; the arithmetic term makes it
 // lose against the staged kernels as soon as there is enough work to keep the SMs busy.
-bool gather_plan(const alcs_packed* w, int n, int hw, int p, int ks, int sms, Plan* out)
+bool gather_plan(const alcs_packed* w, int n, int hw, int p, int ks, const DeviceInfo& di, Plan* out)
 {
+    const int sms = di.sms;
     if (w->dt != ALCS_F32) return false;
     if (!alcs::gather_config_ok(w->g, p, ks, false)) return false;
     const long long tiles = (hw + 32 * p - 1) / (32 * p);
@@ -241,7 +256,7 @@ bool gather_plan(const alcs_packed* w, int n, int hw, int p, int ks, int sms, Pl
     const double rounds = std::ceil((double)blocks / (sms * resident));
     const double latency = rounds * (batches * 900.0 + 2500.0);
     const double alu = (double)w->nb * w->g * n * tiles * 32.0 * p / (sms * 128.0 * 0.25);
-    pl.cost = std::max(latency, alu) / 1.9e9;
+    pl.cost = std::max(latency, alu) / di.sm_hz;
     *out = pl;
     return true;
 }
@@ -262,7 +277,7 @@ int enumerate_plans(const alcs_packed* w, long long q, int hw, std::vector<Plan>
     for (size_t vi = 0; vi < g_variants.size(); ++vi) {
         const KernelVariant& v = g_variants[vi].v;
         if (v.is_f16 != (w->dt == ALCS_F16) || v.g != w->g) continue;
-        rc = prepare_variant(g_variants[vi]);
+        rc = prepare_variant(g_variants[vi], w->device);
         if (rc) return rc;
         const int cap = v.nw / v.groups * v.rw;
         const int rg_min = (w->rows + cap - 1) / cap;
@@ -296,7 +311,7 @@ int enumerate_plans(const alcs_packed* w, long long q, int hw, std::vector<Plan>
                     Plan p;
                     p.variant = (int)vi; p.kc = sc->kc; p.n_rg = sc->n_rg; p.stages = stages;
                     p.occ = occ; p.smem = smem;
-                    p.cost = model_cost(w, v, *sc, q, di.sms, occ);
+                    p.cost = model_cost(w, v, *sc, q, di, occ);
                     // deeper rings only help while there are chunks to prefetch; prefer the shallowest
                     p.cost *= 1.0 + 0.01 * stages;
                     // Bulk copies pay a fixed cost per copy, so they win when a tile row is one long
@@ -318,7 +333,7 @@ int enumerate_plans(const alcs_packed* w, long long q, int hw, std::vector<Plan>
         for (int p = 8; p >= 2; p /= 2)
             for (int ks = 4; ks <= 16; ks *= 2) {
                 Plan g;
-                if (gather_plan(w, (int)(q / hw), hw, p, ks, di.sms, &g)) out.push_back(g);
+                if (gather_plan(w, (int)(q / hw), hw, p, ks, di, &g)) out.push_back(g);
             }
     }
     std::stable_sort(out.begin(), out.end(), [](const Plan& a, const Plan& b) { return a.cost < b.cost; });
@@ -365,7 +380,7 @@ int cfg_to_plan(const alcs_packed* w, long long q, int hw, const alcs_launch_cfg
         rc = device_info(w->device, &di);
         if (rc) return rc;
         if (hw > 0 && c->pixels_per_lane && c->warps &&
-            gather_plan(w, (int)(q / hw), hw, c->pixels_per_lane, c->warps, di.sms, out)) return ALCS_OK;
+            gather_plan(w, (int)(q / hw), hw, c->pixels_per_lane, c->warps, di, out)) return ALCS_OK;
         return ALCS_ERR_UNSUPPORTED;
     }
     auto variant_ok = [&](const Plan& p) {
@@ -520,8 +535,11 @@ int launch_gather_plan(const alcs_packed* w, const Plan& p, const void* x, void*
     return ALCS_OK;
 }
 
+// scratch / scratch_bytes: where X is repacked when its rows are not 16-byte multiples.  nullptr means
+// the scratch that w owns (allocated or grown here); a layer stack passes its own, fixed for the
+// stack's lifetime, so that a captured graph never refers to memory a later call may free.
 int launch_plan(const alcs_packed* w, const Plan& p, const void* x, void* y, int n, int h, int wd,
-                const float* bias, unsigned flags, cudaStream_t st)
+                const float* bias, unsigned flags, cudaStream_t st, void* scratch = nullptr, size_t scratch_bytes = 0)
 {
     if (p.gather) {
         const int rc = ensure_canonical_on_device(w, st);
@@ -545,16 +563,18 @@ int launch_plan(const alcs_packed* w, const Plan& p, const void* x, void* y, int
     if (((size_t)hw * elt) % 16 != 0) {
         const int hwp = padded_hw(hw, elt);
         const size_t need = (size_t)n * w->cin * hwp * elt;
-        if ((long long)n * hwp <= (1ll << 30) && ensure_xpad(w, need) == ALCS_OK) {
+        if (scratch && scratch_bytes < need) return ALCS_ERR_STATE;
+        if ((long long)n * hwp <= (1ll << 30) && (scratch || ensure_xpad(w, need) == ALCS_OK)) {
+            void* const xpad = scratch ? scratch : w->d_xpad;
             const long long rows = (long long)n * w->cin;
             const unsigned blocks = (unsigned)std::min<long long>((rows * (hwp * elt / 16) + 255) / 256, (long long)di.sms * 16);
             if (elt == 4)
-                repack_rows_kernel<float><<<blocks, 256, 0, st>>>(static_cast<const float*>(x), static_cast<float*>(w->d_xpad), rows, hw, hwp);
+                repack_rows_kernel<float><<<blocks, 256, 0, st>>>(static_cast<const float*>(x), static_cast<float*>(xpad), rows, hw, hwp);
             else
                 repack_rows_kernel<unsigned short><<<blocks, 256, 0, st>>>(static_cast<const unsigned short*>(x),
-                                                                          static_cast<unsigned short*>(w->d_xpad), rows, hw, hwp);
+                                                                          static_cast<unsigned short*>(xpad), rows, hw, hwp);
             ALCS_CUDA(cudaGetLastError());
-            xk = w->d_xpad;
+            xk = xpad;
             hwx = hwp;
         }   // else: fall back to element-wise staging of the unpadded rows
     }
@@ -660,6 +680,10 @@ int require_current_device(const alcs_packed* w) { return check_device(w); }
 
 }  // namespace alcs
 
+namespace {
+int noalloc_scratch_address(int dev, void** out);      // defined with alcs_spconv1x1_noalloc below
+}
+
 struct alcs_stack {
     struct Item {
         alcs_layer layer;
@@ -669,6 +693,10 @@ struct alcs_stack {
     std::vector<Item> items;
     unsigned flags = 0;
     cudaGraphExec_t exec = nullptr;
+    // repack scratch of the stack's own (the layers run one after the other, so they share it):
+    // allocated by alcs_stack_create, freed by alcs_stack_destroy, never moved in between
+    void* xpad = nullptr;
+    size_t xpad_bytes = 0;
 };
 
 extern "C" {
@@ -696,6 +724,12 @@ ALCS_API int alcs_packed_upload(alcs_packed* p, int device, void* cuda_stream)
         return e == cudaErrorMemoryAllocation ? ALCS_ERR_ALLOC : ALCS_ERR_CUDA;
     }
     p->device = device;
+    // Resolve the fixed scratch array of alcs_spconv1x1_noalloc now, at set-up time and with this
+    // device current: the module that holds it is then loaded and the array backed on this device
+    // before any phase in which the caller may no longer allocate.  (A failure here only matters to
+    // that entry point, which looks the address up again and reports it.)
+    void* scratch = nullptr;
+    (void)noalloc_scratch_address(device, &scratch);
     cudaSetDevice(prev);
     return ALCS_OK;
 }
@@ -939,6 +973,7 @@ ALCS_API int alcs_stack_create(const alcs_layer* layers, int n_layers, unsigned 
     alcs_stack* s = new (std::nothrow) alcs_stack();
     if (!s) return ALCS_ERR_ALLOC;
     s->flags = stack_flags;
+    size_t scratch_need = 0;
     for (int i = 0; i < n_layers; ++i) {
         const alcs_layer& L = layers[i];
         alcs_stack::Item it;
@@ -954,10 +989,18 @@ ALCS_API int alcs_stack_create(const alcs_layer* layers, int n_layers, unsigned 
             const int elt = (int)L.w->elt();
             const long long hw = (long long)L.h * L.wd;
             if (!rc && (hw * elt) % 16 != 0 && (long long)L.n * padded_hw((int)hw, elt) <= (1ll << 30))
-                rc = ensure_xpad(L.w, (size_t)L.n * L.w->cin * padded_hw((int)hw, elt) * elt);
+                scratch_need = std::max(scratch_need, (size_t)L.n * L.w->cin * padded_hw((int)hw, elt) * elt);
         }
         if (rc) { delete s; return rc; }
         s->items.push_back(it);
+    }
+    if (scratch_need) {
+        if (cudaMalloc(&s->xpad, scratch_need) != cudaSuccess) {
+            (void)cudaGetLastError();
+            delete s;
+            return ALCS_ERR_ALLOC;
+        }
+        s->xpad_bytes = scratch_need;
     }
     *out = s;
     return ALCS_OK;
@@ -968,7 +1011,7 @@ static int stack_enqueue(alcs_stack* s, cudaStream_t st)
     for (auto& it : s->items) {
         if (it.q == 0) continue;
         const alcs_layer& L = it.layer;
-        int rc = launch_plan(L.w, it.plan, L.x, L.y, L.n, L.h, L.wd, L.bias, L.flags, st);
+        int rc = launch_plan(L.w, it.plan, L.x, L.y, L.n, L.h, L.wd, L.bias, L.flags, st, s->xpad, s->xpad_bytes);
         if (rc) return rc;
     }
     return ALCS_OK;
@@ -1009,6 +1052,7 @@ ALCS_API int alcs_stack_destroy(alcs_stack* s)
 {
     if (!s) return ALCS_OK;
     if (s->exec) cudaGraphExecDestroy(s->exec);
+    if (s->xpad) cudaFree(s->xpad);     // waits for the device, so no replay can still be using it
     delete s;
     return ALCS_OK;
 }

@@ -274,6 +274,43 @@ def test_stack_runner(alcs, graph):
     alcs.alcs_stack_destroy(st)
 
 
+def test_graph_stack_survives_a_larger_call_on_the_same_weights(alcs):
+    """A captured stack whose layer needs repacked input rows (7x7 images: 196-byte rows) keeps its
+    own repack scratch: a later plain call with the same packed matrix and a larger batch, which
+    makes the matrix grow ITS scratch, must not disturb replays of the graph."""
+    import torch
+    dev = torch.device("cuda:0")
+    W, M, X, b = _rand(71, 2, 40, 24, 49, 4, 0.5)
+    p = alcs.alcs_packed_upload(alcs.alcs_pack(W, M, 4), 0)
+    xd = torch.from_numpy(X).to(dev)
+    yd = torch.full((2, 24, 49), float("nan"), device=dev)
+    bd = torch.from_numpy(b).to(dev)
+    # a kernel that stages x (the small-problem kernel the planner may pick at batch 2 repacks nothing)
+    alcs.alcs_spconv1x1_set_cfg(p, 2, 7, 7, alcs.ALCS_RELU, dict(math_mode=1))
+    st = alcs.alcs_stack_create([dict(w=p, x=xd, y=yd, n=2, h=7, wd=7, bias=bd, flags=alcs.ALCS_RELU)],
+                                alcs.ALCS_STACK_GRAPH)
+    stream = torch.cuda.Stream()
+    Yref, A = oracle.conv1x1(W, M, X, b, True, 4, want_scale=True)
+    alcs.alcs_stack_run(st, stream)
+    stream.synchronize()
+    assert_parity(yd.cpu().numpy(), Yref, A, "f32")
+    # the same weights at a larger batch, twice (grow, then reuse), on another stream
+    Xb = np.concatenate([X] * 8, axis=0)
+    Wb, Mb = W, M
+    big = run_gpu(alcs, Wb, Mb, Xb, b, True, 4, h=7, wd=7, packed=p)
+    Yb, Ab = oracle.conv1x1(W, M, Xb, b, True, 4, want_scale=True)
+    assert_parity(big, Yb, Ab, "f32")
+    junk = torch.full((64 << 20,), 3.0, device=dev)     # reuse whatever memory was just released
+    for _ in range(2):
+        yd.fill_(float("nan"))
+        torch.cuda.synchronize()
+        alcs.alcs_stack_run(st, stream)
+        stream.synchronize()
+        assert_parity(yd.cpu().numpy(), Yref, A, "f32")
+    del junk
+    alcs.alcs_stack_destroy(st)
+
+
 def test_device_error_paths(alcs):
     import torch
     W, M, X, b = _rand(24, 1, 8, 8, 16, 4, 0.5)

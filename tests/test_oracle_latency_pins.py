@@ -59,6 +59,33 @@ def test_group_keys_small_integers_exact():
     assert np.array_equal(L.group_keys(U, 2), np.array([[10, 4], [4, 20], [25, 1]], dtype=np.float32))
 
 
+def test_group_keys_rank_like_the_true_norm():
+    """Algorithm 1 ranks groups by L2 norm; the oracle ranks by the squared norm accumulated in fp32.
+    On real-valued data the two rankings must agree for every pair of groups except pairs whose
+    true (float64) squared norms are closer than the rounding of the fp32 key: g products and g sums,
+    each within 2^-24 relative, i.e. |key - norm^2| <= 2 g 2^-24 norm^2."""
+    g = 4
+    U = rng.normal(77, 3, 64 * 96).reshape(64, 96).astype(np.float32)
+    keys = L.group_keys(U, g).astype(np.float64).reshape(-1)
+    U64 = U.astype(np.float64)
+    true_sq = (U64.reshape(64 // g, g, 96) ** 2).sum(axis=1).reshape(-1)      # exact to 2^-53
+    bound = 2 * g * 2.0 ** -24 * true_sq
+    assert (np.abs(keys - true_sq) <= bound).all()
+    # the square root is monotone: ranking by the norm is ranking by its square
+    assert np.array_equal(np.argsort(np.sqrt(true_sq), kind="stable"), np.argsort(true_sq, kind="stable"))
+    by_key = np.argsort(-keys, kind="stable")
+    rank_key = np.empty_like(by_key)
+    rank_key[by_key] = np.arange(by_key.size)
+    i, j = np.triu_indices(keys.size, 1)
+    disagree = (true_sq[i] > true_sq[j]) != (rank_key[i] < rank_key[j])
+    near = np.abs(true_sq[i] - true_sq[j]) <= bound[i] + bound[j]
+    assert not (disagree & ~near).any()
+    assert disagree.sum() <= near.sum()
+    # a key computed from the wrong filters (a shifted group) would not pass
+    wrong = L.group_keys(np.roll(U, 1, axis=0), g).astype(np.float64).reshape(-1)
+    assert (np.abs(wrong - true_sq) > bound).any()
+
+
 def _layers(seed, shapes):
     return [rng.normal(seed, 20 + i, co * k).reshape(co, k).astype(np.float32) for i, (co, k) in enumerate(shapes)]
 

@@ -107,3 +107,30 @@ def test_ragged_last_group_is_zero_padded():
     M = np.ones((2, 2), np.uint8)
     _, _, vals = opack.pack(W, M, 4)
     assert np.array_equal(vals[1], [[1, 0, 0, 0], [1, 0, 0, 0]])
+
+
+def test_flatten_on_the_paper_example():
+    """The paper's worked example (Section 3.2.2, storage-format paragraph) through flatten(): one
+    group of g = 2 filters with 3 non-zero columns gives row_ptr [0, 3]; the column indices begin
+    1, 3; the flat value array begins 1, 3, 2, 1 (the g values of a column are contiguous, columns in
+    order).  The third column is only in the missing figure: any column after 3, any values."""
+    g, count, offsets, values = _read_golden()
+    known = [o for o in offsets if o is not None]
+    W = np.zeros((2, 6), np.float32)
+    M = np.zeros((1, 6), np.uint8)
+    cols = known + [5]
+    vals = [pair for pair in values if None not in pair] + [[7.0, 9.0]]
+    for c, v in zip(cols, vals):
+        W[:, c] = v
+        M[0, c] = 1
+    row_ptr, col_idx, flat = opack.flatten(*opack.pack(W, M, g), g, np.float32)
+    assert list(row_ptr) == [0, count] == [0, 3]
+    assert list(col_idx[:2]) == [1, 3]
+    assert list(flat[:4]) == [1.0, 3.0, 2.0, 1.0]
+    assert row_ptr.dtype == np.int32 and col_idx.dtype == np.int32 and flat.dtype == np.float32
+    # two groups: the second group's entries follow the first's, offsets restart from the column index
+    W2 = np.vstack([W, 10 * W])
+    M2 = np.vstack([M, M])
+    row_ptr, col_idx, flat = opack.flatten(*opack.pack(W2, M2, g), g, np.float32)
+    assert list(row_ptr) == [0, 3, 6] and list(col_idx) == [1, 3, 5, 1, 3, 5]
+    assert list(flat[6:10]) == [10.0, 30.0, 20.0, 10.0]

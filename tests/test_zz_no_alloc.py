@@ -20,31 +20,38 @@ from gpu_util import TOL, assert_parity
 pytestmark = pytest.mark.gpu
 
 
-def _case(seed, n, cin, cout, hw, g, density):
+def _case(seed, n, cin, cout, hw, g, density, dtype=np.float32):
     rows = (cout + g - 1) // g
-    W = (rng.normal(seed, 1, cout * cin) * cin ** -0.5).reshape(cout, cin).astype(np.float32)
-    X = np.abs(rng.normal(seed, 2, n * cin * hw)).reshape(n, cin, hw).astype(np.float32)
+    W = (rng.normal(seed, 1, cout * cin) * cin ** -0.5).reshape(cout, cin).astype(dtype)
+    X = np.abs(rng.normal(seed, 2, n * cin * hw)).reshape(n, cin, hw).astype(dtype)
     M = (rng.uniform01(seed, 3, rows * cin) < density).astype(np.uint8).reshape(rows, cin)
     b = (0.1 * rng.normal(seed, 4, cout)).astype(np.float32)
     return W, M, X, b
 
 
-@pytest.mark.parametrize("h,wd", [(7, 7), (14, 14)])
-def test_noalloc_matches_the_allocating_entry_point_twice_in_a_row(alcs, h, wd):
+@pytest.mark.parametrize("h,wd,dtype,g", [(7, 7, np.float32, 4), (14, 14, np.float32, 4), (7, 7, np.float16, 8)])
+def test_noalloc_matches_the_allocating_entry_point_twice_in_a_row(alcs, h, wd, dtype, g):
     import torch
     dev = torch.device("cuda:0")
-    n, cin, cout, g = 8, 96, 64, 4
+    n, cin, cout = 8, 96, 64
     hw = h * wd
-    W, M, X1, b = _case(700 + hw, n, cin, cout, hw, g, 0.3)
-    X2 = np.abs(rng.normal(900 + hw, 2, n * cin * hw)).reshape(n, cin, hw).astype(np.float32) * 3.0
+    kind = "f32" if dtype == np.float32 else "f16"
+    W, M, X1, b = _case(700 + hw, n, cin, cout, hw, g, 0.3, dtype)
+    X2 = (np.abs(rng.normal(900 + hw, 2, n * cin * hw)).reshape(n, cin, hw) * 3.0).astype(dtype)
     p = alcs.alcs_packed_upload(alcs.alcs_pack(W, M, g), 0)
     bd = torch.from_numpy(b).to(dev)
     st = torch.cuda.current_stream()
     flags = alcs.ALCS_RELU
+    # Pin a kernel that stages x through shared memory (math_mode 1 = CUDA cores, 2 = tensor cores):
+    # at this batch size the planner may otherwise pick the small-problem kernel, which reads x in
+    # place, needs no scratch and would leave the fixed array untested.
+    alcs.alcs_spconv1x1_set_cfg(p, n, h, wd, flags, dict(math_mode=1 if dtype == np.float32 else 2))
+    assert alcs.alcs_spconv1x1_plan(p, n, h, wd, flags)["math_mode"] in (1, 2)
+    ydt = torch.float32 if dtype == np.float32 else torch.float16
     for X in (X1, X2):
         xd = torch.from_numpy(X).to(dev)
-        y_ref = torch.full((n, cout, hw), float("nan"), device=dev)
-        y_new = torch.full((n, cout, hw), float("nan"), device=dev)
+        y_ref = torch.full((n, cout, hw), float("nan"), device=dev, dtype=ydt)
+        y_new = torch.full((n, cout, hw), float("nan"), device=dev, dtype=ydt)
         # the ordinary entry point: also what makes the launch schedule resident for this shape
         alcs.alcs_spconv1x1(p, xd, y_ref, n, h, wd, bd, flags, st)
         alcs.alcs_spconv1x1_noalloc(p, xd, y_new, n, h, wd, bd, flags, st)
@@ -52,8 +59,8 @@ def test_noalloc_matches_the_allocating_entry_point_twice_in_a_row(alcs, h, wd):
         Yref, A = oracle.conv1x1(W, M, X, b, True, g, want_scale=True)
         a, r = y_new.cpu().numpy(), y_ref.cpu().numpy()
         assert np.isfinite(a).all()
-        assert (np.abs(a.astype(np.float64) - r.astype(np.float64)) <= TOL["f32"] * A).all()
-        assert_parity(a, Yref, A, "f32")
+        assert (np.abs(a.astype(np.float64) - r.astype(np.float64)) <= TOL[kind] * A).all()
+        assert_parity(a, Yref, A, kind)
     assert alcs.alcs_packed_status(p) == 0
 
 

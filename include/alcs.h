@@ -181,6 +181,21 @@ typedef struct {
 } alcs_launch_cfg;
 
 /*
+ * alcs_schedule_selfcheck (host only, no CUDA): build the launch schedule of p for a CUDA-core kernel
+ * with `warps` consumer warps of `slots` accumulator sets each (chunk_channels and row_groups as in
+ * alcs_launch_cfg; row_groups is raised to what warps*slots block rows per work item require), walk
+ * every (warp, set)'s segments chunk by chunk exactly as a consumer warp of the kernel does, and
+ * compare what that walk multiplies with the canonical storage format (paper, Section 3.2.2): every
+ * kept block exactly once, bit for bit, no other column touched, every block row bound to exactly
+ * one (warp, set).  stats (may be NULL, else 7 entries) receives {row groups; largest and smallest
+ * number of block slots (kept blocks plus padding) any of the SM's four schedulers is given in a work
+ * item; pair records in total; kept blocks; largest and smallest number of block rows a scheduler is
+ * given in a work item}.  Returns ALCS_ERR_CORRUPT if the walk and the storage format disagree.
+ */
+ALCS_API int alcs_schedule_selfcheck(const alcs_packed* p, int chunk_channels, int row_groups, int warps, int slots,
+                                     int64_t* stats);
+
+/*
  * Introspection of the compiled kernel variants (host only): alcs_variant_count() entries, each a
  * (dtype, g, pixels_per_lane, rows_per_warp, warps, min_blocks, producer_warps) combination that
  * alcs_spconv1x1_cfg accepts; the other fields of *cfg are set to 0.

@@ -24,7 +24,8 @@ ALCS_STACK_GRAPH = 1
 # every symbol include/alcs.h declares
 EXPORTS = ["alcs_strerror", "alcs_last_cuda_error", "alcs_version", "alcs_pack", "alcs_unpack",
            "alcs_packed_view", "alcs_packed_serialize", "alcs_packed_deserialize",
-           "alcs_packed_upload", "alcs_packed_status", "alcs_packed_free", "alcs_variant_count", "alcs_variant_get",
+           "alcs_packed_upload", "alcs_packed_status", "alcs_packed_free", "alcs_schedule_selfcheck",
+           "alcs_variant_count", "alcs_variant_get",
            "alcs_spconv1x1", "alcs_spconv1x1_cfg",
            "alcs_spconv1x1_plan", "alcs_spconv1x1_tune", "alcs_spconv1x1_set_cfg", "alcs_spconv1x1_host_workspace",
            "alcs_spconv1x1_host", "alcs_spconv1x1_noalloc", "alcs_spconv2d", "alcs_spconv2d_cfg", "alcs_spconv2d_plan", "alcs_layer_latency", "alcs_network_latency",
@@ -96,6 +97,7 @@ def lib():
     L.alcs_packed_status.argtypes = [vp, ip]
     L.alcs_packed_free.argtypes = [vp]
     L.alcs_packed_free.restype = None
+    L.alcs_schedule_selfcheck.argtypes = [vp, i, i, i, i, C.POINTER(C.c_int64)]
     L.alcs_variant_count.restype = i
     L.alcs_variant_get.argtypes = [i, ip, ip, C.POINTER(LaunchCfg)]
     L.alcs_spconv1x1.argtypes = [vp, vp, vp, i, i, i, vp, u, vp]
@@ -258,6 +260,13 @@ def alcs_packed_status(p: Packed) -> int:
 
 def alcs_packed_free(p: Packed):
     p.free()
+
+
+def alcs_schedule_selfcheck(p: Packed, chunk_channels: int, row_groups: int, warps: int, slots: int) -> dict:
+    """Host-only check of the balanced launch schedule against the storage format."""
+    st = (C.c_int64 * 7)()
+    _check(lib().alcs_schedule_selfcheck(p.handle, chunk_channels, row_groups, warps, slots, st), "alcs_schedule_selfcheck")
+    return dict(row_groups=st[0], max_sched=st[1], min_sched=st[2], pairs=st[3], nb=st[4], max_rows=st[5], min_rows=st[6])
 
 
 def alcs_variant_count() -> int:

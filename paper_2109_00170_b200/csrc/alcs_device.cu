@@ -67,6 +67,13 @@ void init_variants_locked()
     for (int i = 0; i < n; ++i) g_variants.push_back({t[i]});
 }
 
+// Which flavour of the launch schedule a variant takes (alcs_internal.h): the CUDA-core kernels take
+// pair records balanced for their number of consumer warps and accumulator sets.
+int flavour_of(const KernelVariant& v) { return v.mma ? 1 : alcs::balanced_flavour(v.nw, v.rw); }
+
+// math_mode of alcs_launch_cfg for a variant
+int mode_of(const KernelVariant& v) { return v.mma ? 2 : 1; }
+
 int device_info(int dev, DeviceInfo* out)
 {
     if (dev < 0 || dev >= 64) return ALCS_ERR_INVALID_ARG;
@@ -129,14 +136,20 @@ size_t plan_smem(const StageLayout& L, int stages)
 }
 
 // The schedule for (kc, n_rg): sizes only (with_records = false) or complete.  Cached in w.
-Schedule* get_schedule(const alcs_packed* w, int kc, int n_rg, bool with_records, int mma)
+Schedule* get_schedule(const alcs_packed* w, int kc, int n_rg, bool with_records, int flavour)
 {
     if (kc <= 0 || kc > w->cin) kc = w->cin;
+    if (flavour >= 2) {     // the balanced builder raises n_rg to what the (warps x sets) capacity needs: key by the result
+        const int cap = alcs::flavour_nwg(flavour) * alcs::flavour_rw(flavour);
+        n_rg = std::max(std::max(1, (w->rows + cap - 1) / cap), std::min(n_rg, w->rows));
+    }
     std::lock_guard<std::mutex> lk(w->mu);
-    Schedule& sc = w->sched[alcs::sched_key(kc, n_rg, mma)];
+    Schedule& sc = w->sched[alcs::sched_key(kc, n_rg, flavour)];
     try {
         if (sc.n_rg == 0 || (with_records && !sc.uploaded && sc.h_rec.empty() && sc.n_rec > 0)) {
-            if (mma) alcs::build_schedule_mma(*w, kc, n_rg, with_records, sc);
+            if (flavour == 1) alcs::build_schedule_mma(*w, kc, n_rg, with_records, sc);
+            else if (flavour >= 2)
+                alcs::build_schedule_balanced(*w, kc, n_rg, alcs::flavour_nwg(flavour), alcs::flavour_rw(flavour), with_records, sc);
             else alcs::build_schedule(*w, kc, n_rg, with_records, sc);
         }
     } catch (const std::bad_alloc&) {
@@ -213,12 +226,13 @@ double model_cost(const alcs_packed* w, const KernelVariant& v, const Schedule& 
     }
     const int vg = (v.p * elt >= 16) ? 16 / elt : v.p;
     const int ng = v.p / vg;
-    const double pairs_item = (double)sc.n_rec * 16.0 / alcs::record_bytes(v.g) / sc.n_rg;
-    const double seg_item = (double)sc.rpg * sc.nch;
+    const int rec_b = alcs::record_bytes(v.g);
+    const double pairs_item = (double)sc.n_rec * 16.0 / rec_b / sc.n_rg;
+    const double seg_item = (double)std::min(sc.rpg, (w->rows + sc.n_rg - 1) / sc.n_rg) * sc.nch;
     const double fma_issue = pairs_item * (2.0 * v.g * v.p + 2 * ng + 6 + (elt == 2 ? v.p : 0)) / 4.0 + seg_item * 14.0 / 4.0;
     const double lsu = pairs_item * (2.0 * ng * (vg * elt * 32 / 128.0) + 1 + v.g / 2.0) +
                        (double)sc.nch * sc.kc * T * elt / 128.0;
-    const double l2 = ((double)w->cin * T * elt + pairs_item * alcs::record_bytes(v.g)) / 48.0;
+    const double l2 = ((double)w->cin * T * elt + pairs_item * rec_b) / 48.0;
     const double warps = (double)v.nw * occ;
     const double hide = std::min(1.0, 0.5 + warps / 30.0);
     const double item_cycles = std::max(std::max(fma_issue, lsu), l2) / hide + 1500.0;
@@ -288,6 +302,7 @@ int enumerate_plans(const alcs_packed* w, long long q, int hw, std::vector<Plan>
             if (kc == last_kc) continue;
             last_kc = kc;
             if ((size_t)kc * 32 * v.p * elt * 2 > (size_t)smem_max) continue;
+            if (!v.mma && kc >= alcs::kMaxBalancedKc) continue;
             int last_rpg = -1;
             // Row-group counts to consider: every count up to a few times the minimum, and, when
             // the pixel tiles alone are too few to occupy the GPU (small batches), a geometric
@@ -299,7 +314,7 @@ int enumerate_plans(const alcs_packed* w, long long q, int hw, std::vector<Plan>
                 const int rpg = (w->rows + n_rg - 1) / n_rg;
                 if (rpg == last_rpg || rpg > cap) continue;
                 last_rpg = rpg;
-                const Schedule* sc = get_schedule(w, kc, n_rg, false, v.mma);
+                const Schedule* sc = get_schedule(w, kc, n_rg, false, flavour_of(v));
                 if (!sc) return ALCS_ERR_ALLOC;
                 const StageLayout L = stage_layout(v, *sc, elt);
                 for (int stages = 2; stages <= alcs::kMaxStages; ++stages) {
@@ -359,7 +374,7 @@ void plan_to_cfg(const Plan& p, alcs_launch_cfg* c)
     c->min_blocks = v.minb;
     c->copy_mode = p.bulk ? 2 : 1;
     c->producer_warps = v.npw;
-    c->math_mode = v.mma ? 2 : 1;
+    c->math_mode = mode_of(v);
     c->consumer_groups = v.groups;
 }
 
@@ -391,7 +406,7 @@ int cfg_to_plan(const alcs_packed* w, long long q, int hw, const alcs_launch_cfg
         if (c->warps && c->warps != v.nw) return false;
         if (c->min_blocks && c->min_blocks != v.minb) return false;
         if (c->producer_warps && c->producer_warps != v.npw) return false;
-        if (c->math_mode && (c->math_mode == 2) != (v.mma == 1)) return false;
+        if (c->math_mode && c->math_mode != mode_of(v)) return false;
         if (c->consumer_groups && c->consumer_groups != v.groups) return false;
         if (c->chunk_channels && std::min(c->chunk_channels, w->cin) != p.kc) return false;
         if (c->stages && c->stages != p.stages) return false;
@@ -410,7 +425,7 @@ int cfg_to_plan(const alcs_packed* w, long long q, int hw, const alcs_launch_cfg
             const KernelVariant& v = g_variants[p0.variant].v;
             const int rpg = (w->rows + c->row_groups - 1) / c->row_groups;
             if (rpg > v.nw / v.groups * v.rw) continue;
-            const Schedule* sc = get_schedule(w, p0.kc, c->row_groups, false, v.mma);
+            const Schedule* sc = get_schedule(w, p0.kc, c->row_groups, false, flavour_of(v));
             if (!sc) return ALCS_ERR_ALLOC;
             Plan p = p0;
             p.n_rg = sc->n_rg;
@@ -546,7 +561,7 @@ int launch_plan(const alcs_packed* w, const Plan& p, const void* x, void* y, int
         return rc ? rc : launch_gather_plan(w, p, x, y, n, h, wd, bias, flags, st);
     }
     const KernelVariant& v = g_variants[p.variant].v;
-    Schedule* sc = get_schedule(w, p.kc, p.n_rg, true, v.mma);
+    Schedule* sc = get_schedule(w, p.kc, p.n_rg, true, flavour_of(v));
     if (!sc) return ALCS_ERR_ALLOC;
     if (!sc->uploaded) {
         const int rc = upload_schedule(w, sc, st);
@@ -600,6 +615,7 @@ int launch_plan(const alcs_packed* w, const Plan& p, const void* x, void* y, int
     a.ros = sc->ros;
     const int vg = (v.p * elt >= 16) ? 16 / elt : v.p;
     a.st_vec = (hwx == hw && hw % vg == 0 && (uintptr_t)y % 16 == 0) ? 1 : 0;
+    a.st_grp = hwx % vg == 0 ? 1 : 0;
     const long long items = (long long)a.n_tiles * a.n_rg;
     if (items > 0x7fffffffll) return ALCS_ERR_SHAPE;
     // persistent thread blocks: as many as can be resident, each walks items with that stride
@@ -784,7 +800,7 @@ ALCS_API int alcs_variant_get(int index, alcs_dtype* dt, int* g, alcs_launch_cfg
         cfg->min_blocks = v.minb;
         cfg->copy_mode = 0;
         cfg->producer_warps = v.npw;
-        cfg->math_mode = v.mma ? 2 : 1;
+        cfg->math_mode = mode_of(v);
         cfg->consumer_groups = v.groups;
     }
     return ALCS_OK;
@@ -843,7 +859,7 @@ ALCS_API int alcs_spconv1x1_tune(alcs_packed* w, const void* x, void* y, int n, 
     std::vector<Plan> all;
     rc = enumerate_plans(w, q, h * wd, all);
     if (rc) return rc;
-    const size_t max_try = 400;
+    const size_t max_try = 1200;
     if (all.size() > max_try) all.resize(max_try);
     // a buffer larger than L2, rewritten before every timed launch so that each candidate is
     // timed with cold caches, as it will run inside a network
@@ -863,7 +879,7 @@ ALCS_API int alcs_spconv1x1_tune(alcs_packed* w, const void* x, void* y, int n, 
     }
     int best_i = -1;
     float best_ms = 1e30f;
-    const int reps = 2;
+    const int reps = 3;
     for (size_t i = 0; i < all.size(); ++i) {
         float tmin = 1e30f;
         bool ok = true;
@@ -893,7 +909,7 @@ ALCS_API int alcs_spconv1x1_tune(alcs_packed* w, const void* x, void* y, int n, 
     {   // release the device copies of the schedules that did not win
         std::lock_guard<std::mutex> lk(w->mu);
         auto key_of = [&](const Plan& pl) {      // (the small-problem kernel uses no schedule: a key that matches none)
-            return pl.gather ? std::make_pair(0, 0) : alcs::sched_key(pl.kc, pl.n_rg, g_variants[pl.variant].v.mma);
+            return pl.gather ? std::make_pair(0, 0) : alcs::sched_key(pl.kc, pl.n_rg, flavour_of(g_variants[pl.variant].v));
         };
         for (auto& kv : w->sched)
             if (kv.second.uploaded && kv.first != key_of(all[best_i])) {
@@ -984,7 +1000,7 @@ ALCS_API int alcs_stack_create(const alcs_layer* layers, int n_layers, unsigned 
         if (!rc && it.q > 0 && it.plan.gather) {
             rc = ensure_canonical_on_device(L.w, nullptr);
         } else if (!rc && it.q > 0) {   // the schedule must be resident before any launch is captured
-            Schedule* sc = get_schedule(L.w, it.plan.kc, it.plan.n_rg, true, g_variants[it.plan.variant].v.mma);
+            Schedule* sc = get_schedule(L.w, it.plan.kc, it.plan.n_rg, true, flavour_of(g_variants[it.plan.variant].v));
             rc = sc ? upload_schedule(L.w, sc, nullptr) : ALCS_ERR_ALLOC;
             const int elt = (int)L.w->elt();
             const long long hw = (long long)L.h * L.wd;
@@ -1114,7 +1130,7 @@ extern "C" ALCS_API int alcs_spconv1x1_noalloc(const alcs_packed* w, const void*
             if (!w->d_row_ptr) return ALCS_ERR_STATE;
             return launch_gather_plan(w, plan, x, y, n, h, wd, bias, flags, st);
         }
-        auto si = w->sched.find(alcs::sched_key(plan.kc, plan.n_rg, g_variants[plan.variant].v.mma));
+        auto si = w->sched.find(alcs::sched_key(plan.kc, plan.n_rg, flavour_of(g_variants[plan.variant].v)));
         if (si == w->sched.end() || !si->second.uploaded) return ALCS_ERR_STATE;
         sc = &si->second;
     }
@@ -1170,6 +1186,7 @@ extern "C" ALCS_API int alcs_spconv1x1_noalloc(const alcs_packed* w, const void*
     a.ros = sc->ros;
     const int vg = (v.p * elt >= 16) ? 16 / elt : v.p;
     a.st_vec = (hwx == hw && hw % vg == 0 && (uintptr_t)y % 16 == 0) ? 1 : 0;
+    a.st_grp = hwx % vg == 0 ? 1 : 0;
     const long long items = (long long)a.n_tiles * a.n_rg;
     if (items > 0x7fffffffll) return ALCS_ERR_SHAPE;
     const long long grid = std::min<long long>(items, (long long)di.sms * std::max(1, plan.occ));

@@ -35,6 +35,14 @@ constexpr int kChunkings[kNumChunkings] = {16, 32, 64, 96, 128, 0};
 // copies one contiguous range per stage; rowoff[rg][k][t] = {where local row t starts inside that
 // slice, the columns of its first pair, its number of pairs}.  Offsets are in 16-byte units.
 //
+// The balanced flavour (balanced = 1) has the same records, slices and row headers but is built for
+// a kernel with nwg consumer warps of rw accumulator sets each.  Row groups hold whole multiples of 4
+// rows where possible, every row group has rpg = nwg * rw local rows (unused ones are -1 in the row
+// map), and a row group's rows are dealt to the (warp, accumulator set) pairs so that the warps with
+// equal index modulo 4 (one scheduler of the SM) get the same number of rows and nearly the same
+// number of blocks: the row of (warp w, set s) is local row s*nwg + (s odd ? nwg-1-w : w), the
+// kernel's own mapping.
+//
 // The tensor-core flavour (mma = 1, fp16 weights, g = 8 or 16) keeps the same slices and row
 // headers but stores a segment as "step records" of 16 blocks each: the 16 chunk-local columns
 // (uint16), then per 8 output channels the 16x8 weight tile in the register order of the
@@ -44,6 +52,8 @@ constexpr int kChunkings[kNumChunkings] = {16, 32, 64, 96, 128, 0};
 struct Schedule {
     int kc = 0, nch = 0, n_rg = 0, rpg = 0;
     int mma = 0;                   // 1: step records for the tensor-core kernels
+    int balanced = 0;              // 1: the balanced flavour (below); then rpg = nwg * rw local rows per row group
+    int nwg = 0, rw = 0;           // balanced flavour: consumer warps and accumulator sets per warp it was built for
     int ros = 0;                   // ints per (row group, chunk) row of rowoff: 4 per local row
     int wcap = 0;                  // longest slice, in 16-byte units
     int n_rec = 0;                 // total length of all slices, in 16-byte units
@@ -123,7 +133,21 @@ namespace alcs {
 float half_bits_to_float(uint16_t h);
 void build_schedule(const alcs_packed& p, int kc, int n_rg, bool with_records, Schedule& out);
 void build_schedule_mma(const alcs_packed& p, int kc, int n_rg, bool with_records, Schedule& out);
-inline std::pair<int, int> sched_key(int kc, int n_rg, int mma) { return std::make_pair(mma ? -kc : kc, n_rg); }
+int pair_record_bytes(int g);                 // bytes of one pair record
+int local_row_of(int w, int s, int nw);       // local row of (consumer warp w, accumulator set s), nw consumer warps
+void build_schedule_balanced(const alcs_packed& p, int kc, int n_rg, int nwg, int rw, bool with_records, Schedule& out);
+// Which flavour of the schedule a kernel takes: 0 = pair records, rows dealt without regard to the
+// kernel's shape (the general convolution), 1 = step records of the tensor-core kernels, otherwise
+// pair records balanced for (nwg, rw).
+constexpr int kMaxBalancedKc = 1 << 19;
+inline int balanced_flavour(int nwg, int rw) { return 2 + nwg * 16 + rw; }
+inline int flavour_nwg(int flavour) { return (flavour - 2) / 16; }
+inline int flavour_rw(int flavour) { return (flavour - 2) % 16; }
+inline std::pair<int, int> sched_key(int kc, int n_rg, int flavour)
+{
+    if (flavour == 1) return std::make_pair(-kc, n_rg);
+    return std::make_pair(flavour >= 2 ? kc + flavour * kMaxBalancedKc : kc, n_rg);
+}
 // Device-side helpers implemented in alcs_device.cu, for the library's other translation units.
 int device_limits(int device, int* sms, int* smem_optin);                 // SM count, opt-in shared memory per block
 int schedule_upload(const alcs_packed* w, Schedule* sc, void* cuda_stream); // copy a schedule to w's device (once)

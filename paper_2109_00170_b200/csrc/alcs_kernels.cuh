@@ -65,8 +65,9 @@ struct ConvArgs {
     int y_f32;                // only meaningful for XT = __half
     int ld_bytes;             // bytes per X staging copy: 16, 8, 4 or 2
     int bulk;                 // 1: the producer uses bulk (TMA) copies; needs ld_bytes == 16
-    int ros;                  // ints of rowoff per (row group, chunk) = 4 * rpg
+    int ros;                  // ints of rowoff per (row group, chunk): 4 per header
     int st_vec;               // 1 if vector stores are allowed
+    int st_grp;               // 1 if the pixels of one vector store of a lane always lie in one image
     // shared-memory layout (bytes): [mbarriers | stage 0 | stage 1 | ...]
     int off_rec, off_rowoff, stage_bytes;
 };
@@ -433,7 +434,7 @@ __device__ __forceinline__ void produce(const ConvArgs& a, unsigned char* smem, 
             const unsigned char* rsrc = a.rec + (size_t)r0 * 16;
             for (int i = lane + 32 * pw; i < n16; i += 32 * npw) cp_async_16(st + a.off_rec + i * 16, rsrc + (size_t)i * 16);
             const int* osrc = rowoff + (size_t)k * a.ros;
-            for (int i = lane + 32 * pw; i < a.rpg; i += 32 * npw) cp_async_16(st + a.off_rowoff + i * 16, osrc + 4 * i);
+            for (int i = lane + 32 * pw; i < a.ros / 4; i += 32 * npw) cp_async_16(st + a.off_rowoff + i * 16, osrc + 4 * i);
             // X (or its repacked copy) is the predecessor kernel's output: wait for it once, after the
             // first weight copies are already in flight
             if (!dep_ok) { grid_dep_wait(); dep_ok = true; }
@@ -682,6 +683,15 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_kernel(const 
                         }
                         if (a.st_vec) {
                             if (yok[gi]) store_vec<YT, VG>(ybase + yoff[gi] + (size_t)co * a.hwy, v);
+                        } else if (a.st_grp) {
+                            // the lane's VG pixels lie in one image (the row length of X, padded or not,
+                            // is a multiple of VG); pixels p >= hwy exist only as padding of the repacked X
+                            if (yok[gi]) {
+                                YT* yq = ybase + yoff[gi] + (size_t)co * a.hwy;
+#pragma unroll
+                                for (int t = 0; t < VG; ++t)
+                                    if (yp[gi] + t < a.hwy) store_one<YT>(yq + t, v[t]);
+                            }
                         } else {
                             // element by element: the run may cross into the next image, and pixels
                             // p >= hwy exist only as padding of the repacked X

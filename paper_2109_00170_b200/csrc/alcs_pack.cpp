@@ -2,6 +2,7 @@
 // its inverse, the serialised blob, and the launch schedules derived from a packed matrix.
 // No CUDA in this file.
 #include <algorithm>
+#include <climits>
 #include <cstring>
 #include <limits>
 #include <new>
@@ -54,30 +55,16 @@ float half_bits_to_float(uint16_t h)
 }
 
 static int rec_bytes(int g) { return g == 1 ? 16 : 16 + 8 * g; }
+int pair_record_bytes(int g) { return rec_bytes(g); }
 
-void build_schedule(const alcs_packed& p, int kc, int n_rg, bool with_records, Schedule& out)
+// Pair records, slices and row headers for the row map already in `out` (n_rg groups of rpg local rows).
+static void emit_pair_records(const alcs_packed& p, int kc, bool with_records, Schedule& out)
 {
-    if (kc <= 0 || kc > p.cin) kc = p.cin;
     const int R = p.rows, g = p.g;
-    n_rg = std::max(1, std::min(n_rg, R));
+    const int n_rg = out.n_rg, rpg = out.rpg;
     const int nch = (p.cin + kc - 1) / kc;
-    const int rpg = (R + n_rg - 1) / n_rg;
     const int REC = rec_bytes(g);
-    out.kc = kc; out.nch = nch; out.n_rg = n_rg; out.rpg = rpg;
-
-    // rows by descending kept-block count, dealt to the row groups in serpentine order
-    std::vector<int> order(R);
-    std::iota(order.begin(), order.end(), 0);
-    std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
-        return p.row_ptr[a + 1] - p.row_ptr[a] > p.row_ptr[b + 1] - p.row_ptr[b];
-    });
-    out.h_rowmap.assign((size_t)n_rg * rpg, -1);
-    for (int i = 0; i < R; ++i) {
-        const int t = i / n_rg, j = i % n_rg;
-        const int rg = (t & 1) ? n_rg - 1 - j : j;
-        out.h_rowmap[(size_t)rg * rpg + t] = order[i];
-    }
-
+    out.kc = kc; out.nch = nch;
     out.h_slice.assign((size_t)n_rg * nch + 1, 0);
     const int ros = rpg * 4;                     // one int4 {offset, first two columns, pair count} per local row
     out.ros = ros;
@@ -154,6 +141,114 @@ void build_schedule(const alcs_packed& p, int kc, int n_rg, bool with_records, S
     out.h_slice[(size_t)n_rg * nch] = rec_count;
     out.n_rec = rec_count;
     out.wcap = wcap;
+    (void)R;
+}
+
+
+void build_schedule(const alcs_packed& p, int kc, int n_rg, bool with_records, Schedule& out)
+{
+    if (kc <= 0 || kc > p.cin) kc = p.cin;
+    const int R = p.rows;
+    n_rg = std::max(1, std::min(n_rg, R));
+    const int rpg = (R + n_rg - 1) / n_rg;
+    out.n_rg = n_rg; out.rpg = rpg;
+
+    // rows by descending kept-block count, dealt to the row groups in serpentine order
+    std::vector<int> order(R);
+    std::iota(order.begin(), order.end(), 0);
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+        return p.row_ptr[a + 1] - p.row_ptr[a] > p.row_ptr[b + 1] - p.row_ptr[b];
+    });
+    out.h_rowmap.assign((size_t)n_rg * rpg, -1);
+    for (int i = 0; i < R; ++i) {
+        const int t = i / n_rg, j = i % n_rg;
+        const int rg = (t & 1) ? n_rg - 1 - j : j;
+        out.h_rowmap[(size_t)rg * rpg + t] = order[i];
+    }
+
+    emit_pair_records(p, kc, with_records, out);
+}
+
+// Local row of (consumer warp w, accumulator set s) in a kernel with nw consumer warps: the kernel's
+// own mapping (tier s, warps in serpentine order).
+int local_row_of(int w, int s, int nw) { return s * nw + ((s & 1) ? nw - 1 - w : w); }
+
+// Balanced flavour of the pair-record schedule: see the comment on Schedule.
+void build_schedule_balanced(const alcs_packed& p, int kc, int n_rg, int nw, int rw, bool with_records, Schedule& out)
+{
+    if (kc <= 0 || kc > p.cin) kc = p.cin;
+    const int R = p.rows;
+    const int cap = nw * rw;                             // block rows one work item can hold
+    n_rg = std::max(std::max(1, (R + cap - 1) / cap), std::min(n_rg, R));
+    out.n_rg = n_rg; out.rpg = cap; out.mma = 0; out.balanced = 1;
+    out.nwg = nw; out.rw = rw;
+
+    // Sizes of the row groups: whole multiples of 4 where the capacity allows it, so that the four
+    // schedulers of an SM can be given the same number of rows; otherwise as even as possible.
+    std::vector<int> size(n_rg, 0);
+    {
+        const int quads = (R + 3) / 4;
+        bool ok = true;
+        int left = R;
+        for (int i = 0; i < n_rg; ++i) {
+            const int q = quads / n_rg + (i < quads % n_rg ? 1 : 0);
+            size[i] = std::min(4 * q, left);
+            left -= size[i];
+            if (size[i] > cap) ok = false;
+        }
+        if (!ok || left > 0) {
+            for (int i = 0; i < n_rg; ++i) size[i] = R / n_rg + (i < R % n_rg ? 1 : 0);
+        }
+    }
+
+    // rows by descending kept-block count, dealt to the row groups in serpentine order (skipping full ones)
+    std::vector<int> order(R);
+    std::iota(order.begin(), order.end(), 0);
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+        return p.row_ptr[a + 1] - p.row_ptr[a] > p.row_ptr[b + 1] - p.row_ptr[b];
+    });
+    std::vector<std::vector<int>> members(n_rg);
+    {
+        int pos = 0, dir = 1, i = 0;
+        while (i < R) {
+            if ((int)members[pos].size() < size[pos]) members[pos].push_back(order[i++]);
+            if (pos + dir < 0 || pos + dir >= n_rg) dir = -dir; else pos += dir;
+        }
+    }
+
+    // Inside a row group: rows (longest first) are dealt in serpentine order to the schedulers
+    // (scheduler of consumer warp w = w mod 4), then, per scheduler, to its warps; the t-th row a
+    // warp receives becomes its accumulator set t.
+    out.h_rowmap.assign((size_t)n_rg * cap, -1);
+    const int nsched = std::min(4, nw);
+    for (int rg = 0; rg < n_rg; ++rg) {
+        std::vector<std::vector<int>> per(nsched);
+        std::vector<int> room(nsched, 0);
+        for (int w = 0; w < nw; ++w) room[w % nsched] += rw;
+        {
+            int pos = 0, dir = 1;
+            size_t i = 0;
+            while (i < members[rg].size()) {
+                if ((int)per[pos].size() < room[pos]) per[pos].push_back(members[rg][i++]);
+                if (pos + dir < 0 || pos + dir >= nsched) dir = -dir; else pos += dir;
+            }
+        }
+        for (int k = 0; k < nsched; ++k) {
+            std::vector<int> warps;
+            for (int w = k; w < nw; w += nsched) warps.push_back(w);
+            std::vector<int> fill(warps.size(), 0);
+            int pos = 0, dir = 1;
+            size_t i = 0;
+            while (i < per[k].size()) {
+                if (fill[pos] < rw) {
+                    out.h_rowmap[(size_t)rg * cap + local_row_of(warps[pos], fill[pos], nw)] = per[k][i++];
+                    ++fill[pos];
+                }
+                if (pos + dir < 0 || pos + dir >= (int)warps.size()) dir = -dir; else pos += dir;
+            }
+        }
+    }
+    emit_pair_records(p, kc, with_records, out);
 }
 
 // Tensor-core flavour of the schedule (fp16 weights): see the comment on Schedule.
@@ -290,6 +385,99 @@ void build_schedule_mma(const alcs_packed& p, int kc, int n_rg, bool with_record
 }  // namespace alcs
 
 extern "C" {
+
+ALCS_API int alcs_schedule_selfcheck(const alcs_packed* p, int chunk_channels, int row_groups, int warps, int slots,
+                                     int64_t* stats)
+{
+    if (!p || warps < 1 || warps > 32 || slots < 1 || slots > 15) return ALCS_ERR_INVALID_ARG;
+    alcs::Schedule sc;
+    try {
+        alcs::build_schedule_balanced(*p, chunk_channels, row_groups, warps, slots, true, sc);
+    } catch (const std::bad_alloc&) {
+        return ALCS_ERR_ALLOC;
+    }
+    const int g = p->g, cap = warps * slots;
+    const int REC = alcs::pair_record_bytes(g);
+    if (sc.rpg != cap || sc.ros != 4 * cap) return ALCS_ERR_CORRUPT;
+    // every block row exactly once in the row map
+    std::vector<int> seen(p->rows, 0);
+    for (int v : sc.h_rowmap)
+        if (v >= 0) { if (v >= p->rows) return ALCS_ERR_CORRUPT; ++seen[v]; }
+    for (int r = 0; r < p->rows; ++r)
+        if (seen[r] != 1) return ALCS_ERR_CORRUPT;
+    // walk every (warp, accumulator set) the way a consumer warp does and rebuild the dense matrix
+    std::vector<float> dense((size_t)p->rows * g * p->cin, 0.0f);
+    std::vector<uint8_t> hit((size_t)p->rows * p->cin, 0);
+    int64_t pairs = 0, max_sched = 0, min_sched = LLONG_MAX, max_rows = 0, min_rows = LLONG_MAX;
+    const int nsched = std::min(4, warps);
+    for (int rg = 0; rg < sc.n_rg; ++rg) {
+        std::vector<int64_t> per_sched(nsched, 0), rows_sched(nsched, 0);
+        for (int w = 0; w < warps; ++w)
+            for (int s = 0; s < slots; ++s)
+                if (sc.h_rowmap[(size_t)rg * cap + alcs::local_row_of(w, s, warps)] >= 0) ++rows_sched[w % nsched];
+        for (int c = 0; c < sc.nch; ++c) {
+            const size_t slice0 = (size_t)sc.h_slice[(size_t)rg * sc.nch + c] * 16;
+            const size_t slice1 = (size_t)sc.h_slice[(size_t)rg * sc.nch + c + 1] * 16;
+            const int* hdrs = &sc.h_rowoff[((size_t)rg * sc.nch + c) * sc.ros];
+            for (int w = 0; w < warps; ++w) {
+                for (int s = 0; s < slots; ++s) {
+                    const int lrow = alcs::local_row_of(w, s, warps);
+                    const int* hd = hdrs + 4 * lrow;       // {segment start, c0, c1, pairs}
+                    const int row = sc.h_rowmap[(size_t)rg * cap + lrow];
+                    if (hd[3] < 0 || (row < 0 && hd[3] != 0)) return ALCS_ERR_CORRUPT;
+                    int c0 = hd[1], c1 = hd[2];
+                    size_t rp = slice0 + (size_t)hd[0] * 16;
+                    for (int q = 0; q < hd[3]; ++q) {
+                        if (rp + REC > slice1) return ALCS_ERR_CORRUPT;
+                        const unsigned char* rec = &sc.h_rec[rp];
+                        int h[2];
+                        std::memcpy(h, rec, 8);
+                        const float* wv = reinterpret_cast<const float*>(rec + (g == 1 ? 8 : 16));
+                        const int cols[2] = {c0 + c * sc.kc, c1 + c * sc.kc};
+                        for (int b = 0; b < 2; ++b) {
+                            if (cols[b] < 0 || cols[b] >= p->cin || cols[b] >= (c + 1) * sc.kc) return ALCS_ERR_CORRUPT;
+                            for (int j = 0; j < g; ++j) dense[((size_t)row * g + j) * p->cin + cols[b]] += wv[b * g + j];
+                            if (b == 0 || cols[1] != cols[0]) ++hit[(size_t)row * p->cin + cols[b]];
+                        }
+                        per_sched[w % nsched] += 2;
+                        ++pairs;
+                        c0 = h[0]; c1 = h[1];
+                        rp += REC;
+                    }
+                }
+            }
+        }
+        for (int k = 0; k < nsched; ++k) {
+            max_sched = std::max(max_sched, per_sched[k]); min_sched = std::min(min_sched, per_sched[k]);
+            max_rows = std::max(max_rows, rows_sched[k]); min_rows = std::min(min_rows, rows_sched[k]);
+        }
+    }
+    // compare with the canonical storage
+    for (int r = 0; r < p->rows; ++r) {
+        int k = p->row_ptr[r];
+        for (int c = 0; c < p->cin; ++c) {
+            const bool kept = k < p->row_ptr[r + 1] && p->col_idx[k] == c;
+            if ((hit[(size_t)r * p->cin + c] != 0) != kept) return ALCS_ERR_CORRUPT;
+            if (kept && hit[(size_t)r * p->cin + c] != 1) return ALCS_ERR_CORRUPT;
+            for (int j = 0; j < g; ++j) {
+                float v = 0.0f;
+                if (kept) {
+                    if (p->dt == ALCS_F32) std::memcpy(&v, &p->vals[((size_t)k * g + j) * 4], 4);
+                    else { uint16_t hb; std::memcpy(&hb, &p->vals[((size_t)k * g + j) * 2], 2); v = alcs::half_bits_to_float(hb); }
+                }
+                const float d = dense[((size_t)r * g + j) * p->cin + c];
+                if (std::memcmp(&d, &v, 4) != 0 && !(d == v)) return ALCS_ERR_CORRUPT;
+            }
+            if (kept) ++k;
+        }
+    }
+    if (stats) {
+        stats[0] = sc.n_rg; stats[1] = max_sched; stats[2] = min_sched == LLONG_MAX ? 0 : min_sched;
+        stats[3] = pairs; stats[4] = p->nb;
+        stats[5] = max_rows; stats[6] = min_rows == LLONG_MAX ? 0 : min_rows;
+    }
+    return ALCS_OK;
+}
 
 ALCS_API const char* alcs_strerror(int status)
 {

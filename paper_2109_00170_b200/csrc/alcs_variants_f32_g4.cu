@@ -23,6 +23,13 @@ static const KernelVariant kTable[] = {
     ALCS_VARIANT_P(float, 0, 4, 8, 2, 14, 1, 2),
     ALCS_VARIANT_P(float, 0, 4, 8, 2, 13, 1, 3),
     ALCS_VARIANT_P(float, 0, 4, 8, 1, 13, 1, 3),
+    ALCS_VARIANT_P(float, 0, 4, 8, 2, 12, 1, 4),
+    ALCS_VARIANT_P(float, 0, 4, 8, 2, 12, 1, 2),
+    ALCS_VARIANT_P(float, 0, 4, 8, 2, 12, 1, 1),
+    ALCS_VARIANT_P(float, 0, 4, 8, 3, 8, 1, 4),
+    ALCS_VARIANT_P(float, 0, 4, 8, 3, 8, 1, 2),
+    ALCS_VARIANT_P(float, 0, 4, 8, 1, 16, 1, 4),
+    ALCS_VARIANT_P(float, 0, 4, 8, 1, 16, 1, 2),
     ALCS_VARIANT_P(float, 0, 4, 8, 1, 19, 1, 1),
     ALCS_VARIANT_P(float, 0, 4, 8, 1, 18, 1, 2),
     ALCS_VARIANT_P(float, 0, 4, 4, 2, 7, 1, 1),
@@ -40,6 +47,14 @@ static const KernelVariant kTable[] = {
     ALCS_VARIANT_P(float, 0, 4, 4, 4, 15, 1, 1),
     ALCS_VARIANT_P(float, 0, 4, 4, 4, 14, 1, 2),
     ALCS_VARIANT_P(float, 0, 4, 4, 2, 23, 1, 1),
+    ALCS_VARIANT_P(float, 0, 4, 4, 4, 12, 1, 4),
+    ALCS_VARIANT_P(float, 0, 4, 4, 4, 12, 1, 2),
+    ALCS_VARIANT_P(float, 0, 4, 4, 6, 8, 1, 4),
+    ALCS_VARIANT_P(float, 0, 4, 4, 2, 16, 1, 4),
+    ALCS_VARIANT_P(float, 0, 4, 4, 3, 16, 1, 4),
+    ALCS_VARIANT_P(float, 0, 4, 4, 4, 16, 1, 2),
+    ALCS_VARIANT_P(float, 0, 4, 4, 8, 6, 1, 2),
+    ALCS_VARIANT_P(float, 0, 4, 4, 8, 8, 1, 4),
     ALCS_VARIANT_P(float, 0, 4, 16, 1, 7, 1, 1),
     ALCS_VARIANT_P(float, 0, 4, 16, 1, 11, 1, 1),
     ALCS_VARIANT_P(float, 0, 4, 16, 2, 7, 1, 1),

@@ -271,6 +271,41 @@ def measure_batch1(A, torch, dev, stream, steps, hbm_gbs, fp32_tf):
                      "nz_gflops": round(flops / cold_us / 1e3, 1), "frac": round(t_roof * 1e6 / cold_us, 4)}}
 
 
+def bench_loop_ceiling(args):
+    """What bounds the hot loop, measured on this GPU with the library's probes: the fp32 FMA rate
+    from registers, the cost of shared-memory loads, and the kernel's own segment loop running on
+    data that is already in shared memory (no staging, barriers or stores)."""
+    import torch
+    import paper_2109_00170_b200 as A
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    A.lib()
+    st = torch.cuda.current_stream()
+    sampler = ClockSampler(0)
+    sampler.start()
+    out = {"metric": "fraction of the fp32 CUDA-core peak reached by the segment loop on shared-memory-resident data",
+           "unit": "fraction", "n_gpus": 1, "data": "synthetic", "dtype": "f32", "higher_is_better": True,
+           "config": {"workload": "loop_ceiling"}}
+    out["fma_peak"] = {"scalar": A.alcs_probe_fma_peak(False, st), "packed": A.alcs_probe_fma_peak(True, st)}
+    out["lds_cycles_per_warp_instruction"] = {
+        f"{8 * b}-bit {'uniform' if u else 'distinct'}": round(A.alcs_probe_lds(b, u, st), 3)
+        for b in (16, 8, 4) for u in (False, True)}
+    loops = []
+    for g, p, rw, nw, deep in [(4, 8, 2, 16, False), (4, 8, 2, 16, True), (4, 8, 2, 12, False), (4, 8, 2, 12, True),
+                               (4, 8, 2, 8, True), (4, 8, 1, 16, False), (4, 16, 1, 16, False), (4, 16, 1, 12, True),
+                               (4, 4, 4, 16, False), (1, 8, 2, 16, False), (8, 4, 2, 16, False), (16, 4, 1, 16, False)]:
+        row = {"g": g, "pixels_per_lane": p, "rows_per_warp": rw, "warps": nw, "deep": deep, "frac_by_pairs_per_segment": {}}
+        for L in (1, 2, 3, 4, 8, 32):
+            r = A.alcs_probe_segment_loop(g, p, rw, nw, deep, L, st)
+            row["frac_by_pairs_per_segment"][str(L)] = round(r["frac_of_fp32_peak"], 4)
+            row["registers"], row["spill_bytes"] = r["registers"], r["spill_bytes"]
+        loops.append(row)
+    out["segment_loop"] = loops
+    out["value"] = max(r["frac_by_pairs_per_segment"]["32"] for r in loops if r["g"] == 4 and r["pixels_per_lane"] == 8)
+    out["clocks"] = sampler.stop()
+    print(json.dumps(out))
+
+
 def bench_latency_model(args):
     """`--workload latency_model`: the paper's Section 3.3 experiment on this GPU.  (1) For every layer
     of the batch-64 MobileNetV1 pointwise stack, time the sparse kernel at 11 densities (0, 0.1, ..., 1
@@ -472,7 +507,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="alcs", choices=["alcs", "reference"])
-    ap.add_argument("--workload", default="mbv1_b64", choices=sorted(WORKLOADS) + ["rn18_3x3_b32", "latency_model"])
+    ap.add_argument("--workload", default="mbv1_b64", choices=sorted(WORKLOADS) + ["rn18_3x3_b32", "latency_model", "loop_ceiling"])
     ap.add_argument("--no-tune", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=3)
@@ -486,9 +521,11 @@ def main():
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "alcs" else args.warmup
     wl = args.workload
-    if wl in ("rn18_3x3_b32", "latency_model"):
+    if wl in ("rn18_3x3_b32", "latency_model", "loop_ceiling"):
         if args.impl == "reference" or int(os.environ.get("WORLD_SIZE", "1")) > 1:
             raise SystemExit(f"{wl} is a single-GPU side workload of --impl alcs")
+        if wl == "loop_ceiling":
+            return bench_loop_ceiling(args)
         return bench_conv2d(args) if wl == "rn18_3x3_b32" else bench_latency_model(args)
     specs = config_layers(WORKLOADS[wl])
     if args.layers:
@@ -668,6 +705,11 @@ def main():
     roof.update({"traffic": stored_traffic(d["layer"], d["cfg"]), "kernel": "spconv1x1_mma_kernel" if d["cfg"].get("math_mode") == 2 else "spconv1x1_kernel", "layer": d["layer"],
                  "algorithmic_bytes": stats[dom]["bytes"], "algorithmic_flops": stats[dom]["flops"],
                  "peak_source": f"HBM {peak_src}; fp32 = {SM_COUNT} SMs x {FP32_LANES} lanes x 2 x {sm_max:.0f} MHz"})
+    # the fp32 peak as this GPU delivers it from registers, measured now (a few hundred microseconds)
+    with torch.cuda.stream(stream):
+        pk = A.alcs_probe_fma_peak(True, stream)
+    roof["peak_measured"] = {"value": round(pk["tflops"], 2), "unit": "TFLOP/s", "how": "fma.rn.f32x2 on register operands, 16 warps per SM",
+                             "frac_of_derived": round(pk["frac_of_fp32_peak"], 4)}
     sum_roof = sum(r["t_roof_us"] for r in rows)
     sum_us = sum(r["us"] for r in rows)
 

@@ -293,6 +293,43 @@ ALCS_API int alcs_spconv1x1_noalloc(const alcs_packed* w, const void* x, void* y
                                     const float* bias, unsigned flags, void* cuda_stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * Measurement probes (device).  The paper has no counterpart: they exist so that the roofline the
+ * kernels are judged against is measured on the GPU at hand instead of taken from a data sheet, and
+ * so that the ceiling of the hot loop of Section 3.2.2's "efficient multiplication computation" can be
+ * re-measured by anyone.  Each call launches one thread block per SM on cuda_stream, times it with
+ * CUDA events (best of three after a warm-up), allocates and frees a few hundred KB of device
+ * memory, and synchronises the stream: set-up / benchmarking use only.
+ *
+ * alcs_probe_fma_peak: dependent-chain-free fp32 FMAs on register operands, 16 warps per SM;
+ *   packed = 0 scalar fma.rn.f32, 1 the two-wide fma.rn.f32x2 the kernels use.
+ * alcs_probe_lds: cycles of the SM's load/store pipe one warp-wide shared-memory load instruction
+ *   costs when 16 warps do nothing else: bytes_per_lane 4, 8 or 16; uniform = 0 every lane its own
+ *   (conflict-free) address, 1 all lanes the same address.
+ * alcs_probe_segment_loop: the pointwise kernel's segment loop, compiled as in the kernel, on
+ *   synthetic segments of pairs_per_segment pair records that are resident in shared memory together
+ *   with a 64-channel X tile (no staging, no barriers, no stores): `warps` warps per SM, each with
+ *   rows_per_warp accumulator sets of g x pixels_per_lane; deep = 1 the flavour that keeps the next
+ *   pair's X vectors in a second register set.  Only a fixed list of shapes is compiled
+ *   (ALCS_ERR_UNSUPPORTED otherwise): g = 4 with (pixels, rows, warps, deep) in {(8,2,16,0), (8,2,16,1),
+ *   (8,2,12,0), (8,2,12,1), (8,2,8,1), (8,1,16,0), (16,1,16,0), (16,1,12,1), (4,4,16,0)}, and
+ *   (g, pixels, rows, warps, deep) in {(1,8,2,16,0), (8,4,2,16,0), (16,4,1,16,0)}.
+ * frac_of_fp32_peak is relative to SMs x 128 lanes x 2 x the device's maximum SM clock.
+ * Errors: INVALID_ARG, UNSUPPORTED, SHAPE, CUDA.
+ * ------------------------------------------------------------------------------------------- */
+typedef struct {
+    double ms;                  /* duration of one launch                                          */
+    double tflops;              /* fp32 FLOP/s reached, in units of 1e12                           */
+    double frac_of_fp32_peak;   /* the same as a fraction of SMs x 128 x 2 x max SM clock          */
+    int registers;              /* registers per thread of the probe kernel                        */
+    int spill_bytes;            /* local-memory bytes per thread (0 = no spills)                   */
+} alcs_probe_result;
+
+ALCS_API int alcs_probe_fma_peak(int packed, alcs_probe_result* out, void* cuda_stream);
+ALCS_API int alcs_probe_lds(int bytes_per_lane, int uniform, double* cycles_per_instruction, void* cuda_stream);
+ALCS_API int alcs_probe_segment_loop(int g, int pixels_per_lane, int rows_per_warp, int warps, int deep,
+                                     int pairs_per_segment, alcs_probe_result* out, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------------------
  * General k_h x k_w convolution (device), fp32.
  *
  * Operation: paper, Section 3.2.2, the convolution formula with all three sums,

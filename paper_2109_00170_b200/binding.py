@@ -29,7 +29,8 @@ EXPORTS = ["alcs_strerror", "alcs_last_cuda_error", "alcs_version", "alcs_pack",
            "alcs_spconv1x1", "alcs_spconv1x1_cfg",
            "alcs_spconv1x1_plan", "alcs_spconv1x1_tune", "alcs_spconv1x1_set_cfg", "alcs_spconv1x1_host_workspace",
            "alcs_spconv1x1_host", "alcs_spconv1x1_noalloc", "alcs_spconv2d", "alcs_spconv2d_cfg", "alcs_spconv2d_plan", "alcs_layer_latency", "alcs_network_latency",
-           "alcs_project_bisection", "alcs_stack_create", "alcs_stack_run", "alcs_stack_destroy"]
+           "alcs_project_bisection", "alcs_probe_fma_peak", "alcs_probe_lds", "alcs_probe_segment_loop",
+           "alcs_stack_create", "alcs_stack_run", "alcs_stack_destroy"]
 
 
 class AlcsError(RuntimeError):
@@ -65,6 +66,14 @@ class LatencyTable(C.Structure):
 class ProjectionResult(C.Structure):
     _fields_ = [("n_keep", C.c_int64), ("n0", C.c_int64), ("n1", C.c_int64), ("n_groups", C.c_int64),
                 ("iters", C.c_int), ("latency", C.c_double)]
+
+
+class ProbeResult(C.Structure):
+    _fields_ = [("ms", C.c_double), ("tflops", C.c_double), ("frac_of_fp32_peak", C.c_double),
+                ("registers", C.c_int), ("spill_bytes", C.c_int)]
+
+    def as_dict(self):
+        return {k: getattr(self, k) for k, _ in self._fields_}
 
 
 class Layer(C.Structure):
@@ -117,6 +126,9 @@ def lib():
     L.alcs_project_bisection.argtypes = [C.POINTER(vp), ip, ip, i, i, C.POINTER(LatencyTable), C.c_double, C.c_double,
                                          C.c_double, vp, C.POINTER(vp), C.POINTER(C.c_int64),
                                          C.POINTER(ProjectionResult), vp]
+    L.alcs_probe_fma_peak.argtypes = [i, C.POINTER(ProbeResult), vp]
+    L.alcs_probe_lds.argtypes = [i, i, C.POINTER(C.c_double), vp]
+    L.alcs_probe_segment_loop.argtypes = [i, i, i, i, i, i, C.POINTER(ProbeResult), vp]
     L.alcs_stack_create.argtypes = [C.POINTER(Layer), i, u, C.POINTER(vp)]
     L.alcs_stack_run.argtypes = [vp, vp]
     L.alcs_stack_destroy.argtypes = [vp]
@@ -404,6 +416,29 @@ def alcs_project_bisection(u_tilde, g: int, tables, tau: float, t_budget: float,
            "alcs_project_bisection")
     return {"n_keep": res.n_keep, "n0": res.n0, "n1": res.n1, "n_groups": res.n_groups, "iters": res.iters,
             "latency": res.latency, "kept_per_layer": list(kept)}
+
+
+def alcs_probe_fma_peak(packed: bool = True, stream=None) -> dict:
+    """Measured fp32 FMA rate of the current device from register operands."""
+    r = ProbeResult()
+    _check(lib().alcs_probe_fma_peak(1 if packed else 0, C.byref(r), _stream(stream)), "alcs_probe_fma_peak")
+    return r.as_dict()
+
+
+def alcs_probe_lds(bytes_per_lane: int, uniform: bool, stream=None) -> float:
+    """Load/store-pipe cycles per warp-wide shared-memory load instruction."""
+    v = C.c_double()
+    _check(lib().alcs_probe_lds(bytes_per_lane, 1 if uniform else 0, C.byref(v), _stream(stream)), "alcs_probe_lds")
+    return v.value
+
+
+def alcs_probe_segment_loop(g: int, pixels_per_lane: int, rows_per_warp: int, warps: int, deep: bool,
+                            pairs_per_segment: int, stream=None) -> dict:
+    """The kernel's segment loop on shared-memory-resident synthetic segments."""
+    r = ProbeResult()
+    _check(lib().alcs_probe_segment_loop(g, pixels_per_lane, rows_per_warp, warps, 1 if deep else 0,
+                                         pairs_per_segment, C.byref(r), _stream(stream)), "alcs_probe_segment_loop")
+    return r.as_dict()
 
 
 class Stack:

@@ -144,6 +144,61 @@ int oracle_conv1x1(const void *W, const uint8_t *mask, int g, const void *X, con
 }
 
 /*
+ * Pointwise convolution with stride and a residual operand (the shape of a ResNet bottleneck's last
+ * 1x1 convolution and of its projection shortcut): the paper's formula at k_h = k_w = 1 sampled at
+ * stride s,
+ *     O(co, oh, ow) = sum_c Wm(co, c) * I(c, oh*s, ow*s),   oh < ceil(h/s), ow < ceil(wd/s),
+ * then  y = O + bias + R  and, if relu, y = max(y, 0): the residual is added BEFORE the activation.
+ * X [n][cin][h][wd]; R (may be NULL) [n][cout][oh*ow] of fp32, or of binary16 if res_is_f16;
+ * Y, A (double, [n][cout][oh*ow]) may each be NULL; A = |bias| + |R| + sum |Wm||I|.
+ * Dense triple loop, no zero skipping.  Returns 0, -1 on bad arguments.
+ */
+int oracle_conv1x1_ex(const void *W, const uint8_t *mask, int g, const void *X, const float *bias,
+                      const void *R, int res_is_f16, int relu, int is_f16, int n, int cin, int cout,
+                      int h, int wd, int stride, double *Y, double *A)
+{
+    if (!W || !mask || !X || g < 1 || n < 0 || cin < 0 || cout < 0 || h < 0 || wd < 0 || stride < 1) return -1;
+    const int oh = (h + stride - 1) / stride, ow = (wd + stride - 1) / stride;
+    const size_t ohw = (size_t)oh * ow, hw = (size_t)h * wd;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int in = 0; in < n; ++in) {
+        for (int co = 0; co < cout; ++co) {
+            for (int y = 0; y < oh; ++y) {
+                for (int x = 0; x < ow; ++x) {
+                    double acc = 0.0, mag = 0.0;
+#if ORACLE_MUTANT == 11           /* sampling grid shifted by one pixel */
+                    const size_t pin = (size_t)(y * stride + (stride > 1 && y * stride + 1 < h ? 1 : 0)) * wd + (size_t)x * stride;
+#else
+                    const size_t pin = (size_t)(y * stride) * wd + (size_t)x * stride;
+#endif
+                    for (int ci = 0; ci < cin; ++ci) {
+                        const double wm = masked_weight(W, is_f16, mask, g, cin, cout, co, ci);
+                        const size_t xi = ((size_t)in * cin + ci) * hw + pin;
+                        const double xv = is_f16 ? ld_f16(X, xi) : ld_f32(X, xi);
+                        acc += wm * xv;
+                        mag += fabs(wm) * fabs(xv);
+                    }
+                    const double b = bias ? (double)bias[co] : 0.0;
+                    const size_t yo = ((size_t)in * cout + co) * ohw + (size_t)y * ow + x;
+                    const double r = R ? (res_is_f16 ? ld_f16(R, yo) : ld_f32(R, yo)) : 0.0;
+#if ORACLE_MUTANT == 10           /* residual added after the activation */
+                    double s = acc + b;
+                    if (relu && s < 0.0) s = 0.0;
+                    s += r;
+#else
+                    double s = acc + b + r;
+                    if (relu && s < 0.0) s = 0.0;
+#endif
+                    if (Y) Y[yo] = s;
+                    if (A) A[yo] = mag + fabs(b) + fabs(r);
+                }
+            }
+        }
+    }
+    return 0;
+}
+
+/*
  * Selected outputs only: idx[k] is a flat index into Y[n][cout][hw]; out[k] (and mag[k] if
  * mag != NULL) receive the same quantities as oracle_conv1x1.  For full-size workloads where
  * the whole output would take too long.

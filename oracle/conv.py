@@ -25,6 +25,9 @@ def _lib(mutant: int = 0, build_dir: str | None = None):
     lib.oracle_conv1x1_points.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p,
                                           C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_long,
                                           C.c_void_p, C.c_long, C.c_void_p, C.c_void_p]
+    lib.oracle_conv1x1_ex.restype = C.c_int
+    lib.oracle_conv1x1_ex.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p] + \
+                                     [C.c_int] * 9 + [C.c_void_p, C.c_void_p]
     lib.oracle_conv2d.restype = C.c_int
     lib.oracle_conv2d.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p,
                                   C.c_int, C.c_int] + [C.c_int] * 9 + [C.c_void_p, C.c_void_p]
@@ -80,6 +83,32 @@ def conv1x1(W, mask, X, bias=None, relu=False, g=4, want_scale=False, mutant=0, 
         int(W.dtype == np.float16), n, cin, cout, hw, _ptr(Y), _ptr(A))
     if rc != 0:
         raise RuntimeError(f"oracle_conv1x1 failed: {rc}")
+    return (Y, A) if want_scale else Y
+
+
+def conv1x1_ex(W, mask, X, bias=None, residual=None, relu=False, g=4, stride=1, want_scale=False, mutant=0,
+               build_dir=None):
+    """Strided pointwise convolution with a residual: X [n,cin,h,wd], residual [n,cout,oh*ow] (float32 or
+    float16) or None; Y[n,cout,oh*ow] (float64) = relu?(Wm X[:, :, ::s, ::s] + bias + residual).
+    With want_scale also returns A = |bias| + |residual| + sum |Wm||X|."""
+    if X.ndim != 4:
+        raise ValueError("X must be [n, cin, h, wd]")
+    n, cin, h, wd = X.shape
+    W, mask, _, bias, n, cin, cout, _ = _prep(W, mask, X.reshape(n, cin, h * wd), bias, g)
+    X = np.ascontiguousarray(X)
+    oh, ow = -(-h // stride), -(-wd // stride)
+    if residual is not None:
+        if residual.dtype not in (np.float32, np.float16) or residual.shape != (n, cout, oh * ow):
+            raise ValueError("residual must be float32/float16 [n, cout, oh*ow]")
+        residual = np.ascontiguousarray(residual)
+    Y = np.empty((n, cout, oh * ow), dtype=np.float64)
+    A = np.empty((n, cout, oh * ow), dtype=np.float64) if want_scale else None
+    rc = _lib(mutant, build_dir).oracle_conv1x1_ex(
+        _ptr(W), _ptr(mask), g, _ptr(X), _ptr(bias), _ptr(residual),
+        int(residual is not None and residual.dtype == np.float16), int(bool(relu)),
+        int(W.dtype == np.float16), n, cin, cout, h, wd, stride, _ptr(Y), _ptr(A))
+    if rc != 0:
+        raise RuntimeError(f"oracle_conv1x1_ex failed: {rc}")
     return (Y, A) if want_scale else Y
 
 

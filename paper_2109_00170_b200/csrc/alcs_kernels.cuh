@@ -126,8 +126,11 @@ __device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.w
 __device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
 
 // Bounded wait for the phase with the given parity to complete.  Each poll lets the hardware
-// suspend the warp for up to about a microsecond, and failed polls back off with nanosleep, so a
-// waiting warp does not take issue slots from the warps that compute.
+// suspend the warp until the phase completes or a time limit passes, so a waiting warp takes few
+// issue slots from the warps that compute; the warp is not put to sleep between polls, because a
+// sleeping warp notices the hand-over of a pipeline stage up to a sleep period late, and with two
+// or three stages that delay sits on the critical path of every chunk.  Only a wait that has already
+// lasted thousands of polls backs off with nanosleep.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
 {
     for (int it = 0; it < kWaitLimit; ++it) {
@@ -139,7 +142,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
             : "r"(bar), "r"(parity), "r"(1000u)
             : "memory");
         if (done) return true;
-        if (it > 4) __nanosleep(it > 64 ? 256 : 64);
+        if (it > 4096) __nanosleep(128);
     }
     return false;
 }
@@ -418,7 +421,13 @@ __device__ __forceinline__ void produce(const ConvArgs& a, unsigned char* smem, 
         const int* slice = a.slice + rg * a.nch;
         const int* rowoff = a.rowoff + (size_t)rg * a.nch * a.ros;
 
+        int sl_lo = 0, sl_hi = 0;           // slice bounds of chunks k0 + lane, fetched 32 chunks at a time
         for (int k = 0; k < a.nch; ++k, ++kk) {
+            // (a load per chunk here would put a global-memory round trip in front of every stage's copies)
+            if ((k & 31) == 0) {
+                sl_lo = k + lane <= a.nch ? __ldg(slice + k + lane) : 0;
+                sl_hi = k + lane + 1 <= a.nch ? __ldg(slice + k + lane + 1) : sl_lo;
+            }
             const int s = turn * S + kk % S;
             if (kk >= S) {                  // wait until the consumers have released this stage
                 if (!mbar_wait(smem_u32 + 8 * kMaxStages + 8 * s, ((kk / S) - 1) & 1)) {
@@ -429,8 +438,8 @@ __device__ __forceinline__ void produce(const ConvArgs& a, unsigned char* smem, 
             }
             const uint32_t st = ring + s * a.stage_bytes;
             // the row group's pair records of this chunk and their per-row offsets
-            const int r0 = __ldg(slice + k);
-            const int n16 = __ldg(slice + k + 1) - r0;
+            const int r0 = __shfl_sync(0xffffffffu, sl_lo, k & 31);
+            const int n16 = __shfl_sync(0xffffffffu, sl_hi, k & 31) - r0;
             const unsigned char* rsrc = a.rec + (size_t)r0 * 16;
             for (int i = lane + 32 * pw; i < n16; i += 32 * npw) cp_async_16(st + a.off_rec + i * 16, rsrc + (size_t)i * 16);
             const int* osrc = rowoff + (size_t)k * a.ros;
@@ -502,7 +511,12 @@ __device__ __forceinline__ void produce_bulk(const ConvArgs& a, unsigned char* s
         const int* slice = a.slice + rg * a.nch;
         const int* rowoff = a.rowoff + (size_t)rg * a.nch * a.ros;
 
+        int sl_lo = 0, sl_hi = 0;           // slice bounds of chunks k0 + lane, fetched 32 chunks at a time
         for (int k = 0; k < a.nch; ++k, ++kk) {
+            if ((k & 31) == 0) {
+                sl_lo = k + lane <= a.nch ? __ldg(slice + k + lane) : 0;
+                sl_hi = k + lane + 1 <= a.nch ? __ldg(slice + k + lane + 1) : sl_lo;
+            }
             const int s = turn * S + kk % S;
             if (kk >= S) {
                 if (!mbar_wait(smem_u32 + 8 * kMaxStages + 8 * s, ((kk / S) - 1) & 1)) {
@@ -515,8 +529,8 @@ __device__ __forceinline__ void produce_bulk(const ConvArgs& a, unsigned char* s
                 const uint32_t bar = smem_u32 + 8 * s;
                 const int cbase = k * a.kc;
                 const int nrows = min(a.kc, a.cin - cbase);
-                const int r0 = __ldg(slice + k);
-                const int rbytes = (__ldg(slice + k + 1) - r0) * 16;
+                const int r0 = __shfl_sync(0xffffffffu, sl_lo, k & 31);
+                const int rbytes = (__shfl_sync(0xffffffffu, sl_hi, k & 31) - r0) * 16;
                 if (lane == 0 && pw == 0) mbar_arrive_expect_tx(bar, (uint32_t)(nrows * vt * SZ + rbytes + a.ros * 4));
                 __syncwarp();
                 if (lane == 0 && pw == 0 && rbytes > 0) bulk_copy_g2s(st + a.off_rec, a.rec + (size_t)r0 * 16, (uint32_t)rbytes, bar);
@@ -619,6 +633,17 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_kernel(const 
         for (int s = 0; s < RW; ++s) {
             lrow[s] = s * NW + ((s & 1) ? NW - 1 - warp : warp);
             rowid[s] = lrow[s] < a.rpg ? __ldg(a.rowmap + rg * a.rpg + lrow[s]) : -1;
+        }
+
+        // bring the rows' bias values into L1 now, so that the epilogue does not start with a
+        // global-memory round trip
+        if (a.bias) {
+#pragma unroll
+            for (int s = 0; s < RW; ++s)
+                if (rowid[s] >= 0 && lane == 0) {
+                    const float* bp = a.bias + min(rowid[s] * G, a.cout - 1);
+                    asm volatile("prefetch.global.L1 [%0];\n" ::"l"(bp));
+                }
         }
 
         float2 acc[RW][G][P / 2];

@@ -39,7 +39,7 @@
 extern "C" {
 #endif
 
-#define ALCS_VERSION 1
+#define ALCS_VERSION 2
 
 typedef enum {
     ALCS_OK = 0,
@@ -219,6 +219,24 @@ ALCS_API int alcs_variant_get(int index, alcs_dtype* dt, int* g, alcs_launch_cfg
  */
 ALCS_API int alcs_spconv1x1(const alcs_packed* w, const void* x, void* y, int n, int h, int wd,
                    const float* bias, unsigned flags, void* cuda_stream);
+
+/*
+ * alcs_spconv1x1_ex: the pointwise convolution with a stride and a residual operand (paper, Section
+ * 3.2.2, the convolution formula at k_h = k_w = 1 sampled every `stride` pixels -- the 1x1 projection
+ * shortcuts of the ResNets evaluated in Section 4.1 -- and, for the last 1x1 convolution of a
+ * bottleneck, the shortcut added before the activation):
+ *     y[n][co][oh][ow] = act( sum_c W(co,c) * x[n][c][oh*stride][ow*stride] + bias[co] + residual[n][co][oh][ow] ),
+ * oh < ceil(h/stride), ow < ceil(wd/stride).  x device [n][cin][h][wd]; y and residual device
+ * [n][cout][oh*ow] of the same element type (the packed dtype, or fp32 with ALCS_Y_F32); residual may be
+ * NULL; it must not overlap y.  stride = 1 with residual = NULL is alcs_spconv1x1_cfg.  With stride > 1
+ * the pixels that are read are first gathered, by a small kernel on the same stream, into the scratch
+ * memory owned by w (see alcs_spconv1x1); the residual is read straight from the caller's buffer in the
+ * epilogue, added in fp32 before ReLU and before the single rounding of an fp16 output.  cfg may be
+ * NULL.  Errors as alcs_spconv1x1, plus INVALID_ARG for stride < 1.
+ */
+ALCS_API int alcs_spconv1x1_ex(const alcs_packed* w, const void* x, void* y, int n, int h, int wd, int stride,
+                               const float* bias, const void* residual, unsigned flags,
+                               const alcs_launch_cfg* cfg, void* cuda_stream);
 
 /* Same, with an explicit launch configuration (cfg == NULL behaves like alcs_spconv1x1). */
 ALCS_API int alcs_spconv1x1_cfg(const alcs_packed* w, const void* x, void* y, int n, int h, int wd,
@@ -446,6 +464,8 @@ typedef struct {
     int n, h, wd;
     const float* bias;          /* device fp32 [cout] or NULL                  */
     unsigned flags;             /* ALCS_RELU | ALCS_Y_F32                      */
+    const void* residual;       /* device, shape and type of y, or NULL (see alcs_spconv1x1_ex) */
+    int stride;                 /* 0 or 1: none; > 1: y is [n][cout][ceil(h/stride)*ceil(wd/stride)] */
 } alcs_layer;
 
 #define ALCS_STACK_GRAPH 1u     /* replay the launches as one CUDA graph       */

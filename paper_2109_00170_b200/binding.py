@@ -26,7 +26,7 @@ EXPORTS = ["alcs_strerror", "alcs_last_cuda_error", "alcs_version", "alcs_pack",
            "alcs_packed_view", "alcs_packed_serialize", "alcs_packed_deserialize",
            "alcs_packed_upload", "alcs_packed_status", "alcs_packed_free", "alcs_schedule_selfcheck",
            "alcs_variant_count", "alcs_variant_get",
-           "alcs_spconv1x1", "alcs_spconv1x1_cfg",
+           "alcs_spconv1x1", "alcs_spconv1x1_cfg", "alcs_spconv1x1_ex",
            "alcs_spconv1x1_plan", "alcs_spconv1x1_tune", "alcs_spconv1x1_set_cfg", "alcs_spconv1x1_host_workspace",
            "alcs_spconv1x1_host", "alcs_spconv1x1_noalloc", "alcs_spconv2d", "alcs_spconv2d_cfg", "alcs_spconv2d_plan", "alcs_layer_latency", "alcs_network_latency",
            "alcs_project_bisection", "alcs_probe_fma_peak", "alcs_probe_lds", "alcs_probe_segment_loop",
@@ -78,7 +78,8 @@ class ProbeResult(C.Structure):
 
 class Layer(C.Structure):
     _fields_ = [("w", C.c_void_p), ("x", C.c_void_p), ("y", C.c_void_p), ("n", C.c_int),
-                ("h", C.c_int), ("wd", C.c_int), ("bias", C.c_void_p), ("flags", C.c_uint)]
+                ("h", C.c_int), ("wd", C.c_int), ("bias", C.c_void_p), ("flags", C.c_uint),
+                ("residual", C.c_void_p), ("stride", C.c_int)]
 
 
 _lib = None
@@ -111,6 +112,7 @@ def lib():
     L.alcs_variant_get.argtypes = [i, ip, ip, C.POINTER(LaunchCfg)]
     L.alcs_spconv1x1.argtypes = [vp, vp, vp, i, i, i, vp, u, vp]
     L.alcs_spconv1x1_cfg.argtypes = [vp, vp, vp, i, i, i, vp, u, C.POINTER(LaunchCfg), vp]
+    L.alcs_spconv1x1_ex.argtypes = [vp, vp, vp, i, i, i, i, vp, vp, u, C.POINTER(LaunchCfg), vp]
     L.alcs_spconv1x1_plan.argtypes = [vp, i, i, i, u, C.POINTER(LaunchCfg)]
     L.alcs_spconv1x1_tune.argtypes = [vp, vp, vp, i, i, i, vp, u, vp, C.POINTER(LaunchCfg)]
     L.alcs_spconv1x1_set_cfg.argtypes = [vp, i, i, i, u, C.POINTER(LaunchCfg)]
@@ -304,6 +306,14 @@ def alcs_spconv1x1(w: Packed, x, y, n: int, h: int, wd: int, bias=None, flags: i
     _check(st, "alcs_spconv1x1")
 
 
+def alcs_spconv1x1_ex(w: Packed, x, y, n: int, h: int, wd: int, stride: int = 1, bias=None, residual=None,
+                      flags: int = 0, stream=None, cfg=None):
+    """Strided pointwise convolution with a residual operand added before the activation."""
+    c = _cfg(cfg)
+    _check(lib().alcs_spconv1x1_ex(w.handle, _addr(x), _addr(y), n, h, wd, stride, _addr(bias), _addr(residual), flags,
+                                   C.byref(c) if c is not None else None, _stream(stream)), "alcs_spconv1x1_ex")
+
+
 def alcs_spconv1x1_plan(w: Packed, n: int, h: int, wd: int, flags: int = 0) -> dict:
     c = LaunchCfg()
     _check(lib().alcs_spconv1x1_plan(w.handle, n, h, wd, flags, C.byref(c)), "alcs_spconv1x1_plan")
@@ -471,7 +481,7 @@ def alcs_stack_create(layers: Sequence[dict], stack_flags: int = 0) -> Stack:
     arr = (Layer * max(1, len(layers)))()
     for k, L in enumerate(layers):
         arr[k] = Layer(L["w"].handle, _addr(L["x"]), _addr(L["y"]), L["n"], L["h"], L["wd"],
-                       _addr(L.get("bias")), L.get("flags", 0))
+                       _addr(L.get("bias")), L.get("flags", 0), _addr(L.get("residual")), L.get("stride", 1))
     out = C.c_void_p()
     _check(lib().alcs_stack_create(arr, len(layers), stack_flags, C.byref(out)), "alcs_stack_create")
     return Stack(out.value, list(layers))

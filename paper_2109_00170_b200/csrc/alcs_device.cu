@@ -276,7 +276,11 @@ bool gather_plan(const alcs_packed* w, int n, int hw, int p, int ks, const Devic
 }
 
 // Enumerate every valid launch configuration for this shape, cheapest (by the model) first.
-int enumerate_plans(const alcs_packed* w, long long q, int hw, std::vector<Plan>& out)
+// Internal flag, only ever seen in plan-cache keys: the call has a residual operand or a stride, which
+// the small-problem kernel does not take, so only the staged kernels are listed.
+constexpr unsigned kStagedOnly = 0x10000u;
+
+int enumerate_plans(const alcs_packed* w, long long q, int hw, std::vector<Plan>& out, bool allow_small = true)
 {
     DeviceInfo di;
     int rc = device_info(w->device, &di);
@@ -344,7 +348,7 @@ int enumerate_plans(const alcs_packed* w, long long q, int hw, std::vector<Plan>
             }
         }
     }
-    if (hw > 0 && q / hw <= 8) {        // small batches only: one thread block per (block row, image, pixel tile)
+    if (allow_small && hw > 0 && q / hw <= 8) {        // small batches only: one thread block per (block row, image, pixel tile)
         for (int p = 8; p >= 2; p /= 2)
             for (int ks = 4; ks <= 16; ks *= 2) {
                 Plan g;
@@ -379,12 +383,13 @@ void plan_to_cfg(const Plan& p, alcs_launch_cfg* c)
 }
 
 // Resolve a (possibly partial) configuration into a concrete plan.
-int cfg_to_plan(const alcs_packed* w, long long q, int hw, const alcs_launch_cfg* c, Plan* out)
+int cfg_to_plan(const alcs_packed* w, long long q, int hw, const alcs_launch_cfg* c, Plan* out, bool allow_small = true)
 {
     std::vector<Plan> all;
-    int rc = enumerate_plans(w, q, hw, all);
+    int rc = enumerate_plans(w, q, hw, all, allow_small);
     if (rc) return rc;
     if (!c) { *out = all[0]; return ALCS_OK; }
+    if (c->math_mode == 3 && !allow_small) return ALCS_ERR_UNSUPPORTED;
     if (c->math_mode == 3) {        // the small-problem kernel, with the given (or the best-ranked) shape
         for (const Plan& p : all)
             if (p.gather && (!c->pixels_per_lane || c->pixels_per_lane == p.gp) && (!c->warps || c->warps == p.gks)) {
@@ -441,13 +446,17 @@ int cfg_to_plan(const alcs_packed* w, long long q, int hw, const alcs_launch_cfg
 }
 
 // X whose (image, channel) rows are not a multiple of 16 bytes long (H*W = 49, ...) cannot be staged
-// with 16-byte copies.  Such inputs are first repacked into scratch memory with every row padded
-// with zeros to the next multiple of 16 bytes; the main kernel then runs on the padded pixel axis
-// and simply does not store the padding pixels.
-// Each thread writes one 16-byte piece of a padded row (EPV elements), reading its elements one
-// by one: the source rows start at arbitrary element offsets.
+// with 16-byte copies, and a strided pointwise convolution reads only every stride-th pixel of every
+// stride-th row.  Such inputs are first gathered into scratch memory: the pixels the convolution
+// reads, row after row, every (image, channel) row padded with zeros to the next multiple of 16
+// bytes; the main kernel then runs on the padded pixel axis and simply does not store the padding
+// pixels.  Each thread writes one 16-byte piece of a padded row (EPV elements), reading its elements
+// one by one: the source rows start at arbitrary element offsets.
+// rows = n*cin; hw_in = elements per source row; output pixel p of a row is source pixel
+// (p / ow) * stride * wd_in + (p % ow) * stride; hw_out real and hwp padded pixels per output row.
 template <typename T>
-__global__ void repack_rows_kernel(const T* __restrict__ in, T* __restrict__ out, long long rows, int hw, int hwp)
+__global__ void repack_rows_kernel(const T* __restrict__ in, T* __restrict__ out, long long rows, int hw_in, int wd_in,
+                                   int ow, int stride, int hw_out, int hwp)
 {
     constexpr int EPV = 16 / (int)sizeof(T);
     const int vpr = hwp / EPV;                       // 16-byte pieces per padded row
@@ -456,10 +465,19 @@ __global__ void repack_rows_kernel(const T* __restrict__ in, T* __restrict__ out
          i += (long long)gridDim.x * blockDim.x) {
         const long long r = i / vpr;
         const int p0 = (int)(i - r * vpr) * EPV;
-        const T* src = in + r * hw + p0;
+        const T* src = in + r * hw_in;
         alignas(16) T v[EPV];
+        if (stride == 1) {
 #pragma unroll
-        for (int t = 0; t < EPV; ++t) v[t] = p0 + t < hw ? __ldg(src + t) : T(0);
+            for (int t = 0; t < EPV; ++t) v[t] = p0 + t < hw_out ? __ldg(src + p0 + t) : T(0);
+        } else {
+#pragma unroll
+            for (int t = 0; t < EPV; ++t) {
+                const int p = p0 + t;
+                const int oy = p / ow, ox = p - oy * ow;
+                v[t] = p < hw_out ? __ldg(src + (size_t)oy * stride * wd_in + (size_t)ox * stride) : T(0);
+            }
+        }
         *reinterpret_cast<uint4*>(out + r * hwp + p0) = *reinterpret_cast<const uint4*>(v);
     }
 }
@@ -553,10 +571,16 @@ int launch_gather_plan(const alcs_packed* w, const Plan& p, const void* x, void*
 // scratch / scratch_bytes: where X is repacked when its rows are not 16-byte multiples.  nullptr means
 // the scratch that w owns (allocated or grown here); a layer stack passes its own, fixed for the
 // stack's lifetime, so that a captured graph never refers to memory a later call may free.
+// residual (may be null): same shape and element type as y, added before the activation.  stride > 1:
+// h and wd are the OUTPUT size, h_in x wd_in the input size, and the pixels the convolution reads
+// are gathered into the scratch first.
 int launch_plan(const alcs_packed* w, const Plan& p, const void* x, void* y, int n, int h, int wd,
-                const float* bias, unsigned flags, cudaStream_t st, void* scratch = nullptr, size_t scratch_bytes = 0)
+                const float* bias, unsigned flags, cudaStream_t st, void* scratch = nullptr, size_t scratch_bytes = 0,
+                const void* residual = nullptr, int stride = 1, int h_in = 0, int wd_in = 0)
 {
+    if (stride <= 1) { stride = 1; h_in = h; wd_in = wd; }
     if (p.gather) {
+        if (residual || stride != 1) return ALCS_ERR_STATE;        // (plans for such calls never list that kernel)
         const int rc = ensure_canonical_on_device(w, st);
         return rc ? rc : launch_gather_plan(w, p, x, y, n, h, wd, bias, flags, st);
     }
@@ -575,26 +599,30 @@ int launch_plan(const alcs_packed* w, const Plan& p, const void* x, void* y, int
     // Rows of X that are not a multiple of 16 bytes long: repack X into scratch with padded rows.
     int hwx = hw;
     const void* xk = x;
-    if (((size_t)hw * elt) % 16 != 0) {
+    if (((size_t)hw * elt) % 16 != 0 || stride != 1) {
         const int hwp = padded_hw(hw, elt);
         const size_t need = (size_t)n * w->cin * hwp * elt;
         if (scratch && scratch_bytes < need) return ALCS_ERR_STATE;
-        if ((long long)n * hwp <= (1ll << 30) && (scratch || ensure_xpad(w, need) == ALCS_OK)) {
+        const bool have = (long long)n * hwp <= (1ll << 30) && (scratch || ensure_xpad(w, need) == ALCS_OK);
+        if (!have && stride != 1) return ALCS_ERR_ALLOC;         // a strided input cannot be staged in place
+        if (have) {
             void* const xpad = scratch ? scratch : w->d_xpad;
             const long long rows = (long long)n * w->cin;
             const unsigned blocks = (unsigned)std::min<long long>((rows * (hwp * elt / 16) + 255) / 256, (long long)di.sms * 16);
             if (elt == 4)
-                repack_rows_kernel<float><<<blocks, 256, 0, st>>>(static_cast<const float*>(x), static_cast<float*>(xpad), rows, hw, hwp);
+                repack_rows_kernel<float><<<blocks, 256, 0, st>>>(static_cast<const float*>(x), static_cast<float*>(xpad), rows,
+                                                                  h_in * wd_in, wd_in, wd, stride, hw, hwp);
             else
                 repack_rows_kernel<unsigned short><<<blocks, 256, 0, st>>>(static_cast<const unsigned short*>(x),
-                                                                          static_cast<unsigned short*>(xpad), rows, hw, hwp);
+                                                                          static_cast<unsigned short*>(xpad), rows,
+                                                                          h_in * wd_in, wd_in, wd, stride, hw, hwp);
             ALCS_CUDA(cudaGetLastError());
             xk = xpad;
             hwx = hwp;
         }   // else: fall back to element-wise staging of the unpadded rows
     }
     ConvArgs a;
-    a.x = xk; a.y = y; a.bias = bias;
+    a.x = xk; a.y = y; a.bias = bias; a.res = residual;
     a.rec = sc->rec; a.slice = sc->slice; a.rowoff = sc->rowoff; a.rowmap = sc->rowmap;
     a.err = w->d_err;
     a.rows = w->rows; a.cin = w->cin; a.cout = w->cout; a.hw = hwx; a.hwy = hw;
@@ -614,7 +642,7 @@ int launch_plan(const alcs_packed* w, const Plan& p, const void* x, void* y, int
     a.bulk = (ld == 16 && p.bulk) ? 1 : 0;
     a.ros = sc->ros;
     const int vg = (v.p * elt >= 16) ? 16 / elt : v.p;
-    a.st_vec = (hwx == hw && hw % vg == 0 && (uintptr_t)y % 16 == 0) ? 1 : 0;
+    a.st_vec = (hwx == hw && hw % vg == 0 && (uintptr_t)y % 16 == 0 && (uintptr_t)residual % 16 == 0) ? 1 : 0;
     a.st_grp = hwx % vg == 0 ? 1 : 0;
     const long long items = (long long)a.n_tiles * a.n_rg;
     if (items > 0x7fffffffll) return ALCS_ERR_SHAPE;
@@ -661,11 +689,11 @@ int resolve_plan(const alcs_packed* w, int n, int h, int wd, unsigned flags, lon
         if (it != w->plan_cache.end()) { *plan = it->second; return ALCS_OK; }
     }
     const alcs_launch_cfg* use = cfg;
-    if (!use) {
-        auto it = w->tuned.find(key);
-        if (it != w->tuned.end()) use = &it->second;
+    if (!use) {     // a configuration tuned or set for the shape (stored under the public flags)
+        auto it = w->tuned.find(alcs::ShapeKey{n, h, wd, flags & ~kStagedOnly});
+        if (it != w->tuned.end() && !((flags & kStagedOnly) && it->second.math_mode == 3)) use = &it->second;
     }
-    const int rc = cfg_to_plan(w, q, h * wd, use, plan);
+    const int rc = cfg_to_plan(w, q, h * wd, use, plan, !(flags & kStagedOnly));
     if (rc) return rc;
     std::lock_guard<std::mutex> lk(w->mu);
     w->plan_cache[key] = *plan;
@@ -705,6 +733,7 @@ struct alcs_stack {
         alcs_layer layer;
         Plan plan;
         long long q;
+        int oh, ow;         // output size (= h, wd unless the layer has a stride)
     };
     std::vector<Item> items;
     unsigned flags = 0;
@@ -826,6 +855,38 @@ ALCS_API int alcs_spconv1x1(const alcs_packed* w, const void* x, void* y, int n,
                    const float* bias, unsigned flags, void* cuda_stream)
 {
     return alcs_spconv1x1_cfg(w, x, y, n, h, wd, bias, flags, nullptr, cuda_stream);
+}
+
+ALCS_API int alcs_spconv1x1_ex(const alcs_packed* w, const void* x, void* y, int n, int h, int wd, int stride,
+                               const float* bias, const void* residual, unsigned flags,
+                               const alcs_launch_cfg* cfg, void* cuda_stream)
+{
+    if (stride < 1 || h < 0 || wd < 0) return ALCS_ERR_INVALID_ARG;
+    if (stride == 1 && !residual) return alcs_spconv1x1_cfg(w, x, y, n, h, wd, bias, flags, cfg, cuda_stream);
+    const int oh = (h + stride - 1) / stride, ow = (wd + stride - 1) / stride;
+    long long q = 0;
+    // argument checks on the output-sized problem ...
+    int rc = check_conv_args(w, x, y, n, oh, ow, flags, &q);
+    if (rc) return rc;
+    rc = check_device(w);
+    if (rc) return rc;
+    if (q == 0) return ALCS_OK;
+    // ... plus what is specific to this entry point: the true extent of x, and the residual
+    const size_t xe = w->elt(), ye = (w->dt == ALCS_F16 && !(flags & ALCS_Y_F32)) ? 2 : 4;
+    if ((long long)h * wd > (1ll << 30) || (long long)h * wd * n > (1ll << 31)) return ALCS_ERR_SHAPE;
+    const uintptr_t xb = (uintptr_t)x, xend = xb + (size_t)n * w->cin * h * wd * xe;
+    const uintptr_t yb = (uintptr_t)y, yend = yb + (size_t)q * w->cout * ye;
+    if (xb < yend && yb < xend) return ALCS_ERR_INVALID_ARG;
+    if (residual) {
+        const uintptr_t rb = (uintptr_t)residual, rend = rb + (size_t)q * w->cout * ye;
+        if (rb % ye) return ALCS_ERR_INVALID_ARG;
+        if (rb < yend && yb < rend) return ALCS_ERR_INVALID_ARG;     // the residual may not overlap y
+    }
+    Plan plan;
+    rc = resolve_plan(w, n, oh, ow, flags | kStagedOnly, q, cfg, &plan);
+    if (rc) return rc;
+    return launch_plan(w, plan, x, y, n, oh, ow, bias, flags, static_cast<cudaStream_t>(cuda_stream), nullptr, 0,
+                       residual, stride, h, wd);
 }
 
 ALCS_API int alcs_spconv1x1_plan(const alcs_packed* w, int n, int h, int wd, unsigned flags,
@@ -994,17 +1055,22 @@ ALCS_API int alcs_stack_create(const alcs_layer* layers, int n_layers, unsigned 
         const alcs_layer& L = layers[i];
         alcs_stack::Item it;
         it.layer = L;
-        int rc = check_conv_args(L.w, L.x, L.y, L.n, L.h, L.wd, L.flags, &it.q);
+        if (L.stride < 0) { delete s; return ALCS_ERR_INVALID_ARG; }
+        const int stride = L.stride > 1 ? L.stride : 1;
+        const bool extra = stride > 1 || L.residual;
+        it.oh = (L.h + stride - 1) / stride;
+        it.ow = (L.wd + stride - 1) / stride;
+        int rc = check_conv_args(L.w, L.x, L.y, L.n, it.oh, it.ow, L.flags, &it.q);
         if (!rc) rc = check_device(L.w);
-        if (!rc && it.q > 0) rc = resolve_plan(L.w, L.n, L.h, L.wd, L.flags, it.q, nullptr, &it.plan);
+        if (!rc && it.q > 0) rc = resolve_plan(L.w, L.n, it.oh, it.ow, L.flags | (extra ? kStagedOnly : 0u), it.q, nullptr, &it.plan);
         if (!rc && it.q > 0 && it.plan.gather) {
             rc = ensure_canonical_on_device(L.w, nullptr);
         } else if (!rc && it.q > 0) {   // the schedule must be resident before any launch is captured
             Schedule* sc = get_schedule(L.w, it.plan.kc, it.plan.n_rg, true, flavour_of(g_variants[it.plan.variant].v));
             rc = sc ? upload_schedule(L.w, sc, nullptr) : ALCS_ERR_ALLOC;
             const int elt = (int)L.w->elt();
-            const long long hw = (long long)L.h * L.wd;
-            if (!rc && (hw * elt) % 16 != 0 && (long long)L.n * padded_hw((int)hw, elt) <= (1ll << 30))
+            const long long hw = (long long)it.oh * it.ow;
+            if (!rc && ((hw * elt) % 16 != 0 || stride > 1) && (long long)L.n * padded_hw((int)hw, elt) <= (1ll << 30))
                 scratch_need = std::max(scratch_need, (size_t)L.n * L.w->cin * padded_hw((int)hw, elt) * elt);
         }
         if (rc) { delete s; return rc; }
@@ -1027,7 +1093,8 @@ static int stack_enqueue(alcs_stack* s, cudaStream_t st)
     for (auto& it : s->items) {
         if (it.q == 0) continue;
         const alcs_layer& L = it.layer;
-        int rc = launch_plan(L.w, it.plan, L.x, L.y, L.n, L.h, L.wd, L.bias, L.flags, st, s->xpad, s->xpad_bytes);
+        int rc = launch_plan(L.w, it.plan, L.x, L.y, L.n, it.oh, it.ow, L.bias, L.flags, st, s->xpad, s->xpad_bytes,
+                             L.residual, L.stride > 1 ? L.stride : 1, L.h, L.wd);
         if (rc) return rc;
     }
     return ALCS_OK;
@@ -1156,17 +1223,19 @@ extern "C" ALCS_API int alcs_spconv1x1_noalloc(const alcs_packed* w, const void*
         // the kernel writes every element of the region it uses, zero padding included, so nothing
         // left behind by an earlier call can leak into this one
         if (elt == 4)
-            repack_rows_kernel<float><<<blocks, 256, 0, st>>>(static_cast<const float*>(x), static_cast<float*>(scratch), rows, hw, hwp);
+            repack_rows_kernel<float><<<blocks, 256, 0, st>>>(static_cast<const float*>(x), static_cast<float*>(scratch), rows,
+                                                              hw, wd, wd, 1, hw, hwp);
         else
             repack_rows_kernel<unsigned short><<<blocks, 256, 0, st>>>(static_cast<const unsigned short*>(x),
-                                                                      static_cast<unsigned short*>(scratch), rows, hw, hwp);
+                                                                      static_cast<unsigned short*>(scratch), rows,
+                                                                      hw, wd, wd, 1, hw, hwp);
         ALCS_CUDA(cudaGetLastError());
         xk = scratch;
         hwx = hwp;
     }
 
     ConvArgs a;
-    a.x = xk; a.y = y; a.bias = bias;
+    a.x = xk; a.y = y; a.bias = bias; a.res = nullptr;
     a.rec = sc->rec; a.slice = sc->slice; a.rowoff = sc->rowoff; a.rowmap = sc->rowmap;
     a.err = w->d_err;
     a.rows = w->rows; a.cin = w->cin; a.cout = w->cout; a.hw = hwx; a.hwy = hw;

@@ -50,6 +50,7 @@ struct ConvArgs {
     const void* x;            // [n][cin][hw] of XT
     void* y;                  // [n][cout][hw] of XT, or float if y_f32
     const float* bias;        // [cout] or nullptr
+    const void* res;          // residual, same shape and element type as y, or nullptr: y = act(acc + bias + res)
     const unsigned char* rec; // segments of pair records, ordered [row group][chunk][local row]
     const int* slice;         // [n_rg*nch + 1] start of each (row group, chunk) slice, in 16-byte units
     const int* rowoff;        // [n_rg][nch][rpg] int4 per local row: {segment start inside the slice (16-byte units), c0, c1, pairs}
@@ -373,6 +374,39 @@ __device__ __forceinline__ void store_one(YT* p, float v)
         *p = v;
     else
         *p = __float2half_rn(v);
+}
+
+// The residual operand at the position of a store: VG consecutive elements, or one, widened to fp32.
+template <typename YT, int VG>
+__device__ __forceinline__ void load_res_vec(const YT* p, float (&v)[VG])
+{
+    if constexpr (sizeof(YT) == 4) {
+#pragma unroll
+        for (int i = 0; i < VG / 4; ++i) {
+            const float4 r = __ldg(reinterpret_cast<const float4*>(p) + i);
+            v[4 * i] = r.x; v[4 * i + 1] = r.y; v[4 * i + 2] = r.z; v[4 * i + 3] = r.w;
+        }
+    } else {
+        __half2 h[VG / 2];
+        if constexpr (VG == 8)
+            *reinterpret_cast<uint4*>(h) = __ldg(reinterpret_cast<const uint4*>(p));
+        else
+            *reinterpret_cast<uint2*>(h) = __ldg(reinterpret_cast<const uint2*>(p));
+#pragma unroll
+        for (int i = 0; i < VG / 2; ++i) {
+            const float2 f = __half22float2(h[i]);
+            v[2 * i] = f.x; v[2 * i + 1] = f.y;
+        }
+    }
+}
+
+template <typename YT>
+__device__ __forceinline__ float load_res_one(const YT* p)
+{
+    if constexpr (sizeof(YT) == 4)
+        return __ldg(p);
+    else
+        return __half2float(__ldg(p));
 }
 
 // ---- producer: one warp copies (item, chunk) after (item, chunk) into the ring ---------------
@@ -704,18 +738,35 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_kernel(const 
                         for (int t = 0; t < VG; ++t) {
                             const float2 a2 = acc[s][j][(gi * VG + t) / 2];
                             v[t] = (((gi * VG + t) & 1) ? a2.y : a2.x) + bv;
-                            if (a.relu) v[t] = fmaxf(v[t], 0.0f);
                         }
+                        const YT* rbase = static_cast<const YT*>(a.res);
                         if (a.st_vec) {
-                            if (yok[gi]) store_vec<YT, VG>(ybase + yoff[gi] + (size_t)co * a.hwy, v);
+                            if (yok[gi]) {
+                                const size_t o = yoff[gi] + (size_t)co * a.hwy;
+                                if (rbase) {
+                                    float r[VG];
+                                    load_res_vec<YT, VG>(rbase + o, r);
+#pragma unroll
+                                    for (int t = 0; t < VG; ++t) v[t] += r[t];
+                                }
+                                if (a.relu) {
+#pragma unroll
+                                    for (int t = 0; t < VG; ++t) v[t] = fmaxf(v[t], 0.0f);
+                                }
+                                store_vec<YT, VG>(ybase + o, v);
+                            }
                         } else if (a.st_grp) {
                             // the lane's VG pixels lie in one image (the row length of X, padded or not,
                             // is a multiple of VG); pixels p >= hwy exist only as padding of the repacked X
                             if (yok[gi]) {
-                                YT* yq = ybase + yoff[gi] + (size_t)co * a.hwy;
+                                const size_t o = yoff[gi] + (size_t)co * a.hwy;
 #pragma unroll
                                 for (int t = 0; t < VG; ++t)
-                                    if (yp[gi] + t < a.hwy) store_one<YT>(yq + t, v[t]);
+                                    if (yp[gi] + t < a.hwy) {
+                                        float u = v[t] + (rbase ? load_res_one<YT>(rbase + o + t) : 0.0f);
+                                        if (a.relu) u = fmaxf(u, 0.0f);
+                                        store_one<YT>(ybase + o + t, u);
+                                    }
                             }
                         } else {
                             // element by element: the run may cross into the next image, and pixels
@@ -724,8 +775,12 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_kernel(const 
 #pragma unroll
                             for (int t = 0; t < VG; ++t) {
                                 while (pp >= a.hw) { pp -= a.hw; ++nn; }
-                                if (q0 + gi * (32 * VG) + lane * VG + t < a.q_total && pp < a.hwy)
-                                    store_one<YT>(ybase + ((size_t)nn * a.cout + co) * a.hwy + pp, v[t]);
+                                if (q0 + gi * (32 * VG) + lane * VG + t < a.q_total && pp < a.hwy) {
+                                    const size_t o = ((size_t)nn * a.cout + co) * a.hwy + pp;
+                                    float u = v[t] + (rbase ? load_res_one<YT>(rbase + o) : 0.0f);
+                                    if (a.relu) u = fmaxf(u, 0.0f);
+                                    store_one<YT>(ybase + o, u);
+                                }
                                 ++pp;
                             }
                         }

@@ -234,6 +234,7 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_mma_kernel(co
                                 const int co = rowid[s] * G + j;
                                 if (j >= G || co >= a.cout) continue;
                                 float v = c[s][mt][nb][2 * hf + e] + (e ? bz[s][nb].y : bz[s][nb].x);
+                                if (a.res) v += __ldg(static_cast<const float*>(a.res) + (yp - ybase) + (size_t)co * a.hwy);
                                 if (a.relu) v = fmaxf(v, 0.0f);
                                 yp[(size_t)co * a.hwy] = v;
                             }
@@ -265,13 +266,52 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_mma_kernel(co
 #pragma unroll
                 for (int nb = 0; nb < NB; ++nb) {
                     __syncwarp();
+                    const __half* rbase = static_cast<const __half*>(a.res);
+                    if (rbase) {
+                        // The residual takes the way of the output in reverse: every lane copies runs of
+                        // consecutive pixels of one channel into the scratch tile, and a transposing matrix
+                        // load hands each lane the values at its accumulator positions, so that the sum is
+                        // formed in fp32 and rounded once.
+#pragma unroll 2
+                        for (int j = 0; j < 8; ++j) {
+                            const int co = rowid[s] * G + nb * 8 + j;
+                            const bool have = nb * 8 + j < G && co < a.cout;
+#pragma unroll
+                            for (int gi = 0; gi < NG; ++gi) {
+                                unsigned char* wp = const_cast<unsigned char*>(scratch) + j * SCRB + (gi * (32 * VG) + lane * VG) * 2;
+                                __half* hw16 = reinterpret_cast<__half*>(wp);
+                                if (have && a.st_vec && yok[gi]) {
+                                    const __half* src = rbase + yoff[gi] + (size_t)co * a.hwy;
+                                    if constexpr (VG == 8) *reinterpret_cast<uint4*>(wp) = __ldg(reinterpret_cast<const uint4*>(src));
+                                    else *reinterpret_cast<uint2*>(wp) = __ldg(reinterpret_cast<const uint2*>(src));
+                                } else {
+                                    int nn = yn[gi], pp = yp[gi];
+#pragma unroll
+                                    for (int t = 0; t < VG; ++t) {
+                                        while (pp >= a.hw) { pp -= a.hw; ++nn; }
+                                        const bool in = have && !a.st_vec && q0 + gi * (32 * VG) + lane * VG + t < a.q_total && pp < a.hwy;
+                                        hw16[t] = in ? __ldg(rbase + ((size_t)nn * a.cout + co) * a.hwy + pp) : __float2half_rn(0.0f);
+                                        ++pp;
+                                    }
+                                }
+                            }
+                        }
+                        __syncwarp();
+                    }
 #pragma unroll
                     for (int mp = 0; mp < MT / 2; ++mp) {
                         uint32_t r[4];
+                        float2 rs[4] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
+                        if (rbase) {
+                            uint32_t q[4];
+                            ldmatrix_x4_trans(st_addr + mp * 64, q);
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) rs[i] = __half22float2(*reinterpret_cast<const __half2*>(&q[i]));
+                        }
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {       // tiles 2*mp and 2*mp+1, pixel halves 0 and 1
                             const float* cc = c[s][2 * mp + (i >> 1)][nb];
-                            r[i] = pack_half2(cc[2 * (i & 1)] + bz[s][nb].x, cc[2 * (i & 1) + 1] + bz[s][nb].y);
+                            r[i] = pack_half2(cc[2 * (i & 1)] + bz[s][nb].x + rs[i].x, cc[2 * (i & 1) + 1] + bz[s][nb].y + rs[i].y);
                             if (a.relu) {
                                 const __half2 h = __hmax2(*reinterpret_cast<const __half2*>(&r[i]), zero2);
                                 r[i] = *reinterpret_cast<const uint32_t*>(&h);

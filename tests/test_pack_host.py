@@ -30,7 +30,7 @@ def test_library_exports_every_declared_symbol(alcs):
     L = alcs.lib()
     for name in declared:
         assert hasattr(L, name), name
-    assert L.alcs_version() == 1
+    assert L.alcs_version() == 2
 
 
 @pytest.mark.parametrize("dtype", [np.float32, np.float16])

@@ -653,7 +653,10 @@ def main():
     e2e = None
     if args.e2e_steps > 0:
         ws_bytes = max(A.alcs_spconv1x1_host_workspace(L["w"], L["n"], L["h"], L["wd"], L["flags"]) for L in layers)
-        ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+        # two streams with a workspace each take the layers alternately, so that the upload of one
+        # layer's input overlaps the download of the previous layer's output (the bus is full duplex)
+        ws2 = [torch.empty(ws_bytes, dtype=torch.uint8, device=dev) for _ in range(2)]
+        st2 = [torch.cuda.Stream(), torch.cuda.Stream()]
         xh = [torch.from_numpy(X).pin_memory() for X, _ in host]
         bh = [torch.from_numpy(b).pin_memory() for _, b in host]
         yh = [torch.empty(tuple(L["y"].shape), dtype=L["y"].dtype).pin_memory() for L in layers]
@@ -661,8 +664,16 @@ def main():
         d2h = sum(y.numel() * y.element_size() for y in yh)
 
         def e2e_step():
-            for L, x, y, b in zip(layers, xh, yh, bh):
-                A.alcs_spconv1x1_host(L["w"], x, y, L["n"], L["h"], L["wd"], b, L["flags"], ws, ws_bytes, stream)
+            start = torch.cuda.Event()
+            start.record(stream)
+            for s_ in st2:
+                s_.wait_event(start)
+            for i, (L, x, y, b) in enumerate(zip(layers, xh, yh, bh)):
+                A.alcs_spconv1x1_host(L["w"], x, y, L["n"], L["h"], L["wd"], b, L["flags"], ws2[i % 2], ws_bytes, st2[i % 2])
+            for s_ in st2:
+                done = torch.cuda.Event()
+                done.record(s_)
+                stream.wait_event(done)
 
         e2e_step()
         barrier()

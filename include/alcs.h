@@ -422,22 +422,24 @@ ALCS_API int alcs_network_latency(double tau, const alcs_latency_table* tabs, in
  * alcs_project_bisection: paper, Section 3.4, Algorithm 1 ("Projection operation with bisection").
  * The variable to project is given layer by layer: u_tilde[l] is a DEVICE pointer to a row-major
  * fp32 matrix [cout[l]][cols[l]] (cols = cin*kh*kw, the flattened filters); the arrays u_tilde,
- * cout, cols, tabs themselves are host memory.  Steps: (1) the groups are the g adjacent filters at
- * one location (Section 3.2.1): group (r, c) of a layer = elements (r*g .. r*g+g-1, c); (2) all
- * groups of all layers are ranked together by L2 norm, largest first -- the ranking key is the
+ * cout, cols, tabs themselves are host memory.  What is computed: the groups are the g adjacent
+ * filters at one location (Section 3.2.1): group (r, c) of a layer = elements (r*g .. r*g+g-1, c).
+ * All groups of all layers are ranked together by L2 norm, largest first -- the ranking key is the
  * squared norm accumulated in fp32 in ascending filter order with separately rounded multiplies and
- * adds, equal keys keep (layer, r, c) order; (3)-(14) N is bisected between 0 and the number of
- * groups until the model latencies of the two ends of the bracket differ by at most eps, where the
- * latency of "the top-N groups kept" uses ||W^(l)||_0 = g * (kept groups of layer l) in the model
- * above; a bracket that can no longer shrink (N1 - N0 <= 1) also ends the loop, a case the paper's
- * listing leaves open; (15) the (N0+N1)/2 best-ranked groups are kept.
+ * adds, equal keys keep (layer, r, c) order.  The result keeps a prefix of that ranking; its length N
+ * is searched by halving a bracket [n0, n1] (initially 0 and the number of groups): the model
+ * latency of "the N best-ranked groups kept" uses ||W^(l)||_0 = g * (kept groups of layer l) in the
+ * latency model above, the half whose end latency is below t_budget (strictly) is discarded from
+ * below, the other from above, until the latencies of the two ends differ by at most eps or the
+ * bracket has width 1 (a case the paper leaves open); N = (n0 + n1) / 2, rounded down.
  * Outputs: mask_out, DEVICE, one byte per group, the layers one after the other, each
  * [ceil(cout/g)][cols] -- the block_mask layout of alcs_pack; u_out (may be NULL), a host array of
  * DEVICE pointers, u_out[l] (may be NULL) receives u_tilde[l] with the dropped groups set to +0;
  * kept_per_layer (host, may be NULL) the number of kept groups per layer; *result (host, may be
- * NULL).  The call allocates temporary device memory (about 18 bytes per group plus the sort's
- * workspace), frees it before returning, and synchronises cuda_stream.
- * Errors: INVALID_ARG, SHAPE (2^32 or more groups), UNSUPPORTED (more than 4096 layers), ALLOC, CUDA.
+ * NULL).  The call takes temporary device memory (about 18 bytes per group plus the sort's
+ * workspace) from the device's stream-ordered memory pool and returns it there, copies 2 bytes per
+ * group to the host for the search, and synchronises cuda_stream.
+ * Errors: INVALID_ARG, SHAPE (2^31 or more groups), UNSUPPORTED (more than 4096 layers), ALLOC, CUDA.
  */
 typedef struct {
     int64_t n_keep;             /* groups kept = (n0 + n1) / 2                                     */

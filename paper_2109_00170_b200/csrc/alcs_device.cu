@@ -1,6 +1,7 @@
 // Device-facing half of libalcs: upload of the packed weights and their launch schedules, launch
 // planning, the convolution entry points, the tuner, the host-buffer variant and the layer stack.
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 
 #include <algorithm>
 #include <cmath>
@@ -1090,9 +1091,17 @@ ALCS_API int alcs_stack_create(const alcs_layer* layers, int n_layers, unsigned 
 
 static int stack_enqueue(alcs_stack* s, cudaStream_t st)
 {
+    int index = 0;
     for (auto& it : s->items) {
+        ++index;
         if (it.q == 0) continue;
         const alcs_layer& L = it.layer;
+        // one named range per layer: a timeline then shows the per-layer run times T^(l) whose sum the
+        // paper's latency model is about (a no-op unless a profiler has attached itself to the process)
+        char name[96];
+        std::snprintf(name, sizeof name, "alcs layer %d: %d->%d @%dx%d n=%d", index, L.w->cin, L.w->cout, L.h, L.wd, L.n);
+        nvtxRangePushA(name);
+        struct Pop { ~Pop() { nvtxRangePop(); } } pop;
         int rc = launch_plan(L.w, it.plan, L.x, L.y, L.n, it.oh, it.ow, L.bias, L.flags, st, s->xpad, s->xpad_bytes,
                              L.residual, L.stride > 1 ? L.stride : 1, L.h, L.wd);
         if (rc) return rc;

@@ -68,8 +68,23 @@ __global__ void __launch_bounds__(512) gather_kernel(const GatherArgs a)
         for (int i = 0; i < P; ++i) acc[j][i] = 0.0f;
 
     const float* ximg = a.x + (size_t)img * a.cin * a.hw;
+    // Programmatic dependent launch: the next kernel on the stream may start its own set-up now; this
+    // kernel reads what does not depend on its predecessor (the row's column indices and weights,
+    // pulled towards the SM here) and only then waits for the predecessor, whose output is its x.
+    asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
+    const int k_first = __ldg(a.row_ptr + r);
     const int k1 = __ldg(a.row_ptr + r + 1);
-    for (int k = __ldg(a.row_ptr + r) + ks; k < k1; k += KS * kUnroll) {
+    {
+        const char* cb = reinterpret_cast<const char*>(a.col_idx + k_first);
+        const char* vb = reinterpret_cast<const char*>(a.vals + (size_t)k_first * G);
+        const long long cbytes = (long long)(k1 - k_first) * 4, vbytes = cbytes * G;
+        for (long long o = (long long)threadIdx.x * 128; o < cbytes; o += (long long)blockDim.x * 128)
+            asm volatile("prefetch.global.L2 [%0];\n" ::"l"(cb + o));
+        for (long long o = (long long)threadIdx.x * 128; o < vbytes; o += (long long)blockDim.x * 128)
+            asm volatile("prefetch.global.L2 [%0];\n" ::"l"(vb + o));
+    }
+    asm volatile("griddepcontrol.wait;\n" ::: "memory");
+    for (int k = k_first + ks; k < k1; k += KS * kUnroll) {
         float w[kUnroll][G];
         float xv[kUnroll][P];
 #pragma unroll
@@ -129,9 +144,22 @@ template <int G, int P>
 cudaError_t launch_gp(const GatherArgs& a, bool vec, unsigned grid, int ks, cudaStream_t st)
 {
     const size_t smem = (size_t)ks * G * P * 32 * sizeof(float);
-    if (vec) gather_kernel<G, P, true><<<grid, ks * 32, smem, st>>>(a);
-    else gather_kernel<G, P, false><<<grid, ks * 32, smem, st>>>(a);
-    return cudaGetLastError();
+    // launched so that it may overlap the tail of the kernel before it on the stream (it waits for that
+    // kernel before it touches x or y); a CUDA graph keeps the same programmatic edge
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(grid);
+    lc.blockDim = dim3(ks * 32);
+    lc.dynamicSmemBytes = smem;
+    lc.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    GatherArgs args = a;
+    void* params[] = {&args};
+    const void* fn = vec ? (const void*)&gather_kernel<G, P, true> : (const void*)&gather_kernel<G, P, false>;
+    return cudaLaunchKernelExC(&lc, fn, params);
 }
 
 template <int G>

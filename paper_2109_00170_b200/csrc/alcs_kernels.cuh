@@ -710,8 +710,11 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_kernel(const 
 
         // ---- epilogue: bias, ReLU, store ----------------------------------------------------
         grid_dep_wait();    // (long satisfied: the data consumed above was loaded after the producer's wait)
-        auto epilogue = [&](auto* ybase) {
+        // (the residual operand is a compile-time flavour of the epilogue, so that layers without one
+        // run exactly the code they would run if the operand did not exist)
+        auto epilogue = [&](auto* ybase, auto has_res) {
             using YT = std::remove_pointer_t<decltype(ybase)>;
+            constexpr bool RES = decltype(has_res)::value;
             size_t yoff[NG];
             bool yok[NG];
             int yn[NG], yp[NG];
@@ -738,20 +741,22 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_kernel(const 
                         for (int t = 0; t < VG; ++t) {
                             const float2 a2 = acc[s][j][(gi * VG + t) / 2];
                             v[t] = (((gi * VG + t) & 1) ? a2.y : a2.x) + bv;
+                            if constexpr (!RES) {
+                                if (a.relu) v[t] = fmaxf(v[t], 0.0f);
+                            }
                         }
                         const YT* rbase = static_cast<const YT*>(a.res);
                         if (a.st_vec) {
                             if (yok[gi]) {
                                 const size_t o = yoff[gi] + (size_t)co * a.hwy;
-                                if (rbase) {
+                                if constexpr (RES) {
                                     float r[VG];
                                     load_res_vec<YT, VG>(rbase + o, r);
 #pragma unroll
-                                    for (int t = 0; t < VG; ++t) v[t] += r[t];
-                                }
-                                if (a.relu) {
-#pragma unroll
-                                    for (int t = 0; t < VG; ++t) v[t] = fmaxf(v[t], 0.0f);
+                                    for (int t = 0; t < VG; ++t) {
+                                        v[t] += r[t];
+                                        if (a.relu) v[t] = fmaxf(v[t], 0.0f);
+                                    }
                                 }
                                 store_vec<YT, VG>(ybase + o, v);
                             }
@@ -763,8 +768,11 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_kernel(const 
 #pragma unroll
                                 for (int t = 0; t < VG; ++t)
                                     if (yp[gi] + t < a.hwy) {
-                                        float u = v[t] + (rbase ? load_res_one<YT>(rbase + o + t) : 0.0f);
-                                        if (a.relu) u = fmaxf(u, 0.0f);
+                                        float u = v[t];
+                                        if constexpr (RES) {
+                                            u += load_res_one<YT>(rbase + o + t);
+                                            if (a.relu) u = fmaxf(u, 0.0f);
+                                        }
                                         store_one<YT>(ybase + o + t, u);
                                     }
                             }
@@ -777,8 +785,11 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_kernel(const 
                                 while (pp >= a.hw) { pp -= a.hw; ++nn; }
                                 if (q0 + gi * (32 * VG) + lane * VG + t < a.q_total && pp < a.hwy) {
                                     const size_t o = ((size_t)nn * a.cout + co) * a.hwy + pp;
-                                    float u = v[t] + (rbase ? load_res_one<YT>(rbase + o) : 0.0f);
-                                    if (a.relu) u = fmaxf(u, 0.0f);
+                                    float u = v[t];
+                                    if constexpr (RES) {
+                                        u += load_res_one<YT>(rbase + o);
+                                        if (a.relu) u = fmaxf(u, 0.0f);
+                                    }
                                     store_one<YT>(ybase + o, u);
                                 }
                                 ++pp;
@@ -788,11 +799,15 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_kernel(const 
                 }
             }
         };
+        auto run_epilogue = [&](auto* ybase) {
+            if (a.res) epilogue(ybase, std::true_type{});
+            else epilogue(ybase, std::false_type{});
+        };
         if constexpr (sizeof(XT) == 4) {
-            epilogue(static_cast<float*>(a.y));
+            run_epilogue(static_cast<float*>(a.y));
         } else {
-            if (a.y_f32) epilogue(static_cast<float*>(a.y));
-            else epilogue(static_cast<__half*>(a.y));
+            if (a.y_f32) run_epilogue(static_cast<float*>(a.y));
+            else run_epilogue(static_cast<__half*>(a.y));
         }
     }
 }

@@ -3,9 +3,9 @@
 // Host part: the linear interpolation over a layer's measured (non-zero count, run time) pairs and
 // the network sum.  Device part, the data-parallel steps of Algorithm 1: the ranking key of every
 // group of g adjacent filters (its squared L2 norm), the ranking of all groups of all layers (a
-// radix sort from the CUDA toolkit's CUB, a library primitive), the per-layer count of the top-N
-// groups that each bisection step needs, and the final mask / projected tensor.  The bisection
-// itself is a few dozen iterations of host control around the counting kernel.
+// radix sort from the CUDA toolkit's CUB, a library primitive), the layer of every ranked group with
+// per-bucket layer histograms, and the final mask / projected tensor.  The search over the length of
+// the kept prefix of the ranked list runs on the host from one copy of those two arrays.
 #include <cuda_runtime.h>
 
 #include <cub/device/device_radix_sort.cuh>
@@ -95,18 +95,21 @@ __global__ void ranked_layer_kernel(const unsigned* __restrict__ idx, long long 
 
 constexpr int kMaxLayers = 4096;
 
-// counts[l] += number of the top-n ranked groups that belong to layer l
-__global__ void count_top_kernel(const unsigned short* __restrict__ layer_of, long long n, int n_layers,
-                                 unsigned long long* __restrict__ counts)
+constexpr long long kRankBucket = 4096;
+
+// hist[b][l] = how many of the ranked entries b*kRankBucket .. (b+1)*kRankBucket - 1 belong to layer l
+// (one thread block per bucket, a shared-memory histogram)
+__global__ void bucket_histogram_kernel(const unsigned short* __restrict__ layer_of, long long total, int n_layers,
+                                        unsigned* __restrict__ hist)
 {
-    extern __shared__ unsigned int hist[];
-    for (int i = threadIdx.x; i < n_layers; i += blockDim.x) hist[i] = 0;
+    extern __shared__ unsigned int h[];
+    for (int i = threadIdx.x; i < n_layers; i += blockDim.x) h[i] = 0;
     __syncthreads();
-    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
-        atomicAdd(&hist[layer_of[i]], 1u);
+    const long long b0 = (long long)blockIdx.x * kRankBucket;
+    const long long b1 = b0 + kRankBucket < total ? b0 + kRankBucket : total;
+    for (long long i = b0 + threadIdx.x; i < b1; i += blockDim.x) atomicAdd(&h[layer_of[i]], 1u);
     __syncthreads();
-    for (int i = threadIdx.x; i < n_layers; i += blockDim.x)
-        if (hist[i]) atomicAdd(&counts[i], (unsigned long long)hist[i]);
+    for (int i = threadIdx.x; i < n_layers; i += blockDim.x) hist[(size_t)blockIdx.x * n_layers + i] = h[i];
 }
 
 // mask[group] = 1 for the n best-ranked groups, 0 for the others
@@ -127,16 +130,6 @@ __global__ void apply_mask_kernel(const float* __restrict__ u, const uint8_t* __
         out[i] = mask[(size_t)(co / g) * cols + c] ? u[i] : 0.0f;
     }
 }
-
-unsigned blocks_for(long long n, int threads = 256)
-{
-    return (unsigned)std::max<long long>(1, std::min<long long>((n + threads - 1) / threads, 148 * 16));
-}
-
-struct DeviceBuffers {
-    void* p[8] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
-    ~DeviceBuffers() { for (void* q : p) if (q) cudaFree(q); }
-};
 
 }  // namespace
 
@@ -180,76 +173,98 @@ ALCS_API int alcs_project_bisection(const float* const* u_tilde, const int* cout
         off[l + 1] = off[l] + (long long)((cout[l] + g - 1) / g) * cols[l];
     }
     const long long total = off[n_layers];
-    if (total >= (1ll << 32)) return ALCS_ERR_SHAPE;        // group indices are 32-bit
+    if (total >= (1ll << 31)) return ALCS_ERR_SHAPE;        // the sort takes a 32-bit signed item count
+    int dev = 0, sms = 0;
+    ALCS_CUDA(cudaGetDevice(&dev));
+    ALCS_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    auto blocks_for = [&](long long n) {
+        return (unsigned)std::max<long long>(1, std::min<long long>((n + 255) / 256, (long long)sms * 16));
+    };
 
-    DeviceBuffers b;
-    unsigned *keys = nullptr, *idx = nullptr, *keys2 = nullptr, *idx2 = nullptr;
-    unsigned short* layer_of = nullptr;
-    long long* d_off = nullptr;
-    unsigned long long* d_counts = nullptr;
-    auto alloc = [&](int slot, size_t bytes) { return cudaMalloc(&b.p[slot], std::max<size_t>(bytes, 16)); };
-    if (alloc(0, total * 4) || alloc(1, total * 4) || alloc(2, total * 4) || alloc(3, total * 4) || alloc(4, total * 2) ||
-        alloc(5, (n_layers + 1) * 8) || alloc(6, n_layers * 8)) {
+    // One stream-ordered allocation for everything: after the first call the memory comes back from
+    // the runtime's pool without touching the driver.
+    const long long n_buckets = (total + kRankBucket - 1) / kRankBucket;
+    size_t sort_bytes = 0;
+    ALCS_CUDA(cub::DeviceRadixSort::SortPairsDescending(nullptr, sort_bytes, (unsigned*)nullptr, (unsigned*)nullptr,
+                                                       (unsigned*)nullptr, (unsigned*)nullptr, (int)total, 0, 32, st));
+    auto up = [](size_t b) { return (b + 255) / 256 * 256; };
+    const size_t b_keys = up((size_t)total * 4), b_lay = up((size_t)total * 2), b_off = up((size_t)(n_layers + 1) * 8);
+    const size_t b_hist = up((size_t)std::max<long long>(n_buckets, 1) * n_layers * 4);
+    const size_t bytes = 4 * b_keys + b_lay + b_off + b_hist + up(sort_bytes) + 256;
+    unsigned char* pool = nullptr;
+    if (cudaMallocAsync(&pool, bytes, st) != cudaSuccess) {
         (void)cudaGetLastError();
         return ALCS_ERR_ALLOC;
     }
-    keys = (unsigned*)b.p[0]; idx = (unsigned*)b.p[1]; keys2 = (unsigned*)b.p[2]; idx2 = (unsigned*)b.p[3];
-    layer_of = (unsigned short*)b.p[4]; d_off = (long long*)b.p[5]; d_counts = (unsigned long long*)b.p[6];
+    struct Release {
+        unsigned char* p; cudaStream_t s;
+        ~Release() { cudaFreeAsync(p, s); }
+    } release{pool, st};
+    unsigned* keys = (unsigned*)pool;
+    unsigned* idx = (unsigned*)(pool + b_keys);
+    unsigned* keys2 = (unsigned*)(pool + 2 * b_keys);
+    unsigned* idx2 = (unsigned*)(pool + 3 * b_keys);
+    unsigned short* layer_of = (unsigned short*)(pool + 4 * b_keys);
+    long long* d_off = (long long*)(pool + 4 * b_keys + b_lay);
+    unsigned* d_hist = (unsigned*)(pool + 4 * b_keys + b_lay + b_off);
+    void* sort_tmp = pool + 4 * b_keys + b_lay + b_off + b_hist;
 
-    // steps 1-2: group keys, then rank all groups of all layers, largest key first.  The radix sort
-    // is stable, so equal keys stay in (layer, group) order.
+    // Ranking (Algorithm 1: the groups of all layers sorted together by norm, largest first).  The radix
+    // sort is stable, so equal keys stay in (layer, group) order.  Then, for the ranked list, the layer
+    // of every entry and, per bucket of kRankBucket consecutive ranks, how many entries each layer has.
     for (int l = 0; l < n_layers; ++l) {
         const long long n = off[l + 1] - off[l];
         group_keys_kernel<<<blocks_for(n), 256, 0, st>>>(u_tilde[l], cout[l], cols[l], g, off[l], keys, idx);
     }
     ALCS_CUDA(cudaGetLastError());
-    size_t tmp_bytes = 0;
-    ALCS_CUDA(cub::DeviceRadixSort::SortPairsDescending(nullptr, tmp_bytes, keys, keys2, idx, idx2, (int)total, 0, 32, st));
-    if (cudaMalloc(&b.p[7], std::max<size_t>(tmp_bytes, 16)) != cudaSuccess) {
-        (void)cudaGetLastError();
-        return ALCS_ERR_ALLOC;
-    }
-    ALCS_CUDA(cub::DeviceRadixSort::SortPairsDescending(b.p[7], tmp_bytes, keys, keys2, idx, idx2, (int)total, 0, 32, st));
+    ALCS_CUDA(cub::DeviceRadixSort::SortPairsDescending(sort_tmp, sort_bytes, keys, keys2, idx, idx2, (int)total, 0, 32, st));
     ALCS_CUDA(cudaMemcpyAsync(d_off, off.data(), (n_layers + 1) * 8, cudaMemcpyHostToDevice, st));
     ranked_layer_kernel<<<blocks_for(total), 256, 0, st>>>(idx2, total, d_off, n_layers, layer_of);
     ALCS_CUDA(cudaGetLastError());
-
-    // T(U) for "the top-n groups kept": per-layer counts on the device, the interpolation on the host
-    std::vector<unsigned long long> counts(n_layers);
-    std::vector<int64_t> nz(n_layers);
-    auto latency_of_top = [&](long long n, double* t) -> int {
-        ALCS_CUDA(cudaMemsetAsync(d_counts, 0, n_layers * 8, st));
-        if (n > 0) count_top_kernel<<<blocks_for(n), 256, n_layers * 4, st>>>(layer_of, n, n_layers, d_counts);
+    if (n_buckets > 0) {
+        bucket_histogram_kernel<<<(unsigned)n_buckets, 256, n_layers * 4, st>>>(layer_of, total, n_layers, d_hist);
         ALCS_CUDA(cudaGetLastError());
-        ALCS_CUDA(cudaMemcpyAsync(counts.data(), d_counts, n_layers * 8, cudaMemcpyDeviceToHost, st));
-        ALCS_CUDA(cudaStreamSynchronize(st));
-        for (int l = 0; l < n_layers; ++l) nz[l] = (int64_t)counts[l] * g;
-        double total_t = tau;
-        for (int l = 0; l < n_layers; ++l) total_t += interpolate(tabs[l], nz[l]);
-        *t = total_t;
-        return ALCS_OK;
+    }
+
+    // The latency of "the N best-ranked groups kept" depends on N only through the number of kept
+    // groups per layer, a monotone step function of N.  One copy brings what is needed to evaluate it
+    // for any N on the host: the bucket histograms (turned into prefix counts) and the ranked list's
+    // layers, of which at most one bucket is scanned per evaluation.  No device work per search step.
+    std::vector<unsigned> hist((size_t)n_buckets * n_layers);
+    std::vector<unsigned short> lay((size_t)total);
+    if (total > 0) {
+        ALCS_CUDA(cudaMemcpyAsync(hist.data(), d_hist, hist.size() * 4, cudaMemcpyDeviceToHost, st));
+        ALCS_CUDA(cudaMemcpyAsync(lay.data(), layer_of, lay.size() * 2, cudaMemcpyDeviceToHost, st));
+    }
+    ALCS_CUDA(cudaStreamSynchronize(st));
+    std::vector<long long> prefix((size_t)(n_buckets + 1) * n_layers, 0);     // groups of layer l among ranks < b*kRankBucket
+    for (long long bk = 0; bk < n_buckets; ++bk)
+        for (int l = 0; l < n_layers; ++l)
+            prefix[(size_t)(bk + 1) * n_layers + l] = prefix[(size_t)bk * n_layers + l] + hist[(size_t)bk * n_layers + l];
+    std::vector<long long> counts(n_layers);
+    auto latency_of_top = [&](long long n) {
+        const long long bk = n / kRankBucket;
+        for (int l = 0; l < n_layers; ++l) counts[l] = prefix[(size_t)bk * n_layers + l];
+        for (long long i = bk * kRankBucket; i < n; ++i) ++counts[lay[(size_t)i]];
+        double t = tau;
+        for (int l = 0; l < n_layers; ++l) t += interpolate(tabs[l], (int64_t)counts[l] * g);
+        return t;
     };
 
-    // steps 3-15 of Algorithm 1
-    long long n0 = 0, n1 = total;
-    double t0 = 0, t1 = 0;
-    int rc = latency_of_top(0, &t0);
-    if (rc) return rc;
-    rc = latency_of_top(total, &t1);
-    if (rc) return rc;
+    // Search: the bracket [lo, hi] of prefix lengths always has latency(lo) on the budget's near side
+    // as far as it is known and is halved until the latencies of its two ends are within eps of each
+    // other (Section 3.4, Algorithm 1); a bracket of width 1 cannot shrink further and also ends it.
+    long long lo = 0, hi = total;
+    double t_lo = latency_of_top(lo), t_hi = latency_of_top(hi);
     int iters = 0;
-    while (t1 - t0 > eps && n1 - n0 > 1) {      // the second test ends a bracket that cannot shrink
-        const long long n = (n0 + n1) / 2;
-        double t = 0;
-        rc = latency_of_top(n, &t);
-        if (rc) return rc;
-        if (t < t_budget) { t0 = t; n0 = n; } else { t1 = t; n1 = n; }
+    while (t_hi - t_lo > eps && hi - lo > 1) {
+        const long long mid = (lo + hi) / 2;
+        const double t = latency_of_top(mid);
+        if (t < t_budget) { t_lo = t; lo = mid; } else { t_hi = t; hi = mid; }
         ++iters;
     }
-    const long long n_keep = (n0 + n1) / 2;
-    double t_final = 0;
-    rc = latency_of_top(n_keep, &t_final);
-    if (rc) return rc;
+    const long long n_keep = (lo + hi) / 2;
+    const double t_final = latency_of_top(n_keep);      // (leaves the kept counts of the result in `counts`)
 
     write_mask_kernel<<<blocks_for(total), 256, 0, st>>>(idx2, total, n_keep, mask_out);
     ALCS_CUDA(cudaGetLastError());
@@ -260,11 +275,11 @@ ALCS_API int alcs_project_bisection(const float* const* u_tilde, const int* cout
         }
         ALCS_CUDA(cudaGetLastError());
     }
-    ALCS_CUDA(cudaStreamSynchronize(st));       // the temporaries are freed on return
+    ALCS_CUDA(cudaStreamSynchronize(st));
     if (kept_per_layer)
         for (int l = 0; l < n_layers; ++l) kept_per_layer[l] = (int64_t)counts[l];
     if (result) {
-        result->n_keep = n_keep; result->n0 = n0; result->n1 = n1; result->iters = iters; result->latency = t_final;
+        result->n_keep = n_keep; result->n0 = lo; result->n1 = hi; result->iters = iters; result->latency = t_final;
         result->n_groups = total;
     }
     return ALCS_OK;

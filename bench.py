@@ -377,9 +377,11 @@ def bench_latency_model(args):
     total = sum(s.rows * s.cin for s in specs)
     mask_d = torch.empty((total,), dtype=torch.uint8, device=dev)
     A.alcs_project_bisection(ud, specs[0].g, tables, 0.0, budget, eps, mask_d, None, stream)      # warm-up
-    c0 = time.perf_counter()
-    pr = A.alcs_project_bisection(ud, specs[0].g, tables, 0.0, budget, eps, mask_d, None, stream)
-    proj_ms = (time.perf_counter() - c0) * 1e3
+    proj_ms = 1e30
+    for _ in range(5):              # host wall clock of the whole call (it synchronises); best of five
+        c0 = time.perf_counter()
+        pr = A.alcs_project_bisection(ud, specs[0].g, tables, 0.0, budget, eps, mask_d, None, stream)
+        proj_ms = min(proj_ms, (time.perf_counter() - c0) * 1e3)
     mask_h = mask_d.cpu().numpy()
     real, off = 0.0, 0
     for i, s in enumerate(specs):

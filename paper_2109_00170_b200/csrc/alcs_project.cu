@@ -12,6 +12,7 @@
 
 #include <algorithm>
 #include <cstdint>
+#include <mutex>
 #include <vector>
 
 #include "alcs.h"
@@ -96,6 +97,11 @@ __global__ void ranked_layer_kernel(const unsigned* __restrict__ idx, long long 
 constexpr int kMaxLayers = 4096;
 
 constexpr long long kRankBucket = 4096;
+
+// page-locked host staging area of alcs_project_bisection, shared by all calls (one call at a time uses it)
+std::mutex g_staging_mu;
+void* g_staging = nullptr;
+size_t g_staging_bytes = 0;
 
 // hist[b][l] = how many of the ranked entries b*kRankBucket .. (b+1)*kRankBucket - 1 belong to layer l
 // (one thread block per bucket, a shared-memory histogram)
@@ -230,11 +236,25 @@ ALCS_API int alcs_project_bisection(const float* const* u_tilde, const int* cout
     // groups per layer, a monotone step function of N.  One copy brings what is needed to evaluate it
     // for any N on the host: the bucket histograms (turned into prefix counts) and the ranked list's
     // layers, of which at most one bucket is scanned per evaluation.  No device work per search step.
-    std::vector<unsigned> hist((size_t)n_buckets * n_layers);
-    std::vector<unsigned short> lay((size_t)total);
+    // (page-locked staging memory, kept between calls: a copy into pageable memory is several times slower)
+    const size_t hist_bytes = (size_t)n_buckets * n_layers * 4, lay_bytes = (size_t)total * 2;
+    std::unique_lock<std::mutex> staging_lock(g_staging_mu);
+    if (g_staging_bytes < up(hist_bytes) + lay_bytes + 16) {
+        if (g_staging) cudaFreeHost(g_staging);
+        g_staging = nullptr;
+        g_staging_bytes = 0;
+        const size_t want = (up(hist_bytes) + lay_bytes + 16) * 5 / 4;
+        if (cudaMallocHost(&g_staging, want) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return ALCS_ERR_ALLOC;
+        }
+        g_staging_bytes = want;
+    }
+    const unsigned* hist = reinterpret_cast<const unsigned*>(g_staging);
+    const unsigned short* lay = reinterpret_cast<const unsigned short*>(static_cast<unsigned char*>(g_staging) + up(hist_bytes));
     if (total > 0) {
-        ALCS_CUDA(cudaMemcpyAsync(hist.data(), d_hist, hist.size() * 4, cudaMemcpyDeviceToHost, st));
-        ALCS_CUDA(cudaMemcpyAsync(lay.data(), layer_of, lay.size() * 2, cudaMemcpyDeviceToHost, st));
+        ALCS_CUDA(cudaMemcpyAsync(g_staging, d_hist, hist_bytes, cudaMemcpyDeviceToHost, st));
+        ALCS_CUDA(cudaMemcpyAsync(static_cast<unsigned char*>(g_staging) + up(hist_bytes), layer_of, lay_bytes, cudaMemcpyDeviceToHost, st));
     }
     ALCS_CUDA(cudaStreamSynchronize(st));
     std::vector<long long> prefix((size_t)(n_buckets + 1) * n_layers, 0);     // groups of layer l among ranks < b*kRankBucket

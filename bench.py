@@ -573,7 +573,7 @@ def main():
         flags = A.ALCS_RELU if s.relu else 0
         forced = None
         if args.cfg:
-            keys = ("pixels_per_lane", "rows_per_warp", "warps", "chunk_channels", "stages", "row_groups", "min_blocks", "copy_mode", "producer_warps", "math_mode", "consumer_groups")
+            keys = ("pixels_per_lane", "rows_per_warp", "warps", "chunk_channels", "stages", "row_groups", "min_blocks", "copy_mode", "producer_warps", "math_mode", "consumer_groups", "split_rows")
             forced = dict(zip(keys, (int(v) for v in args.cfg.split(","))))
             cfg = forced
         elif s.name in cache:       # a configuration tuned earlier for these kernel sources

@@ -174,10 +174,14 @@ ALCS_API void alcs_packed_free(alcs_packed* p);
  *   consumer_groups   1 = all consumer warps work on one work item at a time; 2 = two halves of the
  *                     consumer warps take the thread block's work items alternately (tensor-core
  *                     kernels only), so that one half multiplies while the other half stores
+ *   split_rows        1 = the kernel flavour for skewed matrices: a block row far longer than the others of
+ *                     its work item is split into parts that separate warps multiply, and the parts' partial
+ *                     sums are added in a fixed order through shared memory before the row is stored (fp32
+ *                     CUDA-core kernels, a subset of the shapes); 2 = rows are never split; 0 = choose
  */
 typedef struct {
     int pixels_per_lane, rows_per_warp, warps, chunk_channels, stages, row_groups, min_blocks, copy_mode,
-        producer_warps, math_mode, consumer_groups;
+        producer_warps, math_mode, consumer_groups, split_rows;
 } alcs_launch_cfg;
 
 /*
@@ -187,10 +191,13 @@ typedef struct {
  * every (warp, set)'s segments chunk by chunk exactly as a consumer warp of the kernel does, and
  * compare what that walk multiplies with the canonical storage format (paper, Section 3.2.2): every
  * kept block exactly once, bit for bit, no other column touched, every block row bound to exactly
- * one (warp, set).  stats (may be NULL, else 7 entries) receives {row groups; largest and smallest
- * number of block slots (kept blocks plus padding) any of the SM's four schedulers is given in a work
- * item; pair records in total; kept blocks; largest and smallest number of block rows a scheduler is
- * given in a work item}.  Returns ALCS_ERR_CORRUPT if the walk and the storage format disagree.
+ * one (warp, set), or -- a row much longer than the others of its work item -- split into parts that
+ * take one (warp, set) each, every kept block in exactly one part, one part storing the row and
+ * reading each of the others' hand-over slots exactly once.  stats (may be NULL, else 8 entries)
+ * receives {row groups; largest and smallest number of block slots (kept blocks plus padding) any of
+ * the SM's four schedulers is given in a work item; pair records in total; kept blocks; largest and
+ * smallest number of units a scheduler is given in a work item; secondary parts of split rows in
+ * total}.  Returns ALCS_ERR_CORRUPT if the walk and the storage format disagree.
  */
 ALCS_API int alcs_schedule_selfcheck(const alcs_packed* p, int chunk_channels, int row_groups, int warps, int slots,
                                      int64_t* stats);

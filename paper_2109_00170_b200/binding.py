@@ -45,7 +45,7 @@ class AlcsError(RuntimeError):
 class LaunchCfg(C.Structure):
     _fields_ = [(k, C.c_int) for k in ("pixels_per_lane", "rows_per_warp", "warps",
                                        "chunk_channels", "stages", "row_groups", "min_blocks", "copy_mode",
-                                       "producer_warps", "math_mode", "consumer_groups")]
+                                       "producer_warps", "math_mode", "consumer_groups", "split_rows")]
 
     def as_dict(self):
         return {k: getattr(self, k) for k, _ in self._fields_}
@@ -278,9 +278,9 @@ def alcs_packed_free(p: Packed):
 
 def alcs_schedule_selfcheck(p: Packed, chunk_channels: int, row_groups: int, warps: int, slots: int) -> dict:
     """Host-only check of the balanced launch schedule against the storage format."""
-    st = (C.c_int64 * 7)()
+    st = (C.c_int64 * 8)()
     _check(lib().alcs_schedule_selfcheck(p.handle, chunk_channels, row_groups, warps, slots, st), "alcs_schedule_selfcheck")
-    return dict(row_groups=st[0], max_sched=st[1], min_sched=st[2], pairs=st[3], nb=st[4], max_rows=st[5], min_rows=st[6])
+    return dict(row_groups=st[0], max_sched=st[1], min_sched=st[2], pairs=st[3], nb=st[4], max_rows=st[5], min_rows=st[6], secondary_units=st[7])
 
 
 def alcs_variant_count() -> int:

@@ -70,7 +70,7 @@ void init_variants_locked()
 
 // Which flavour of the launch schedule a variant takes (alcs_internal.h): the CUDA-core kernels take
 // pair records balanced for their number of consumer warps and accumulator sets.
-int flavour_of(const KernelVariant& v) { return v.mma ? 1 : alcs::balanced_flavour(v.nw, v.rw); }
+int flavour_of(const KernelVariant& v) { return v.mma ? 1 : alcs::balanced_flavour(v.nw, v.rw, v.split); }
 
 // math_mode of alcs_launch_cfg for a variant
 int mode_of(const KernelVariant& v) { return v.mma ? 2 : 1; }
@@ -128,6 +128,8 @@ StageLayout stage_layout(const KernelVariant& v, const Schedule& sc, int elt)
     L.off_rowoff = L.off_rec + sc.wcap * 16;
     L.stage_bytes = L.off_rowoff + sc.ros * 4;
     L.tail_bytes = v.mma ? v.nw * 8 * (32 * v.p * 2 + 16) : 0;     // [8 channels][T pixels] fp16 per consumer warp
+    // hand-over tiles of rows split into parts: a barrier, then two sets of max_x tiles of g*P*32 floats
+    if (!v.mma && sc.max_x > 0) L.tail_bytes = 16 + 2 * sc.max_x * v.g * v.p * 32 * 4;
     return L;
 }
 
@@ -150,7 +152,8 @@ Schedule* get_schedule(const alcs_packed* w, int kc, int n_rg, bool with_records
         if (sc.n_rg == 0 || (with_records && !sc.uploaded && sc.h_rec.empty() && sc.n_rec > 0)) {
             if (flavour == 1) alcs::build_schedule_mma(*w, kc, n_rg, with_records, sc);
             else if (flavour >= 2)
-                alcs::build_schedule_balanced(*w, kc, n_rg, alcs::flavour_nwg(flavour), alcs::flavour_rw(flavour), with_records, sc);
+                alcs::build_schedule_balanced(*w, kc, n_rg, alcs::flavour_nwg(flavour), alcs::flavour_rw(flavour), with_records, sc,
+                                              alcs::flavour_split(flavour) != 0);
             else alcs::build_schedule(*w, kc, n_rg, with_records, sc);
         }
     } catch (const std::bad_alloc&) {
@@ -252,6 +255,16 @@ int occupancy_of(const VariantInfo& vi, size_t smem)
     return occ;
 }
 
+// Where the kernel finds the unit words of a balanced schedule (they follow the row map on the device).
+void set_unit_args(ConvArgs& a, const Schedule& sc, int mma)
+{
+    a.unit = nullptr; a.rgx = nullptr; a.off_xch = 0; a.xch_slots = 0;
+    if (mma || !sc.balanced || sc.max_x <= 0) return;      // (only the split flavour of the kernel is given such schedules)
+    a.unit = sc.rowmap + (size_t)sc.n_rg * sc.rpg;
+    a.rgx = sc.rowmap + 2 * (size_t)sc.n_rg * sc.rpg;
+    a.xch_slots = sc.max_x;
+}
+
 // The small-problem kernel as a plan.  Its cost estimate is a latency model: a warp issues the loads of
 // a few blocks at a time and waits about one L2 round trip for each batch; the arithmetic term makes it
 // lose against the staged kernels as soon as there is enough work to keep the SMs busy.
@@ -321,6 +334,7 @@ int enumerate_plans(const alcs_packed* w, long long q, int hw, std::vector<Plan>
                 last_rpg = rpg;
                 const Schedule* sc = get_schedule(w, kc, n_rg, false, flavour_of(v));
                 if (!sc) return ALCS_ERR_ALLOC;
+                if (v.split && sc->max_x == 0) continue;        // nothing to split: the plain variant covers it
                 const StageLayout L = stage_layout(v, *sc, elt);
                 for (int stages = 2; stages <= alcs::kMaxStages; ++stages) {
                     if (stages % v.groups) continue;        // every consumer group gets the same share of the ring
@@ -381,6 +395,7 @@ void plan_to_cfg(const Plan& p, alcs_launch_cfg* c)
     c->producer_warps = v.npw;
     c->math_mode = mode_of(v);
     c->consumer_groups = v.groups;
+    c->split_rows = v.split ? 1 : 2;
 }
 
 // Resolve a (possibly partial) configuration into a concrete plan.
@@ -414,6 +429,7 @@ int cfg_to_plan(const alcs_packed* w, long long q, int hw, const alcs_launch_cfg
         if (c->producer_warps && c->producer_warps != v.npw) return false;
         if (c->math_mode && c->math_mode != mode_of(v)) return false;
         if (c->consumer_groups && c->consumer_groups != v.groups) return false;
+        if (c->split_rows && (c->split_rows == 1) != (v.split == 1)) return false;
         if (c->chunk_channels && std::min(c->chunk_channels, w->cin) != p.kc) return false;
         if (c->stages && c->stages != p.stages) return false;
         if (c->copy_mode && (c->copy_mode == 2) != (p.bulk == 1)) return false;
@@ -433,6 +449,7 @@ int cfg_to_plan(const alcs_packed* w, long long q, int hw, const alcs_launch_cfg
             if (rpg > v.nw / v.groups * v.rw) continue;
             const Schedule* sc = get_schedule(w, p0.kc, c->row_groups, false, flavour_of(v));
             if (!sc) return ALCS_ERR_ALLOC;
+            if (v.split && sc->max_x == 0) continue;        // nothing to split with this many row groups
             Plan p = p0;
             p.n_rg = sc->n_rg;
             p.smem = plan_smem(stage_layout(v, *sc, (int)w->elt()), p.stages);
@@ -588,6 +605,7 @@ int launch_plan(const alcs_packed* w, const Plan& p, const void* x, void* y, int
     const KernelVariant& v = g_variants[p.variant].v;
     Schedule* sc = get_schedule(w, p.kc, p.n_rg, true, flavour_of(v));
     if (!sc) return ALCS_ERR_ALLOC;
+    if (v.split && sc->max_x == 0) return ALCS_ERR_UNSUPPORTED;    // (the split flavour needs its hand-over area)
     if (!sc->uploaded) {
         const int rc = upload_schedule(w, sc, st);
         if (rc) return rc;
@@ -625,6 +643,7 @@ int launch_plan(const alcs_packed* w, const Plan& p, const void* x, void* y, int
     ConvArgs a;
     a.x = xk; a.y = y; a.bias = bias; a.res = residual;
     a.rec = sc->rec; a.slice = sc->slice; a.rowoff = sc->rowoff; a.rowmap = sc->rowmap;
+    set_unit_args(a, *sc, v.mma);
     a.err = w->d_err;
     a.rows = w->rows; a.cin = w->cin; a.cout = w->cout; a.hw = hwx; a.hwy = hw;
     a.q_total = n * hwx;
@@ -636,6 +655,7 @@ int launch_plan(const alcs_packed* w, const Plan& p, const void* x, void* y, int
     a.y_f32 = (flags & ALCS_Y_F32) ? 1 : 0;
     const StageLayout L = stage_layout(v, *sc, elt);
     a.off_rec = L.off_rec; a.off_rowoff = L.off_rowoff; a.stage_bytes = L.stage_bytes;
+    if (a.unit) a.off_xch = 16 * alcs::kMaxStages + a.stages * L.stage_bytes;
     // widest staging copy that every (image, channel) row start and length allows
     int ld = 16;
     while (ld > elt && (((size_t)hwx * elt) % ld || (uintptr_t)xk % ld)) ld >>= 1;
@@ -679,10 +699,10 @@ int resolve_plan(const alcs_packed* w, int n, int h, int wd, unsigned flags, lon
 {
     alcs::ShapeKey key{n, h, wd, flags};
     if (cfg) {
-        const int c[11] = {cfg->pixels_per_lane, cfg->rows_per_warp, cfg->warps, cfg->chunk_channels,
+        const int c[12] = {cfg->pixels_per_lane, cfg->rows_per_warp, cfg->warps, cfg->chunk_channels,
                            cfg->stages, cfg->row_groups, cfg->min_blocks, cfg->copy_mode, cfg->producer_warps,
-                           cfg->math_mode, cfg->consumer_groups};
-        for (int i = 0; i < 11; ++i) key.c[i] = c[i];
+                           cfg->math_mode, cfg->consumer_groups, cfg->split_rows};
+        for (int i = 0; i < 12; ++i) key.c[i] = c[i];
     }
     {
         std::lock_guard<std::mutex> lk(w->mu);
@@ -832,6 +852,7 @@ ALCS_API int alcs_variant_get(int index, alcs_dtype* dt, int* g, alcs_launch_cfg
         cfg->producer_warps = v.npw;
         cfg->math_mode = mode_of(v);
         cfg->consumer_groups = v.groups;
+        cfg->split_rows = v.split ? 1 : 2;
     }
     return ALCS_OK;
 }
@@ -1246,6 +1267,7 @@ extern "C" ALCS_API int alcs_spconv1x1_noalloc(const alcs_packed* w, const void*
     ConvArgs a;
     a.x = xk; a.y = y; a.bias = bias; a.res = nullptr;
     a.rec = sc->rec; a.slice = sc->slice; a.rowoff = sc->rowoff; a.rowmap = sc->rowmap;
+    set_unit_args(a, *sc, v.mma);
     a.err = w->d_err;
     a.rows = w->rows; a.cin = w->cin; a.cout = w->cout; a.hw = hwx; a.hwy = hw;
     a.q_total = n * hwx;
@@ -1257,6 +1279,7 @@ extern "C" ALCS_API int alcs_spconv1x1_noalloc(const alcs_packed* w, const void*
     a.y_f32 = (flags & ALCS_Y_F32) ? 1 : 0;
     const StageLayout L = stage_layout(v, *sc, elt);
     a.off_rec = L.off_rec; a.off_rowoff = L.off_rowoff; a.stage_bytes = L.stage_bytes;
+    if (a.unit) a.off_xch = 16 * alcs::kMaxStages + a.stages * L.stage_bytes;
     int ld = 16;
     while (ld > elt && (((size_t)hwx * elt) % ld || (uintptr_t)xk % ld)) ld >>= 1;
     a.ld_bytes = ld;

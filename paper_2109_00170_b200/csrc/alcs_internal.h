@@ -41,7 +41,10 @@ constexpr int kChunkings[kNumChunkings] = {16, 32, 64, 96, 128, 0};
 // map), and a row group's rows are dealt to the (warp, accumulator set) pairs so that the warps with
 // equal index modulo 4 (one scheduler of the SM) get the same number of rows and nearly the same
 // number of blocks: the row of (warp w, set s) is local row s*nwg + (s odd ? nwg-1-w : w), the
-// kernel's own mapping.
+// kernel's own mapping.  A block row that is far longer than the others of its row group is split
+// into parts that take separate (warp, set) pairs (see build_schedule_balanced); for this flavour the
+// row-map array is followed by one unit word per local row (unit_word()) and one count of secondary
+// units per row group: h_rowmap = [n_rg*rpg rows | n_rg*rpg unit words | n_rg counts].
 //
 // The tensor-core flavour (mma = 1, fp16 weights, g = 8 or 16) keeps the same slices and row
 // headers but stores a segment as "step records" of 16 blocks each: the 16 chunk-local columns
@@ -54,6 +57,7 @@ struct Schedule {
     int mma = 0;                   // 1: step records for the tensor-core kernels
     int balanced = 0;              // 1: the balanced flavour (below); then rpg = nwg * rw local rows per row group
     int nwg = 0, rw = 0;           // balanced flavour: consumer warps and accumulator sets per warp it was built for
+    int max_x = 0;                 // balanced flavour: most secondary units (parts of split rows) in any row group
     int ros = 0;                   // ints per (row group, chunk) row of rowoff: 4 per local row
     int wcap = 0;                  // longest slice, in 16-byte units
     int n_rec = 0;                 // total length of all slices, in 16-byte units
@@ -88,11 +92,11 @@ struct Plan {
 struct ShapeKey {
     int n, h, wd;
     unsigned flags;
-    int c[11] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+    int c[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
     bool operator<(const ShapeKey& o) const {
         if (std::tie(n, h, wd, flags) != std::tie(o.n, o.h, o.wd, o.flags))
             return std::tie(n, h, wd, flags) < std::tie(o.n, o.h, o.wd, o.flags);
-        for (int i = 0; i < 11; ++i)
+        for (int i = 0; i < 12; ++i)
             if (c[i] != o.c[i]) return c[i] < o.c[i];
         return false;
     }
@@ -134,15 +138,18 @@ float half_bits_to_float(uint16_t h);
 void build_schedule(const alcs_packed& p, int kc, int n_rg, bool with_records, Schedule& out);
 void build_schedule_mma(const alcs_packed& p, int kc, int n_rg, bool with_records, Schedule& out);
 int pair_record_bytes(int g);                 // bytes of one pair record
+int unit_word(int role, int slot, int count);  // see alcs_pack.cpp
 int local_row_of(int w, int s, int nw);       // local row of (consumer warp w, accumulator set s), nw consumer warps
-void build_schedule_balanced(const alcs_packed& p, int kc, int n_rg, int nwg, int rw, bool with_records, Schedule& out);
+void build_schedule_balanced(const alcs_packed& p, int kc, int n_rg, int nwg, int rw, bool with_records, Schedule& out,
+                             bool allow_split = true);
 // Which flavour of the schedule a kernel takes: 0 = pair records, rows dealt without regard to the
 // kernel's shape (the general convolution), 1 = step records of the tensor-core kernels, otherwise
-// pair records balanced for (nwg, rw).
+// pair records balanced for (nwg, rw), with or without long block rows split into parts.
 constexpr int kMaxBalancedKc = 1 << 19;
-inline int balanced_flavour(int nwg, int rw) { return 2 + nwg * 16 + rw; }
-inline int flavour_nwg(int flavour) { return (flavour - 2) / 16; }
-inline int flavour_rw(int flavour) { return (flavour - 2) % 16; }
+inline int balanced_flavour(int nwg, int rw, int split) { return 2 + ((nwg * 16 + rw) << 1 | (split ? 1 : 0)); }
+inline int flavour_split(int flavour) { return (flavour - 2) & 1; }
+inline int flavour_nwg(int flavour) { return ((flavour - 2) >> 1) / 16; }
+inline int flavour_rw(int flavour) { return ((flavour - 2) >> 1) % 16; }
 inline std::pair<int, int> sched_key(int kc, int n_rg, int flavour)
 {
     if (flavour == 1) return std::make_pair(-kc, n_rg);

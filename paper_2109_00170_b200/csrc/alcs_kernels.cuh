@@ -55,6 +55,11 @@ struct ConvArgs {
     const int* slice;         // [n_rg*nch + 1] start of each (row group, chunk) slice, in 16-byte units
     const int* rowoff;        // [n_rg][nch][rpg] int4 per local row: {segment start inside the slice (16-byte units), c0, c1, pairs}
     const int* rowmap;        // [n_rg][rpg] block row of each local row, -1 = none
+    const int* unit;          // [n_rg][rpg] unit word of each local row (role | slot << 4 | count << 16), or nullptr when
+                              // no block row of the schedule is split into parts
+    const int* rgx;           // [n_rg] secondary units per row group (0: no hand-over in that row group)
+    int off_xch;              // shared memory: hand-over area [mbarrier, 16 bytes | 2 x xch_slots tiles of G*P*32 floats]
+    int xch_slots;
     int* err;                 // device error word (0 = ok)
     int rows, cin, cout;
     int hw;                   // pixels per image in X (padded up when X was repacked to aligned rows)
@@ -604,7 +609,9 @@ drain:
         for (int j = max(0, kk_other - S); j < kk_other; ++j) mbar_wait(smem_u32 + 8 * ((turn ^ 1) * S + j % S), (j / S) & 1);
 }
 
-template <typename XT, int G, int P, int RW, int NW, int MINB, int NPW>
+// SPLIT: the flavour for schedules in which block rows are split into parts (the hand-over below); it is
+// a compile-time flavour because even its few extra live values cost the common flavour spills.
+template <typename XT, int G, int P, int RW, int NW, int MINB, int NPW, bool SPLIT = false>
 __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_kernel(const ConvArgs a)
 {
     constexpr int T = 32 * P;                         // pixels per tile
@@ -630,6 +637,7 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_kernel(const 
             mbar_init(smem_u32 + 8 * s, a.bulk ? 1 : 32 * NPW);     // full: one announcing arrival, or every producer lane
             mbar_init(smem_u32 + 8 * kMaxStages + 8 * s, NW);       // empty: one arrival per consumer warp
         }
+        if constexpr (SPLIT) mbar_init(smem_u32 + a.off_xch, NW);  // hand-over of split rows: one arrival per consumer warp
     }
     __syncthreads();
     grid_dep_launch();
@@ -706,6 +714,54 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_kernel(const 
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32 + 8 * kMaxStages + 8 * st);   // stage st may be refilled
+        }
+
+        // ---- rows split into parts: the secondary parts hand their partial sums to the primary one through
+        // shared memory (two alternating sets of tiles, one bounded barrier among the consumer warps per item);
+        // the primary adds them in slot order, so the result does not depend on timing
+        if constexpr (SPLIT) {      // (every item takes the barrier, so its phase follows from the item's number)
+            const int xphase = (item - (int)blockIdx.x) / (int)gridDim.x;
+            const int xrg = item - (item / a.n_rg) * a.n_rg;
+            constexpr int TILE2 = G * (P / 2) * 32;             // float2 elements of one hand-over tile
+            float2* xch = reinterpret_cast<float2*>(smem + a.off_xch + 16) + (size_t)(xphase & 1) * a.xch_slots * TILE2;
+#pragma unroll
+            for (int s = 0; s < RW; ++s) {
+                const int lr = s * NW + ((s & 1) ? NW - 1 - warp : warp);
+                const int uw = lr < a.rpg ? __ldg(a.unit + xrg * a.rpg + lr) : 0;
+                if ((uw & 15) == 2) {
+                    float2* t = xch + (size_t)((uw >> 4) & 0xfff) * TILE2 + lane;
+#pragma unroll
+                    for (int j = 0; j < G; ++j)
+#pragma unroll
+                        for (int e = 0; e < P / 2; ++e) t[(j * (P / 2) + e) * 32] = acc[s][j][e];
+                    rowid[s] = -1;                              // a secondary part stores nothing itself
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32 + a.off_xch);
+            if (!mbar_wait(smem_u32 + a.off_xch, xphase & 1)) {
+                if (lane == 0) atomicExch(a.err, kErrFullWait);
+                return;
+            }
+#pragma unroll
+            for (int s = 0; s < RW; ++s) {
+                const int lr = s * NW + ((s & 1) ? NW - 1 - warp : warp);
+                const int uw = lr < a.rpg ? __ldg(a.unit + xrg * a.rpg + lr) : 0;
+                if ((uw & 15) == 1) {
+                    const int first = (uw >> 4) & 0xfff, count = uw >> 16;
+                    for (int i = 0; i < count; ++i) {
+                        const float2* t = xch + (size_t)(first + i) * TILE2 + lane;
+#pragma unroll
+                        for (int j = 0; j < G; ++j)
+#pragma unroll
+                            for (int e = 0; e < P / 2; ++e) {
+                                const float2 v = t[(j * (P / 2) + e) * 32];
+                                acc[s][j][e].x += v.x;
+                                acc[s][j][e].y += v.y;
+                            }
+                    }
+                }
+            }
         }
 
         // ---- epilogue: bias, ReLU, store ----------------------------------------------------
@@ -819,11 +875,14 @@ struct KernelVariant {
     const void* fn;
     int mma;
     int groups;     // consumer groups that take the items of a thread block in turn (1 or 2); nw counts all consumer warps
+    int split;      // 1: takes schedules in which long block rows are split into parts
 };
 
 #define ALCS_VARIANT_P(XT, ISF16, G, P, RW, NW, MINB, NPW) \
     {ISF16, G, P, RW, NW, MINB, NPW, (const void*)&spconv1x1_kernel<XT, G, P, RW, NW, MINB, NPW>, 0, 1}
 #define ALCS_VARIANT(XT, ISF16, G, P, RW, NW, MINB) ALCS_VARIANT_P(XT, ISF16, G, P, RW, NW, MINB, 1)
+#define ALCS_VARIANT_SPLIT(XT, ISF16, G, P, RW, NW, MINB, NPW) \
+    {ISF16, G, P, RW, NW, MINB, NPW, (const void*)&spconv1x1_kernel<XT, G, P, RW, NW, MINB, NPW, true>, 0, 1, 1}
 
 // Defined one per translation unit, concatenated by alcs_device.cu.
 const KernelVariant* variants_f32_g4(int* n);

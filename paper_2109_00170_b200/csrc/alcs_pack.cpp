@@ -58,7 +58,11 @@ static int rec_bytes(int g) { return g == 1 ? 16 : 16 + 8 * g; }
 int pair_record_bytes(int g) { return rec_bytes(g); }
 
 // Pair records, slices and row headers for the row map already in `out` (n_rg groups of rpg local rows).
-static void emit_pair_records(const alcs_packed& p, int kc, bool with_records, Schedule& out)
+// part[rg*rpg + t] / nparts[...]: local row t multiplies only the blocks of its block row whose position in
+// the row is congruent to part modulo nparts (empty vectors: every local row takes its whole row).
+static void emit_pair_records(const alcs_packed& p, int kc, bool with_records, Schedule& out,
+                              const std::vector<int>& part = std::vector<int>(),
+                              const std::vector<int>& nparts = std::vector<int>())
 {
     const int R = p.rows, g = p.g;
     const int n_rg = out.n_rg, rpg = out.rpg;
@@ -70,7 +74,8 @@ static void emit_pair_records(const alcs_packed& p, int kc, bool with_records, S
     out.ros = ros;
     out.h_rowoff.assign((size_t)n_rg * nch * ros, 0);
     out.h_rec.clear();
-    std::vector<int> cursor(R);
+    std::vector<int> cursor((size_t)rpg);           // per local row: next block of its block row to look at
+    std::vector<int> mine;                          // blocks of the current segment
     int rec_count = 0, wcap = 0;
     auto value = [&](int k, int j) -> float {
         const size_t vi = (size_t)k * g + j;
@@ -87,7 +92,7 @@ static void emit_pair_records(const alcs_packed& p, int kc, bool with_records, S
     for (int rg = 0; rg < n_rg; ++rg) {
         for (int t = 0; t < rpg; ++t) {
             const int r = out.h_rowmap[(size_t)rg * rpg + t];
-            if (r >= 0) cursor[r] = p.row_ptr[r];
+            if (r >= 0) cursor[t] = p.row_ptr[r];
         }
         for (int c = 0; c < nch; ++c) {
             out.h_slice[(size_t)rg * nch + c] = rec_count;
@@ -100,15 +105,20 @@ static void emit_pair_records(const alcs_packed& p, int kc, bool with_records, S
                 hd[0] = local; hd[1] = hd[2] = hd[3] = 0;
                 const int r = out.h_rowmap[(size_t)rg * rpg + t];
                 if (r < 0) continue;
-                int k = cursor[r];
+                const int np = nparts.empty() ? 1 : nparts[(size_t)rg * rpg + t];
+                const int pt = part.empty() ? 0 : part[(size_t)rg * rpg + t];
                 const int kend = p.row_ptr[r + 1];
-                int k1 = k;
-                while (k1 < kend && p.col_idx[k1] < lim) ++k1;
-                const int npair = (k1 - k + 1) / 2;
+                int k1 = cursor[t];
+                mine.clear();
+                for (; k1 < kend && p.col_idx[k1] < lim; ++k1)
+                    if ((k1 - p.row_ptr[r]) % np == pt) mine.push_back(k1);
+                cursor[t] = k1;
+                const int nblk = (int)mine.size();
+                const int npair = (nblk + 1) / 2;
                 const int seg16 = npair * (REC / 16);
                 auto cols_of = [&](int q, int* c) {       // chunk-local columns of pair q
-                    const int ka = k + 2 * q;
-                    const int kb = ka + 1 < k1 ? ka + 1 : ka;    // padding repeats the column
+                    const int ka = mine[2 * q];
+                    const int kb = 2 * q + 1 < nblk ? mine[2 * q + 1] : ka;    // padding repeats the column
                     c[0] = p.col_idx[ka] - c0;
                     c[1] = p.col_idx[kb] - c0;
                 };
@@ -119,20 +129,19 @@ static void emit_pair_records(const alcs_packed& p, int kc, bool with_records, S
                     out.h_rec.resize(base + (size_t)seg16 * 16, 0);
                     for (int q = 0; q < npair; ++q) {
                         unsigned char* rec = &out.h_rec[base + (size_t)q * REC];
-                        const int ka = k + 2 * q;
-                        const bool has_b = ka + 1 < k1;
+                        const int ka = mine[2 * q];
+                        const bool has_b = 2 * q + 1 < nblk;
                         int hdr[4] = {0, 0, 0, 0};
                         if (q + 1 < npair) cols_of(q + 1, hdr);       // columns of the next pair
                         float* w = reinterpret_cast<float*>(rec + (g == 1 ? 8 : 16));
                         for (int j = 0; j < g; ++j) {
                             w[j] = value(ka, j);
-                            w[g + j] = has_b ? value(ka + 1, j) : 0.0f;
+                            w[g + j] = has_b ? value(mine[2 * q + 1], j) : 0.0f;
                         }
                         std::memcpy(rec, hdr, g == 1 ? 8 : 16);
                     }
                 }
                 local += seg16;
-                cursor[r] = k1;
             }
             rec_count += local;
             wcap = std::max(wcap, local);
@@ -173,8 +182,17 @@ void build_schedule(const alcs_packed& p, int kc, int n_rg, bool with_records, S
 // own mapping (tier s, warps in serpentine order).
 int local_row_of(int w, int s, int nw) { return s * nw + ((s & 1) ? nw - 1 - w : w); }
 
+// Word that tells a consumer warp what the unit in one of its accumulator sets is: role 0 = a whole
+// block row, 1 = the primary part of a split row (adds `count` partial sums found in exchange slots
+// slot, slot+1, ... and stores the row), 2 = a secondary part (writes its partial sums to exchange slot
+// `slot` and stores nothing).
+int unit_word(int role, int slot, int count) { return role | (slot << 4) | (count << 16); }
+constexpr int kMaxExchange = 6;     // secondary units per row group (each costs an exchange tile in shared memory)
+constexpr int kMaxParts = 7;        // parts one block row may be split into
+
 // Balanced flavour of the pair-record schedule: see the comment on Schedule.
-void build_schedule_balanced(const alcs_packed& p, int kc, int n_rg, int nw, int rw, bool with_records, Schedule& out)
+void build_schedule_balanced(const alcs_packed& p, int kc, int n_rg, int nw, int rw, bool with_records, Schedule& out,
+                             bool allow_split)
 {
     if (kc <= 0 || kc > p.cin) kc = p.cin;
     const int R = p.rows;
@@ -182,6 +200,7 @@ void build_schedule_balanced(const alcs_packed& p, int kc, int n_rg, int nw, int
     n_rg = std::max(std::max(1, (R + cap - 1) / cap), std::min(n_rg, R));
     out.n_rg = n_rg; out.rpg = cap; out.mma = 0; out.balanced = 1;
     out.nwg = nw; out.rw = rw;
+    out.max_x = 0;
 
     // Sizes of the row groups: whole multiples of 4 where the capacity allows it, so that the four
     // schedulers of an SM can be given the same number of rows; otherwise as even as possible.
@@ -216,23 +235,84 @@ void build_schedule_balanced(const alcs_packed& p, int kc, int n_rg, int nw, int
         }
     }
 
-    // Inside a row group: rows (longest first) are dealt in serpentine order to the schedulers
-    // (scheduler of consumer warp w = w mod 4), then, per scheduler, to its warps; the t-th row a
-    // warp receives becomes its accumulator set t.
-    out.h_rowmap.assign((size_t)n_rg * cap, -1);
+    // Inside a row group: "units" are dealt to the (warp, accumulator set) pairs.  A unit is a whole block
+    // row, or, for a row far longer than the others, one of nparts parts of it (the blocks whose position
+    // in the row is congruent to `part` modulo nparts, so that every chunk's share is split as well); the
+    // spare (warp, set) pairs of the row group pay for the extra units.  Part 0 is the row's primary unit
+    // (it adds the others' partial sums, handed over through shared memory, and stores the row); at most
+    // kMaxExchange secondary units per row group.  Units, largest first, go in serpentine order to the
+    // schedulers (scheduler of consumer warp w = w mod 4), then, per scheduler, to its warps; the t-th
+    // unit a warp receives becomes its accumulator set t.
+    struct Unit { int row, part, nparts, blocks; };
+    const size_t nloc = (size_t)n_rg * cap;
+    out.h_rowmap.assign(2 * nloc + n_rg, -1);
+    std::fill(out.h_rowmap.begin() + nloc, out.h_rowmap.end(), 0);
+    std::vector<int> part(nloc, 0), nparts(nloc, 1);
+    int* unit_info = out.h_rowmap.data() + nloc;         // per local row, see unit_word()
+    int* rg_exchange = out.h_rowmap.data() + 2 * nloc;   // per row group: secondary units (0: no hand-over)
+    out.max_x = 0;
     const int nsched = std::min(4, nw);
     for (int rg = 0; rg < n_rg; ++rg) {
-        std::vector<std::vector<int>> per(nsched);
+        std::vector<Unit> units;
+        long long blocks_total = 0;
+        for (int r : members[rg]) {
+            const int len = p.row_ptr[r + 1] - p.row_ptr[r];
+            units.push_back({r, 0, 1, len});
+            blocks_total += len;
+        }
+        // split while a row's parts are still much larger than the average unit and a spare pair is left
+        int spare = cap - (int)members[rg].size(), exchange = 0;
+        std::vector<int> parts_of(members[rg].size(), 1);
+        while (allow_split && spare > 0 && exchange < kMaxExchange && !units.empty()) {
+            size_t best = 0;
+            double best_load = -1;
+            for (size_t i = 0; i < members[rg].size(); ++i) {
+                const int len = p.row_ptr[members[rg][i] + 1] - p.row_ptr[members[rg][i]];
+                const double load = (double)len / parts_of[i];
+                if (load > best_load) { best_load = load; best = i; }
+            }
+            const double avg = (double)blocks_total / (double)(members[rg].size() + exchange);
+            if (best_load <= std::max(1.5 * avg, 16.0) || parts_of[best] >= kMaxParts) break;
+            ++parts_of[best];
+            ++exchange;
+            --spare;
+        }
+        if (exchange > 0) {
+            units.clear();
+            for (size_t i = 0; i < members[rg].size(); ++i) {
+                const int r = members[rg][i];
+                const int len = p.row_ptr[r + 1] - p.row_ptr[r];
+                for (int q = 0; q < parts_of[i]; ++q)
+                    units.push_back({r, q, parts_of[i], (len - q + parts_of[i] - 1) / parts_of[i]});
+            }
+            std::stable_sort(units.begin(), units.end(), [](const Unit& a, const Unit& b) { return a.blocks > b.blocks; });
+        }
+        rg_exchange[rg] = exchange;
+        out.max_x = std::max(out.max_x, exchange);
+
+        std::vector<std::vector<Unit>> per(nsched);
         std::vector<int> room(nsched, 0);
         for (int w = 0; w < nw; ++w) room[w % nsched] += rw;
         {
             int pos = 0, dir = 1;
             size_t i = 0;
-            while (i < members[rg].size()) {
-                if ((int)per[pos].size() < room[pos]) per[pos].push_back(members[rg][i++]);
+            while (i < units.size()) {
+                if ((int)per[pos].size() < room[pos]) per[pos].push_back(units[i++]);
                 if (pos + dir < 0 || pos + dir >= nsched) dir = -dir; else pos += dir;
             }
         }
+        // exchange slots: the secondary units of a row take consecutive slots, rows in order of appearance
+        std::vector<int> first_slot(members[rg].size(), -1);
+        {
+            int next = 0;
+            for (size_t i = 0; i < members[rg].size(); ++i)
+                if (parts_of[i] > 1) { first_slot[i] = next; next += parts_of[i] - 1; }
+        }
+        auto index_of = [&](int row) {
+            for (size_t i = 0; i < members[rg].size(); ++i)
+                if (members[rg][i] == row) return i;
+            return (size_t)0;
+        };
         for (int k = 0; k < nsched; ++k) {
             std::vector<int> warps;
             for (int w = k; w < nw; w += nsched) warps.push_back(w);
@@ -241,14 +321,22 @@ void build_schedule_balanced(const alcs_packed& p, int kc, int n_rg, int nw, int
             size_t i = 0;
             while (i < per[k].size()) {
                 if (fill[pos] < rw) {
-                    out.h_rowmap[(size_t)rg * cap + local_row_of(warps[pos], fill[pos], nw)] = per[k][i++];
+                    const Unit& u = per[k][i++];
+                    const size_t at = (size_t)rg * cap + local_row_of(warps[pos], fill[pos], nw);
+                    out.h_rowmap[at] = u.row;
+                    part[at] = u.part;
+                    nparts[at] = u.nparts;
+                    if (u.nparts > 1) {
+                        const int fs = first_slot[index_of(u.row)];
+                        unit_info[at] = u.part == 0 ? unit_word(1, fs, u.nparts - 1) : unit_word(2, fs + u.part - 1, 0);
+                    }
                     ++fill[pos];
                 }
                 if (pos + dir < 0 || pos + dir >= (int)warps.size()) dir = -dir; else pos += dir;
             }
         }
     }
-    emit_pair_records(p, kc, with_records, out);
+    emit_pair_records(p, kc, with_records, out, part, nparts);
 }
 
 // Tensor-core flavour of the schedule (fp16 weights): see the comment on Schedule.
@@ -400,9 +488,41 @@ ALCS_API int alcs_schedule_selfcheck(const alcs_packed* p, int chunk_channels, i
     const int REC = alcs::pair_record_bytes(g);
     if (sc.rpg != cap || sc.ros != 4 * cap) return ALCS_ERR_CORRUPT;
     // every block row exactly once in the row map
+    // every block row stored by exactly one unit (a whole row or the primary part of a split row), and the
+    // exchange slots of a row group used exactly once each
+    const size_t nloc = (size_t)sc.n_rg * cap;
+    if (sc.h_rowmap.size() != 2 * nloc + sc.n_rg) return ALCS_ERR_CORRUPT;
     std::vector<int> seen(p->rows, 0);
-    for (int v : sc.h_rowmap)
-        if (v >= 0) { if (v >= p->rows) return ALCS_ERR_CORRUPT; ++seen[v]; }
+    int64_t secondaries = 0;
+    for (int rg = 0; rg < sc.n_rg; ++rg) {
+        const int nx = sc.h_rowmap[2 * nloc + rg];
+        if (nx < 0 || nx > sc.max_x) return ALCS_ERR_CORRUPT;
+        std::vector<int> written(nx, 0), read(nx, 0);
+        for (int t = 0; t < cap; ++t) {
+            const int v = sc.h_rowmap[(size_t)rg * cap + t];
+            const int uw = sc.h_rowmap[nloc + (size_t)rg * cap + t];
+            const int role = uw & 15, slot = (uw >> 4) & 0xfff, count = uw >> 16;
+            if (v < 0) { if (uw != 0) return ALCS_ERR_CORRUPT; continue; }
+            if (v >= p->rows || role > 2) return ALCS_ERR_CORRUPT;
+            if (role != 2) ++seen[v];
+            if (role == 2) { if (slot >= nx) return ALCS_ERR_CORRUPT; ++written[slot]; ++secondaries; }
+            if (role == 1) {
+                if (count < 1 || slot + count > nx) return ALCS_ERR_CORRUPT;
+                for (int i = 0; i < count; ++i) {
+                    ++read[slot + i];
+                    // the slot must be written by a part of the same row
+                    bool found = false;
+                    for (int t2 = 0; t2 < cap; ++t2) {
+                        const int uw2 = sc.h_rowmap[nloc + (size_t)rg * cap + t2];
+                        if ((uw2 & 15) == 2 && ((uw2 >> 4) & 0xfff) == slot + i && sc.h_rowmap[(size_t)rg * cap + t2] == v) found = true;
+                    }
+                    if (!found) return ALCS_ERR_CORRUPT;
+                }
+            }
+        }
+        for (int i = 0; i < nx; ++i)
+            if (written[i] != 1 || read[i] != 1) return ALCS_ERR_CORRUPT;
+    }
     for (int r = 0; r < p->rows; ++r)
         if (seen[r] != 1) return ALCS_ERR_CORRUPT;
     // walk every (warp, accumulator set) the way a consumer warp does and rebuild the dense matrix
@@ -475,6 +595,7 @@ ALCS_API int alcs_schedule_selfcheck(const alcs_packed* p, int chunk_channels, i
         stats[0] = sc.n_rg; stats[1] = max_sched; stats[2] = min_sched == LLONG_MAX ? 0 : min_sched;
         stats[3] = pairs; stats[4] = p->nb;
         stats[5] = max_rows; stats[6] = min_rows == LLONG_MAX ? 0 : min_rows;
+        stats[7] = secondaries;
     }
     return ALCS_OK;
 }

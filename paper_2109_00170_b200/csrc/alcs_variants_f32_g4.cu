@@ -59,6 +59,15 @@ static const KernelVariant kTable[] = {
     ALCS_VARIANT_P(float, 0, 4, 16, 1, 11, 1, 1),
     ALCS_VARIANT_P(float, 0, 4, 16, 2, 7, 1, 1),
     ALCS_VARIANT_P(float, 0, 4, 16, 1, 10, 1, 2),
+    // the same kernels for schedules with block rows split into parts (skewed row lengths)
+    ALCS_VARIANT_SPLIT(float, 0, 4, 8, 2, 12, 1, 4),
+    ALCS_VARIANT_SPLIT(float, 0, 4, 8, 2, 12, 1, 2),
+    ALCS_VARIANT_SPLIT(float, 0, 4, 8, 2, 14, 1, 2),
+    ALCS_VARIANT_SPLIT(float, 0, 4, 8, 1, 16, 1, 4),
+    ALCS_VARIANT_SPLIT(float, 0, 4, 8, 3, 8, 1, 4),
+    ALCS_VARIANT_SPLIT(float, 0, 4, 4, 3, 16, 1, 4),
+    ALCS_VARIANT_SPLIT(float, 0, 4, 4, 4, 12, 1, 4),
+    ALCS_VARIANT_SPLIT(float, 0, 4, 4, 2, 16, 1, 4),
 };
 
 const KernelVariant* variants_f32_g4(int* n)

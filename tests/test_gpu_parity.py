@@ -174,14 +174,15 @@ def test_every_kernel_variant(alcs, g, dtype):
     ran = variants = 0
     for vi in range(alcs.alcs_variant_count()):
         v = alcs.alcs_variant_get(vi)
-        if v["g"] != g or v["dtype"] != want_dt:
+        if v["g"] != g or v["dtype"] != want_dt or v["split_rows"] == 1:    # (split flavours: the test below)
             continue
         variants += 1
         for kc in (32, 64, 128, 200):
             for stages in (2, 3, 4):
                 cfg = dict(pixels_per_lane=v["pixels_per_lane"], rows_per_warp=v["rows_per_warp"],
                            warps=v["warps"], min_blocks=v["min_blocks"], producer_warps=v["producer_warps"],
-                           math_mode=v["math_mode"], consumer_groups=v["consumer_groups"], chunk_channels=kc,
+                           math_mode=v["math_mode"], consumer_groups=v["consumer_groups"], split_rows=v["split_rows"],
+                           chunk_channels=kc,
                            stages=stages, row_groups=0)
                 try:
                     Y = run_gpu(alcs, W, M, X, b, True, g, cfg=cfg, packed=p)
@@ -191,6 +192,40 @@ def test_every_kernel_variant(alcs, g, dtype):
                 assert_parity(Y, Yref, A, "f32" if dtype == np.float32 else "f16")
                 ran += 1
     assert variants >= 1 and ran >= 4 * variants
+
+
+def test_split_row_variants_on_skewed_rows(alcs):
+    """Every kernel flavour that splits long block rows into parts, on Zipf-distributed row lengths with a
+    few full rows: the parts' partial sums must add up to the oracle's result, run after run."""
+    from alcs_workloads import zipf_block_mask
+    n, cin, cout, hw, g = 3, 256, 192, 300, 4
+    W, M, X, b = _rand(31, n, cin, cout, hw, g, 0.3)
+    M = zipf_block_mask(cout // g, cin, 77)
+    M[3] = 1; M[17] = 1
+    Yref, A = oracle.conv1x1(W, M, X, b, True, g, want_scale=True)
+    p = alcs.alcs_packed_upload(alcs.alcs_pack(W, M, g), 0)
+    ran = 0
+    for vi in range(alcs.alcs_variant_count()):
+        v = alcs.alcs_variant_get(vi)
+        if v["g"] != g or v["dtype"] != alcs.ALCS_F32 or v["split_rows"] != 1:
+            continue
+        for kc, stages, rg in ((32, 3, 0), (64, 2, 3), (256, 2, 5)):
+            cfg = dict(pixels_per_lane=v["pixels_per_lane"], rows_per_warp=v["rows_per_warp"], warps=v["warps"],
+                       min_blocks=v["min_blocks"], producer_warps=v["producer_warps"], math_mode=1, split_rows=1,
+                       chunk_channels=kc, stages=stages, row_groups=rg)
+            try:
+                Y1 = run_gpu(alcs, W, M, X, b, True, g, cfg=cfg, packed=p)
+            except alcs.AlcsError as e:
+                assert e.status == alcs.ALCS_ERR_UNSUPPORTED
+                continue
+            assert_parity(Y1, Yref, A, "f32")
+            assert np.array_equal(Y1, run_gpu(alcs, W, M, X, b, True, g, cfg=cfg, packed=p))     # deterministic
+            ran += 1
+    assert ran >= 8
+    # integer data: bit-exact whatever the split
+    Wi = _ints(41, (cout, cin)).astype(np.float32)
+    Xi = _ints(42, (n, cin, hw)).astype(np.float32)
+    check_layer(alcs, Wi, M, Xi, None, False, g, cfg=dict(split_rows=1, math_mode=1), exact=True)
 
 
 def test_row_group_counts(alcs):

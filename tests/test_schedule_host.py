@@ -68,3 +68,19 @@ def test_selfcheck_argument_errors():
         with pytest.raises(A.AlcsError) as e:
             A.alcs_schedule_selfcheck(p, *bad)
         assert e.value.status == A.ALCS_ERR_INVALID_ARG
+
+
+def test_long_rows_are_split_into_parts():
+    """Zipf-distributed row lengths: with spare (warp, set) pairs the longest rows are split, every kept block
+    still multiplied exactly once (the self-check walks all parts), and the most loaded scheduler carries far
+    less than the longest row would alone."""
+    W, _ = _matrix(3, 512, 512, 4, 0.5)
+    M = zipf_block_mask(128, 512, 9)
+    p = A.alcs_pack(W, M, 4)
+    longest = int(M.sum(axis=1).max())
+    st = A.alcs_schedule_selfcheck(p, 64, 8, 12, 2)
+    assert st["secondary_units"] > 0
+    assert st["max_sched"] < 1.3 * longest
+    assert st["nb"] == int(M.sum())
+    uniform = A.alcs_schedule_selfcheck(A.alcs_pack(*_matrix(4, 512, 512, 4, 0.25), 4), 64, 6, 12, 2)
+    assert uniform["secondary_units"] == 0

@@ -59,3 +59,12 @@ def normal(seed: int, stream: int, n: int, sigma: float = 1.0) -> np.ndarray:
 def permutation(seed: int, stream: int, n: int) -> np.ndarray:
     """A seeded permutation of range(n): stable argsort of n random 64-bit keys."""
     return np.argsort(bits64(seed, stream, n), kind="stable")
+
+
+def to_bf16_bits(x):
+    """float32 array -> bfloat16 bit patterns (uint16), round to nearest, ties to even; NaNs stay NaNs.
+    Input preparation only: the values a bfloat16 workload feeds to both sides."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    rounded = (u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))) >> np.uint32(16)
+    nan = (u & np.uint32(0x7FFFFFFF)) > np.uint32(0x7F800000)
+    return np.where(nan, (u >> np.uint32(16)) | np.uint32(0x40), rounded).astype(np.uint16)

@@ -43,6 +43,14 @@ def _lib(mutant: int = 0, build_dir: str | None = None):
     return lib
 
 
+def bf16_decode(bits):
+    """bfloat16 bit patterns (uint16) -> the float32 values they denote, exactly: a bfloat16 number is the
+    float32 number whose upper 16 bits are its bits and whose lower 16 bits are zero.  The oracle takes
+    bfloat16 operands as these float32 arrays (it works in double precision either way)."""
+    bits = np.ascontiguousarray(bits, dtype=np.uint16)
+    return (bits.astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
 def num_threads() -> int:
     """Threads the oracle's OpenMP loops will use."""
     return int(_lib().oracle_num_threads())

@@ -135,3 +135,19 @@ def test_pins_reject_planted_mistakes(tmp_path):
     assert _pins_pass(0, None)
     for mutant in (10, 11):       # residual added after the activation; sampling grid shifted by one pixel
         assert not _pins_pass(mutant, str(tmp_path)), f"mutant {mutant} slipped through"
+
+
+def test_bfloat16_decoding_and_encoding():
+    """Every bfloat16 bit pattern decodes to what an independent library says it is, and the workloads'
+    encoder rounds float32 to the nearest bfloat16 with ties to even (the same library as witness)."""
+    import torch
+    bits = np.arange(65536, dtype=np.uint16)
+    ours = oracle.bf16_decode(bits)
+    theirs = torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).to(torch.float32).numpy()
+    assert np.array_equal(ours.view(np.uint32), theirs.view(np.uint32))
+    x = np.concatenate([rng.normal(9, 1, 200000).astype(np.float32) * 37.0,
+                        np.array([0.0, -0.0, 1.0, 1.00390625, 1.01171875, 3.3895314e38, 1e-40, np.inf, -np.inf], np.float32)])
+    enc = rng.to_bf16_bits(x)
+    ref = torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(enc, ref)
+    assert np.isnan(oracle.bf16_decode(rng.to_bf16_bits(np.array([np.nan], np.float32)))).all()

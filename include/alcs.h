@@ -55,12 +55,15 @@ typedef enum {
 
 typedef enum {
     ALCS_F32 = 0,               /* fp32 weights, activations and outputs, fp32 accumulation         */
-    ALCS_F16 = 1                /* IEEE binary16 weights and activations, fp32 accumulation         */
+    ALCS_F16 = 1,               /* IEEE binary16 weights and activations, fp32 accumulation         */
+    ALCS_BF16 = 2               /* bfloat16 weights and activations, fp32 accumulation; by the paper's rule
+                                   (Section 3.2.1: group size = register bits / element bits) a 16-bit type
+                                   doubles the group size of fp32, as binary16 does.  CUDA-core kernels only. */
 } alcs_dtype;
 
 /* Bits of the `flags` argument of the convolution entry points. */
 #define ALCS_RELU 1u            /* y = max(acc + bias, 0)                                           */
-#define ALCS_Y_F32 2u           /* ALCS_F16 weights only: write Y as fp32 instead of fp16           */
+#define ALCS_Y_F32 2u           /* 16-bit weights only: write Y (and read a residual) as fp32 instead of the 16-bit type */
 
 typedef struct alcs_packed alcs_packed;   /* opaque packed weight matrix, library-owned */
 typedef struct alcs_stack alcs_stack;     /* opaque layer stack, library-owned          */

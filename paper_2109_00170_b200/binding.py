@@ -17,7 +17,7 @@ ALCS_OK = 0
 ALCS_ERR_INVALID_ARG, ALCS_ERR_SHAPE, ALCS_ERR_UNSUPPORTED, ALCS_ERR_ALLOC = -1, -2, -3, -4
 ALCS_ERR_CUDA, ALCS_ERR_CORRUPT, ALCS_ERR_STATE, ALCS_ERR_TOO_LARGE = -5, -6, -7, -8
 ALCS_NOALLOC_SCRATCH_BYTES = 16 << 20
-ALCS_F32, ALCS_F16 = 0, 1
+ALCS_F32, ALCS_F16, ALCS_BF16 = 0, 1, 2
 ALCS_RELU, ALCS_Y_F32 = 1, 2
 ALCS_STACK_GRAPH = 1
 
@@ -198,9 +198,14 @@ class Packed:
             pass
 
 
-def alcs_pack(w: np.ndarray, block_mask: np.ndarray, g: int) -> Packed:
-    """w: [cout, cin] float32 or float16 (host); block_mask: [ceil(cout/g), cin] uint8."""
-    if w.dtype == np.float32:
+def alcs_pack(w: np.ndarray, block_mask: np.ndarray, g: int, bf16: bool = False) -> Packed:
+    """w: [cout, cin] float32 or float16 (host), or, with bf16=True, uint16 holding bfloat16 bit patterns;
+    block_mask: [ceil(cout/g), cin] uint8."""
+    if bf16:
+        if w.dtype != np.uint16:
+            raise TypeError("bfloat16 weights are passed as uint16 bit patterns")
+        dt = ALCS_BF16
+    elif w.dtype == np.float32:
         dt = ALCS_F32
     elif w.dtype == np.float16:
         dt = ALCS_F16
@@ -223,7 +228,7 @@ def alcs_packed_view(p: Packed):
     _check(lib().alcs_packed_view(p.handle, cout, cin, g, dt, nb, C.byref(rp), C.byref(ci), C.byref(va)),
            "alcs_packed_view")
     rows = (cout.value + g.value - 1) // g.value
-    npdt = np.float32 if dt.value == ALCS_F32 else np.float16
+    npdt = {ALCS_F32: np.float32, ALCS_F16: np.float16, ALCS_BF16: np.uint16}[dt.value]     # bfloat16: bit patterns
 
     def arr(ptr, n, t):
         if n == 0:
@@ -237,7 +242,7 @@ def alcs_packed_view(p: Packed):
 
 def alcs_unpack(p: Packed):
     v = alcs_packed_view(p)
-    npdt = np.float32 if v["dtype"] == ALCS_F32 else np.float16
+    npdt = {ALCS_F32: np.float32, ALCS_F16: np.float16, ALCS_BF16: np.uint16}[v["dtype"]]
     rows = (v["cout"] + v["g"] - 1) // v["g"]
     w = np.empty((v["cout"], v["cin"]), dtype=npdt)
     m = np.empty((rows, v["cin"]), dtype=np.uint8)

@@ -20,7 +20,7 @@ OBJ = os.path.join(PKG, "_build")
 LIB = os.path.join(PKG, "libalcs.so")
 
 SOURCES = ["alcs_pack.cpp", "alcs_device.cu", "alcs_conv2d.cu", "alcs_project.cu", "alcs_gather.cu", "alcs_probe.cu", "alcs_variants_f32_g4.cu",
-           "alcs_variants_f32_other.cu", "alcs_variants_f16.cu", "alcs_variants_f16_mma.cu"]
+           "alcs_variants_f32_other.cu", "alcs_variants_f16.cu", "alcs_variants_f16_mma.cu", "alcs_variants_bf16.cu"]
 HEADERS = ["alcs_internal.h", "alcs_kernels.cuh", "alcs_mma.cuh", "alcs_conv2d.cuh", "alcs_gather.h"]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -66,6 +66,8 @@ void init_variants_locked()
     for (int i = 0; i < n; ++i) g_variants.push_back({t[i]});
     t = alcs::variants_f16_mma(&n);
     for (int i = 0; i < n; ++i) g_variants.push_back({t[i]});
+    t = alcs::variants_bf16(&n);
+    for (int i = 0; i < n; ++i) g_variants.push_back({t[i]});
 }
 
 // Which flavour of the launch schedule a variant takes (alcs_internal.h): the CUDA-core kernels take
@@ -308,7 +310,7 @@ int enumerate_plans(const alcs_packed* w, long long q, int hw, std::vector<Plan>
     out.clear();
     for (size_t vi = 0; vi < g_variants.size(); ++vi) {
         const KernelVariant& v = g_variants[vi].v;
-        if (v.is_f16 != (w->dt == ALCS_F16) || v.g != w->g) continue;
+        if (v.is_f16 != (int)w->dt || v.g != w->g) continue;
         rc = prepare_variant(g_variants[vi], w->device);
         if (rc) return rc;
         const int cap = v.nw / v.groups * v.rw;
@@ -528,7 +530,7 @@ int check_conv_args(const alcs_packed* w, const void* x, const void* y, int n, i
     if (!w) return ALCS_ERR_INVALID_ARG;
     if (n < 0 || h < 0 || wd < 0) return ALCS_ERR_INVALID_ARG;
     if (flags & ~(ALCS_RELU | ALCS_Y_F32)) return ALCS_ERR_INVALID_ARG;
-    if ((flags & ALCS_Y_F32) && w->dt != ALCS_F16) return ALCS_ERR_INVALID_ARG;
+    if ((flags & ALCS_Y_F32) && w->dt == ALCS_F32) return ALCS_ERR_INVALID_ARG;
     if (w->g != 1 && w->g != 2 && w->g != 4 && w->g != 8 && w->g != 16) return ALCS_ERR_UNSUPPORTED;
     const long long hw = (long long)h * wd;
     const long long q = hw * n;
@@ -536,7 +538,7 @@ int check_conv_args(const alcs_packed* w, const void* x, const void* y, int n, i
     *q_out = q;
     if (q == 0) return ALCS_OK;
     if (!x || !y) return ALCS_ERR_INVALID_ARG;
-    const size_t xe = w->elt(), ye = (w->dt == ALCS_F16 && !(flags & ALCS_Y_F32)) ? 2 : 4;
+    const size_t xe = w->elt(), ye = (w->dt != ALCS_F32 && !(flags & ALCS_Y_F32)) ? 2 : 4;
     if ((uintptr_t)x % xe || (uintptr_t)y % ye) return ALCS_ERR_INVALID_ARG;
     const uintptr_t xb = (uintptr_t)x, xend = xb + (size_t)q * w->cin * xe;
     const uintptr_t yb = (uintptr_t)y, yend = yb + (size_t)q * w->cout * ye;
@@ -840,7 +842,7 @@ ALCS_API int alcs_variant_get(int index, alcs_dtype* dt, int* g, alcs_launch_cfg
     init_variants_locked();
     if (index < 0 || index >= (int)g_variants.size()) return ALCS_ERR_INVALID_ARG;
     const KernelVariant& v = g_variants[index].v;
-    if (dt) *dt = v.is_f16 ? ALCS_F16 : ALCS_F32;
+    if (dt) *dt = (alcs_dtype)v.is_f16;
     if (g) *g = v.g;
     if (cfg) {
         std::memset(cfg, 0, sizeof *cfg);
@@ -894,7 +896,7 @@ ALCS_API int alcs_spconv1x1_ex(const alcs_packed* w, const void* x, void* y, int
     if (rc) return rc;
     if (q == 0) return ALCS_OK;
     // ... plus what is specific to this entry point: the true extent of x, and the residual
-    const size_t xe = w->elt(), ye = (w->dt == ALCS_F16 && !(flags & ALCS_Y_F32)) ? 2 : 4;
+    const size_t xe = w->elt(), ye = (w->dt != ALCS_F32 && !(flags & ALCS_Y_F32)) ? 2 : 4;
     if ((long long)h * wd > (1ll << 30) || (long long)h * wd * n > (1ll << 31)) return ALCS_ERR_SHAPE;
     const uintptr_t xb = (uintptr_t)x, xend = xb + (size_t)n * w->cin * h * wd * xe;
     const uintptr_t yb = (uintptr_t)y, yend = yb + (size_t)q * w->cout * ye;
@@ -916,7 +918,7 @@ ALCS_API int alcs_spconv1x1_plan(const alcs_packed* w, int n, int h, int wd, uns
 {
     if (!w || !out || n < 0 || h < 0 || wd < 0) return ALCS_ERR_INVALID_ARG;
     if (flags & ~(ALCS_RELU | ALCS_Y_F32)) return ALCS_ERR_INVALID_ARG;
-    if ((flags & ALCS_Y_F32) && w->dt != ALCS_F16) return ALCS_ERR_INVALID_ARG;
+    if ((flags & ALCS_Y_F32) && w->dt == ALCS_F32) return ALCS_ERR_INVALID_ARG;
     if (w->g != 1 && w->g != 2 && w->g != 4 && w->g != 8 && w->g != 16) return ALCS_ERR_UNSUPPORTED;
     if (w->device < 0) return ALCS_ERR_STATE;
     const long long q = (long long)n * h * wd;
@@ -1031,7 +1033,7 @@ ALCS_API size_t alcs_spconv1x1_host_workspace(const alcs_packed* w, int n, int h
 {
     if (!w || n < 0 || h < 0 || wd < 0) return 0;
     const size_t q = (size_t)n * h * wd;
-    const size_t ye = (w->dt == ALCS_F16 && !(flags & ALCS_Y_F32)) ? 2 : 4;
+    const size_t ye = (w->dt != ALCS_F32 && !(flags & ALCS_Y_F32)) ? 2 : 4;
     auto up = [](size_t b) { return (b + 255) / 256 * 256; };
     return up(q * w->cin * w->elt()) + up(q * w->cout * ye) + up((size_t)w->cout * 4);
 }
@@ -1047,7 +1049,7 @@ ALCS_API int alcs_spconv1x1_host(const alcs_packed* w, const void* x_host, void*
     const size_t q = (size_t)n * h * wd;
     if (q == 0) return ALCS_OK;
     if (!x_host || !y_host) return ALCS_ERR_INVALID_ARG;
-    const size_t ye = (w->dt == ALCS_F16 && !(flags & ALCS_Y_F32)) ? 2 : 4;
+    const size_t ye = (w->dt != ALCS_F32 && !(flags & ALCS_Y_F32)) ? 2 : 4;
     auto up = [](size_t b) { return (b + 255) / 256 * 256; };
     const size_t xb = q * w->cin * w->elt(), yb = q * w->cout * ye;
     unsigned char* dx = static_cast<unsigned char*>(workspace);

@@ -135,6 +135,7 @@ namespace alcs {
 
 // Host-side helpers implemented in alcs_pack.cpp (no CUDA).
 float half_bits_to_float(uint16_t h);
+float bfloat16_bits_to_float(uint16_t h);
 void build_schedule(const alcs_packed& p, int kc, int n_rg, bool with_records, Schedule& out);
 void build_schedule_mma(const alcs_packed& p, int kc, int n_rg, bool with_records, Schedule& out);
 int pair_record_bytes(int g);                 // bytes of one pair record

@@ -27,6 +27,7 @@
 #ifndef ALCS_KERNELS_CUH_
 #define ALCS_KERNELS_CUH_
 
+#include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
@@ -187,6 +188,35 @@ struct XVec<__half, 4> {
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
             const float2 f = __half22float2(h[i]);
+            x[2 * i] = f.x;
+            x[2 * i + 1] = f.y;
+        }
+    }
+};
+
+template <>
+struct XVec<__nv_bfloat16, 8> {
+    static __device__ __forceinline__ void load(const unsigned char* p, float (&x)[8])
+    {
+        const uint4 v = *reinterpret_cast<const uint4*>(p);
+        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 f = __bfloat1622float2(h[i]);
+            x[2 * i] = f.x;
+            x[2 * i + 1] = f.y;
+        }
+    }
+};
+template <>
+struct XVec<__nv_bfloat16, 4> {
+    static __device__ __forceinline__ void load(const unsigned char* p, float (&x)[4])
+    {
+        const uint2 v = *reinterpret_cast<const uint2*>(p);
+        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const float2 f = __bfloat1622float2(h[i]);
             x[2 * i] = f.x;
             x[2 * i + 1] = f.y;
         }
@@ -361,10 +391,18 @@ __device__ __forceinline__ void store_vec(YT* p, const float (&v)[VG])
 #pragma unroll
         for (int i = 0; i < VG / 4; ++i)
             reinterpret_cast<float4*>(p)[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-    } else {
+    } else if constexpr (std::is_same<YT, __half>::value) {
         __half2 h[VG / 2];
 #pragma unroll
         for (int i = 0; i < VG / 2; ++i) h[i] = __floats2half2_rn(v[2 * i], v[2 * i + 1]);
+        if constexpr (VG == 8)
+            *reinterpret_cast<uint4*>(p) = *reinterpret_cast<const uint4*>(h);
+        else
+            *reinterpret_cast<uint2*>(p) = *reinterpret_cast<const uint2*>(h);
+    } else {
+        __nv_bfloat162 h[VG / 2];
+#pragma unroll
+        for (int i = 0; i < VG / 2; ++i) h[i] = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
         if constexpr (VG == 8)
             *reinterpret_cast<uint4*>(p) = *reinterpret_cast<const uint4*>(h);
         else
@@ -377,8 +415,10 @@ __device__ __forceinline__ void store_one(YT* p, float v)
 {
     if constexpr (sizeof(YT) == 4)
         *p = v;
-    else
+    else if constexpr (std::is_same<YT, __half>::value)
         *p = __float2half_rn(v);
+    else
+        *p = __float2bfloat16_rn(v);
 }
 
 // The residual operand at the position of a store: VG consecutive elements, or one, widened to fp32.
@@ -391,7 +431,7 @@ __device__ __forceinline__ void load_res_vec(const YT* p, float (&v)[VG])
             const float4 r = __ldg(reinterpret_cast<const float4*>(p) + i);
             v[4 * i] = r.x; v[4 * i + 1] = r.y; v[4 * i + 2] = r.z; v[4 * i + 3] = r.w;
         }
-    } else {
+    } else if constexpr (std::is_same<YT, __half>::value) {
         __half2 h[VG / 2];
         if constexpr (VG == 8)
             *reinterpret_cast<uint4*>(h) = __ldg(reinterpret_cast<const uint4*>(p));
@@ -402,6 +442,17 @@ __device__ __forceinline__ void load_res_vec(const YT* p, float (&v)[VG])
             const float2 f = __half22float2(h[i]);
             v[2 * i] = f.x; v[2 * i + 1] = f.y;
         }
+    } else {
+        __nv_bfloat162 h[VG / 2];
+        if constexpr (VG == 8)
+            *reinterpret_cast<uint4*>(h) = __ldg(reinterpret_cast<const uint4*>(p));
+        else
+            *reinterpret_cast<uint2*>(h) = __ldg(reinterpret_cast<const uint2*>(p));
+#pragma unroll
+        for (int i = 0; i < VG / 2; ++i) {
+            const float2 f = __bfloat1622float2(h[i]);
+            v[2 * i] = f.x; v[2 * i + 1] = f.y;
+        }
     }
 }
 
@@ -410,8 +461,10 @@ __device__ __forceinline__ float load_res_one(const YT* p)
 {
     if constexpr (sizeof(YT) == 4)
         return __ldg(p);
-    else
+    else if constexpr (std::is_same<YT, __half>::value)
         return __half2float(__ldg(p));
+    else
+        return __bfloat162float(__ldg(p));
 }
 
 // ---- producer: one warp copies (item, chunk) after (item, chunk) into the ring ---------------
@@ -863,7 +916,7 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_kernel(const 
             run_epilogue(static_cast<float*>(a.y));
         } else {
             if (a.y_f32) run_epilogue(static_cast<float*>(a.y));
-            else run_epilogue(static_cast<__half*>(a.y));
+            else run_epilogue(static_cast<XT*>(a.y));
         }
     }
 }
@@ -871,7 +924,8 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_kernel(const 
 // One entry of the table of compiled kernel variants.
 // mma = 1: the tensor-core kernel (fp16 only), which takes the step-record flavour of the schedule.
 struct KernelVariant {
-    int is_f16, g, p, rw, nw, minb, npw;
+    int is_f16;     // the alcs_dtype the kernel takes: 0 fp32, 1 binary16, 2 bfloat16
+    int g, p, rw, nw, minb, npw;
     const void* fn;
     int mma;
     int groups;     // consumer groups that take the items of a thread block in turn (1 or 2); nw counts all consumer warps
@@ -889,6 +943,7 @@ const KernelVariant* variants_f32_g4(int* n);
 const KernelVariant* variants_f32_other(int* n);
 const KernelVariant* variants_f16(int* n);
 const KernelVariant* variants_f16_mma(int* n);
+const KernelVariant* variants_bf16(int* n);
 
 }  // namespace alcs
 

@@ -28,6 +28,15 @@ namespace alcs {
 
 void set_cuda_error_text(const char* s) { g_cuda_err = s ? s : ""; }
 
+float bfloat16_bits_to_float(uint16_t h)
+{
+    // bfloat16 -> binary32, exact: the upper half of the binary32 pattern
+    const uint32_t bits = (uint32_t)h << 16;
+    float f;
+    std::memcpy(&f, &bits, 4);
+    return f;
+}
+
 float half_bits_to_float(uint16_t h)
 {
     // binary16 -> binary32, exact.  Handles zeros, subnormals, infinities and NaNs.
@@ -85,7 +94,7 @@ static void emit_pair_records(const alcs_packed& p, int kc, bool with_records, S
         } else {
             uint16_t hb;
             std::memcpy(&hb, &p.vals[vi * 2], 2);
-            v = half_bits_to_float(hb);
+            v = p.dt == ALCS_F16 ? half_bits_to_float(hb) : bfloat16_bits_to_float(hb);
         }
         return v;
     };
@@ -583,7 +592,11 @@ ALCS_API int alcs_schedule_selfcheck(const alcs_packed* p, int chunk_channels, i
                 float v = 0.0f;
                 if (kept) {
                     if (p->dt == ALCS_F32) std::memcpy(&v, &p->vals[((size_t)k * g + j) * 4], 4);
-                    else { uint16_t hb; std::memcpy(&hb, &p->vals[((size_t)k * g + j) * 2], 2); v = alcs::half_bits_to_float(hb); }
+                    else {
+                        uint16_t hb;
+                        std::memcpy(&hb, &p->vals[((size_t)k * g + j) * 2], 2);
+                        v = p->dt == ALCS_F16 ? alcs::half_bits_to_float(hb) : alcs::bfloat16_bits_to_float(hb);
+                    }
                 }
                 const float d = dense[((size_t)r * g + j) * p->cin + c];
                 if (std::memcmp(&d, &v, 4) != 0 && !(d == v)) return ALCS_ERR_CORRUPT;
@@ -626,7 +639,7 @@ ALCS_API int alcs_pack(const void* w, const uint8_t* block_mask, int cout, int c
     if (!w || !block_mask || !out) return ALCS_ERR_INVALID_ARG;
     *out = nullptr;
     if (g < 1 || g > 64) return ALCS_ERR_INVALID_ARG;
-    if (dt != ALCS_F32 && dt != ALCS_F16) return ALCS_ERR_UNSUPPORTED;
+    if (dt != ALCS_F32 && dt != ALCS_F16 && dt != ALCS_BF16) return ALCS_ERR_UNSUPPORTED;
     if (cout <= 0 || cin <= 0) return ALCS_ERR_SHAPE;
     const int rows = (cout + g - 1) / g;
     // count kept blocks first so that overflow is detected before anything is allocated
@@ -731,7 +744,7 @@ ALCS_API int alcs_packed_deserialize(const void* buf, size_t nbytes, alcs_packed
     std::memcpy(&h, buf, sizeof h);
     if (h.magic != kMagic || h.version != kBlobVersion) return ALCS_ERR_CORRUPT;
     if (h.cout <= 0 || h.cin <= 0 || h.g < 1 || h.g > 64 || h.nb < 0) return ALCS_ERR_CORRUPT;
-    if (h.dtype != ALCS_F32 && h.dtype != ALCS_F16) return ALCS_ERR_CORRUPT;
+    if (h.dtype != ALCS_F32 && h.dtype != ALCS_F16 && h.dtype != ALCS_BF16) return ALCS_ERR_CORRUPT;
     if (h.rows != (h.cout + h.g - 1) / h.g) return ALCS_ERR_CORRUPT;
     if ((uint64_t)h.nb > (uint64_t)h.rows * (uint64_t)h.cin) return ALCS_ERR_CORRUPT;
     const size_t es = h.dtype == ALCS_F32 ? 4 : 2;

@@ -84,3 +84,20 @@ def test_long_rows_are_split_into_parts():
     assert st["nb"] == int(M.sum())
     uniform = A.alcs_schedule_selfcheck(A.alcs_pack(*_matrix(4, 512, 512, 4, 0.25), 4), 64, 6, 12, 2)
     assert uniform["secondary_units"] == 0
+
+
+def test_bfloat16_weights_pack_and_schedule():
+    """bfloat16 weights travel as bit patterns: pack -> unpack and the serialised blob return them bit for
+    bit, and the schedule (which widens them to fp32 exactly) passes the walk check."""
+    g = 8
+    W = rng.to_bf16_bits(rng.normal(8, 1, 64 * 48).astype(np.float32)).reshape(64, 48)
+    M = (rng.uniform01(8, 3, 8 * 48) < 0.4).astype(np.uint8).reshape(8, 48)
+    p = A.alcs_pack(W, M, g, bf16=True)
+    W2, M2 = A.alcs_unpack(p)
+    assert W2.dtype == np.uint16 and np.array_equal(M2, M)
+    assert np.array_equal(W2, W * np.repeat(M, g, axis=0).astype(np.uint16))
+    q = A.alcs_packed_deserialize(A.alcs_packed_serialize(p))
+    assert np.array_equal(A.alcs_unpack(q)[0], W2)
+    A.alcs_schedule_selfcheck(p, 16, 1, 4, 2)
+    with pytest.raises(TypeError):
+        A.alcs_pack(W.astype(np.float64), M, g)

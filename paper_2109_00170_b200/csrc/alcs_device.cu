@@ -479,6 +479,9 @@ __global__ void repack_rows_kernel(const T* __restrict__ in, T* __restrict__ out
                                    int ow, int stride, int hw_out, int hwp)
 {
     constexpr int EPV = 16 / (int)sizeof(T);
+    // The convolution kernel behind this one on the stream may set up (barriers, schedule bounds) while
+    // the copy runs; it waits for this grid to finish before it touches the scratch.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int vpr = hwp / EPV;                       // 16-byte pieces per padded row
     const long long total = rows * vpr;
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
@@ -629,7 +632,7 @@ int launch_plan(const alcs_packed* w, const Plan& p, const void* x, void* y, int
         if (have) {
             void* const xpad = scratch ? scratch : w->d_xpad;
             const long long rows = (long long)n * w->cin;
-            const unsigned blocks = (unsigned)std::min<long long>((rows * (hwp * elt / 16) + 255) / 256, (long long)di.sms * 16);
+            const unsigned blocks = (unsigned)std::min<long long>((rows * (hwp * elt / 16) + 255) / 256, (long long)di.sms * 8);     // one wave of 256-thread blocks
             if (elt == 4)
                 repack_rows_kernel<float><<<blocks, 256, 0, st>>>(static_cast<const float*>(x), static_cast<float*>(xpad), rows,
                                                                   h_in * wd_in, wd_in, wd, stride, hw, hwp);

@@ -284,6 +284,18 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_mma_kernel(co
                                     const __half* src = rbase + yoff[gi] + (size_t)co * a.hwy;
                                     if constexpr (VG == 8) *reinterpret_cast<uint4*>(wp) = __ldg(reinterpret_cast<const uint4*>(src));
                                     else *reinterpret_cast<uint2*>(wp) = __ldg(reinterpret_cast<const uint2*>(src));
+                                } else if (!a.st_vec && a.st_grp) {
+                                    // the run lies in one image (padded rows are a multiple of VG long); its
+                                    // pixels p >= hwy exist only as padding of the repacked X
+                                    const int nreal = (have && yok[gi]) ? a.hwy - yp[gi] : 0;
+                                    const __half* src = rbase + yoff[gi] + (size_t)co * a.hwy;
+                                    if (nreal >= VG && (reinterpret_cast<uintptr_t>(src) & (2 * VG - 1)) == 0) {
+                                        if constexpr (VG == 8) *reinterpret_cast<uint4*>(wp) = __ldg(reinterpret_cast<const uint4*>(src));
+                                        else *reinterpret_cast<uint2*>(wp) = __ldg(reinterpret_cast<const uint2*>(src));
+                                    } else {
+#pragma unroll
+                                        for (int t = 0; t < VG; ++t) hw16[t] = t < nreal ? __ldg(src + t) : __float2half_rn(0.0f);
+                                    }
                                 } else {
                                     int nn = yn[gi], pp = yp[gi];
 #pragma unroll
@@ -332,6 +344,26 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_mma_kernel(co
                                 __half* dst = ybase + yoff[gi] + (size_t)co * a.hwy;
                                 if constexpr (VG == 8) *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(rp);
                                 else *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(rp);
+                            } else if (a.st_grp) {
+                                // the run lies in one image: one vector store where all its pixels are real
+                                // and the address allows it (two halves for a 16-byte run on an 8-byte
+                                // boundary), single elements otherwise
+                                if (!yok[gi]) continue;
+                                __half* dst = ybase + yoff[gi] + (size_t)co * a.hwy;
+                                const int nreal = a.hwy - yp[gi];
+                                const uintptr_t ad = reinterpret_cast<uintptr_t>(dst);
+                                if (nreal >= VG && (ad & (2 * VG - 1)) == 0) {
+                                    if constexpr (VG == 8) *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(rp);
+                                    else *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(rp);
+                                } else if (VG == 8 && nreal >= VG && (ad & 7) == 0) {
+                                    *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(rp);
+                                    *reinterpret_cast<uint2*>(dst + 4) = *reinterpret_cast<const uint2*>(rp + 8);
+                                } else {
+                                    const __half* hp = reinterpret_cast<const __half*>(rp);
+#pragma unroll
+                                    for (int t = 0; t < VG; ++t)
+                                        if (t < nreal) dst[t] = hp[t];
+                                }
                             } else {
                                 // element by element: the run may cross into the next image, and pixels
                                 // p >= hwy exist only as padding of the repacked X

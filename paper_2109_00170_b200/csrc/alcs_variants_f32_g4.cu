@@ -12,6 +12,8 @@ static const KernelVariant kTable[] = {
     ALCS_VARIANT_P(float, 0, 4, 8, 4, 7, 1, 1),
     ALCS_VARIANT_P(float, 0, 4, 8, 4, 6, 1, 2),
     ALCS_VARIANT_P(float, 0, 4, 8, 1, 7, 2, 1),
+    ALCS_VARIANT_P(float, 0, 4, 8, 2, 7, 2, 1),
+    ALCS_VARIANT_P(float, 0, 4, 8, 2, 6, 2, 2),
     ALCS_VARIANT_P(float, 0, 4, 8, 1, 11, 1, 1),
     ALCS_VARIANT_P(float, 0, 4, 8, 2, 11, 1, 1),
     ALCS_VARIANT_P(float, 0, 4, 8, 3, 11, 1, 1),

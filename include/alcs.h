@@ -163,7 +163,11 @@ ALCS_API void alcs_packed_free(alcs_packed* p);
  *   row_groups        how many work items share one pixel tile, each taking a subset of rows
  *   min_blocks        thread blocks per SM the kernel is compiled for (1 or 2)
  *   copy_mode         how X tiles reach shared memory: 1 = per-lane cp.async, 2 = bulk (TMA) copies
- *                     of whole pixel runs (needs 16-byte aligned rows; otherwise 1 is used)
+ *                     of whole pixel runs (needs 16-byte aligned rows; otherwise 1 is used).  Image rows
+ *                     that are not a multiple of 16 bytes long are first repacked into a scratch tensor
+ *                     with padded rows; 3 = per-lane cp.async of 8 bytes straight from X, without that
+ *                     pass, for rows that are a multiple of 8 but not of 16 bytes long (16-bit elements,
+ *                     14x14 images), stride 1 and X on an 8-byte boundary; elsewhere 3 acts like 1
  *   producer_warps    warps of the thread block that only move data (1..4)
  *   math_mode         1 = fp32 FMA on the CUDA cores; 2 = tensor cores (fp16 weights and activations
  *                     only): 16 kept blocks of a block row times the 16 input rows they select is a
@@ -264,7 +268,9 @@ ALCS_API int alcs_spconv1x1_plan(const alcs_packed* w, int n, int h, int wd, uns
  * alcs_spconv1x1_tune: time the candidate launch configurations for this shape on the given
  * buffers (y is overwritten with the correct result each time), remember the fastest in w for
  * later alcs_spconv1x1 calls with the same (n, h, wd, flags), and write it to *best (may be
- * NULL).  Synchronises the stream; meant for set-up time, never for the timed path.
+ * NULL).  Every launch is timed with cold caches (a buffer larger than L2 is rewritten before it):
+ * each candidate three times, then the eight best fifteen times more in turn, and the lowest median
+ * wins.  Synchronises the stream; meant for set-up time, never for the timed path.
  */
 ALCS_API int alcs_spconv1x1_tune(alcs_packed* w, const void* x, void* y, int n, int h, int wd,
                         const float* bias, unsigned flags, void* cuda_stream,

@@ -291,6 +291,10 @@ bool gather_plan(const alcs_packed* w, int n, int hw, int p, int ks, const Devic
     return true;
 }
 
+// Can the producers stage the rows of X as they are, with 8-byte copies, where 16-byte copies would need
+// the rows repacked?
+bool direct_rows_ok(int hw, int elt) { return ((size_t)hw * elt) % 16 == 8; }
+
 // Enumerate every valid launch configuration for this shape, cheapest (by the model) first.
 // Internal flag, only ever seen in plan-cache keys: the call has a residual operand or a stride, which
 // the small-problem kernel does not take, so only the staged kernels are listed.
@@ -361,6 +365,14 @@ int enumerate_plans(const alcs_packed* w, long long q, int hw, std::vector<Plan>
                         p2.cost *= 1.25;
                         out.push_back(p2);
                     }
+                    // Rows that are a multiple of 8 but not of 16 bytes long (16-bit 14x14 images) can also be
+                    // staged as they are, with 8-byte copies: twice the copy instructions, no repacking pass.
+                    if (direct_rows_ok(hw, elt)) {
+                        Plan p3 = p;
+                        p3.bulk = 2;
+                        p3.cost *= 1.1;
+                        out.push_back(p3);
+                    }
                 }
             }
         }
@@ -393,7 +405,7 @@ void plan_to_cfg(const Plan& p, alcs_launch_cfg* c)
     c->stages = p.stages;
     c->row_groups = p.n_rg;
     c->min_blocks = v.minb;
-    c->copy_mode = p.bulk ? 2 : 1;
+    c->copy_mode = p.bulk + 1;
     c->producer_warps = v.npw;
     c->math_mode = mode_of(v);
     c->consumer_groups = v.groups;
@@ -434,7 +446,10 @@ int cfg_to_plan(const alcs_packed* w, long long q, int hw, const alcs_launch_cfg
         if (c->split_rows && (c->split_rows == 1) != (v.split == 1)) return false;
         if (c->chunk_channels && std::min(c->chunk_channels, w->cin) != p.kc) return false;
         if (c->stages && c->stages != p.stages) return false;
-        if (c->copy_mode && (c->copy_mode == 2) != (p.bulk == 1)) return false;
+        if (c->copy_mode) {     // (3 where the rows cannot be staged as they are: like 1)
+            const int want = (c->copy_mode == 3 && !direct_rows_ok(hw, (int)w->elt())) ? 1 : c->copy_mode;
+            if (want != p.bulk + 1) return false;
+        }
         return true;
     };
     for (const Plan& p : all)
@@ -623,7 +638,8 @@ int launch_plan(const alcs_packed* w, const Plan& p, const void* x, void* y, int
     // Rows of X that are not a multiple of 16 bytes long: repack X into scratch with padded rows.
     int hwx = hw;
     const void* xk = x;
-    if (((size_t)hw * elt) % 16 != 0 || stride != 1) {
+    const bool direct = p.bulk == 2 && stride == 1 && direct_rows_ok(hw, elt) && (uintptr_t)x % 8 == 0;
+    if ((((size_t)hw * elt) % 16 != 0 && !direct) || stride != 1) {
         const int hwp = padded_hw(hw, elt);
         const size_t need = (size_t)n * w->cin * hwp * elt;
         if (scratch && scratch_bytes < need) return ALCS_ERR_STATE;
@@ -665,7 +681,7 @@ int launch_plan(const alcs_packed* w, const Plan& p, const void* x, void* y, int
     int ld = 16;
     while (ld > elt && (((size_t)hwx * elt) % ld || (uintptr_t)xk % ld)) ld >>= 1;
     a.ld_bytes = ld;
-    a.bulk = (ld == 16 && p.bulk) ? 1 : 0;
+    a.bulk = (ld == 16 && p.bulk == 1) ? 1 : 0;
     a.ros = sc->ros;
     const int vg = (v.p * elt >= 16) ? 16 / elt : v.p;
     a.st_vec = (hwx == hw && hw % vg == 0 && (uintptr_t)y % 16 == 0 && (uintptr_t)residual % 16 == 0) ? 1 : 0;
@@ -965,23 +981,48 @@ ALCS_API int alcs_spconv1x1_tune(alcs_packed* w, const void* x, void* y, int n, 
         alcs::set_cuda_error_text("cudaEventCreate failed");
         return ALCS_ERR_CUDA;
     }
-    int best_i = -1;
-    float best_ms = 1e30f;
+    // one cold-cache launch of candidate i, in milliseconds (negative: the launch failed)
+    auto time_once = [&](size_t i, int fill) -> float {
+        if (flush) cudaMemsetAsync(flush, fill, flush_bytes, st);
+        cudaEventRecord(e0, st);
+        const bool ok = launch_plan(w, all[i], x, y, n, h, wd, bias, flags, st) == ALCS_OK;
+        cudaEventRecord(e1, st);
+        if (cudaEventSynchronize(e1) != cudaSuccess || !ok) return -1.0f;
+        float ms = 0;
+        cudaEventElapsedTime(&ms, e0, e1);
+        return ms;
+    };
+    // First pass: every candidate, the best of `reps` launches after one untimed launch.
     const int reps = 3;
+    std::vector<std::pair<float, int>> ranked;
     for (size_t i = 0; i < all.size(); ++i) {
         float tmin = 1e30f;
         bool ok = true;
         for (int r = 0; r < reps + 1 && ok; ++r) {
-            if (flush) cudaMemsetAsync(flush, r, flush_bytes, st);
-            cudaEventRecord(e0, st);
-            ok = launch_plan(w, all[i], x, y, n, h, wd, bias, flags, st) == ALCS_OK;
-            cudaEventRecord(e1, st);
-            if (cudaEventSynchronize(e1) != cudaSuccess) { ok = false; break; }
-            float ms = 0;
-            cudaEventElapsedTime(&ms, e0, e1);
-            if (r > 0) tmin = std::min(tmin, ms);
+            const float ms = time_once(i, r);
+            ok = ms >= 0;
+            if (r > 0 && ok) tmin = std::min(tmin, ms);
         }
-        if (ok && tmin < best_ms) { best_ms = tmin; best_i = (int)i; }
+        if (ok) ranked.emplace_back(tmin, (int)i);
+    }
+    // Second pass: the few best candidates differ by less than the noise of three launches, so they
+    // are timed again, in turn, and the one with the lowest median wins.
+    std::sort(ranked.begin(), ranked.end());
+    if (ranked.size() > 8) ranked.resize(8);
+    int best_i = -1;
+    float best_ms = 1e30f;
+    const int rounds = 15;
+    std::vector<std::vector<float>> samples(ranked.size());
+    for (int r = 0; r < rounds; ++r)
+        for (size_t f = 0; f < ranked.size(); ++f) {
+            const float ms = time_once((size_t)ranked[f].second, r);
+            if (ms >= 0) samples[f].push_back(ms);
+        }
+    for (size_t f = 0; f < ranked.size(); ++f) {
+        if (samples[f].size() < (size_t)rounds) continue;
+        std::nth_element(samples[f].begin(), samples[f].begin() + rounds / 2, samples[f].end());
+        const float med = samples[f][rounds / 2];
+        if (med < best_ms) { best_ms = med; best_i = ranked[f].second; }
     }
     cudaError_t e = cudaStreamSynchronize(st);
     cleanup();
@@ -1245,7 +1286,8 @@ extern "C" ALCS_API int alcs_spconv1x1_noalloc(const alcs_packed* w, const void*
     const int hw = h * wd;
     int hwx = hw;
     const void* xk = x;
-    if (((size_t)hw * elt) % 16 != 0) {
+    const bool direct = plan.bulk == 2 && direct_rows_ok(hw, elt) && (uintptr_t)x % 8 == 0;
+    if (((size_t)hw * elt) % 16 != 0 && !direct) {
         // rows that cannot be staged with 16-byte copies: repack into the fixed array
         const int hwp = padded_hw(hw, elt);
         const unsigned long long need = (unsigned long long)n * w->cin * hwp * elt;
@@ -1288,7 +1330,7 @@ extern "C" ALCS_API int alcs_spconv1x1_noalloc(const alcs_packed* w, const void*
     int ld = 16;
     while (ld > elt && (((size_t)hwx * elt) % ld || (uintptr_t)xk % ld)) ld >>= 1;
     a.ld_bytes = ld;
-    a.bulk = (ld == 16 && plan.bulk) ? 1 : 0;
+    a.bulk = (ld == 16 && plan.bulk == 1) ? 1 : 0;
     a.ros = sc->ros;
     const int vg = (v.p * elt >= 16) ? 16 / elt : v.p;
     a.st_vec = (hwx == hw && hw % vg == 0 && (uintptr_t)y % 16 == 0) ? 1 : 0;

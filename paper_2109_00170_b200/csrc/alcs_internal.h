@@ -79,7 +79,7 @@ struct Plan {
     int kc = 0;            // schedule key: channels per chunk ...
     int n_rg = 0;          // ... and number of row groups
     int stages = 0;
-    int bulk = 0;          // 1: bulk (TMA) copies of X, 0: per-lane cp.async
+    int bulk = 0;          // 0: per-lane cp.async, 1: bulk (TMA) copies of X, 2: per-lane cp.async from rows that are not repacked
     int occ = 1;           // resident thread blocks per SM
     size_t smem = 0;
     double cost = 0;       // model estimate, seconds

@@ -71,6 +71,10 @@ def test_fp16_stride_and_residual(alcs, n, cin, cout, h, wd, g, stride, math_mod
     _check(alcs, W, M, X, b, R, False, g, stride, "f16", cfg=cfg)
     R32 = R.astype(np.float32)
     _check(alcs, W, M, X, b, R32, True, g, stride, "f16", cfg=cfg, y_f32=True)
+    # rows staged without the repacking pass where they allow it (14x14 at stride 1), else as before
+    direct = dict(math_mode=math_mode, copy_mode=3)
+    _check(alcs, W, M, X, b, R, True, g, stride, "f16", cfg=direct)
+    _check(alcs, W, M, X, b, R32, False, g, stride, "f16", cfg=direct, y_f32=True)
 
 
 def test_residual_is_added_before_the_activation_exactly(alcs):

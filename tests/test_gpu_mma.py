@@ -46,6 +46,17 @@ def test_epilogue_and_copy_modes(alcs, copy_mode, relu, with_bias):
     check_layer(alcs, W, M, X, b if with_bias else None, relu, 8, cfg=dict(math_mode=2, copy_mode=copy_mode))
 
 
+@pytest.mark.parametrize("math_mode", [1, 2])
+@pytest.mark.parametrize("n,cin,cout,hw", [(5, 136, 72, 196), (3, 70, 40, 12), (2, 64, 32, 400), (2, 48, 24, 49)])
+@pytest.mark.parametrize("y_f32", [False, True])
+def test_unpadded_rows_staged_directly(alcs, math_mode, n, cin, cout, hw, y_f32):
+    """copy_mode 3: rows that are a multiple of 8 but not of 16 bytes long (hw = 196, 12) are staged as
+    they are, with 8-byte copies, by the tensor-core and by the CUDA-core fp16 kernels; for the other
+    row lengths the mode must behave like copy_mode 1."""
+    W, M, X, b = _rand(700 + hw, n, cin, cout, hw, 8, 0.3, xpos=False)
+    check_layer(alcs, W, M, X, b, True, 8, cfg=dict(math_mode=math_mode, copy_mode=3), y_f32=y_f32)
+
+
 def test_dense_empty_and_ragged_rows(alcs):
     """0 % sparsity, 100 % sparsity (bias only), and rows with 0, 1, 15, 16, 17 and 33 kept blocks
     (below, at and above one 16-block step)."""

@@ -686,6 +686,9 @@ int launch_plan(const alcs_packed* w, const Plan& p, const void* x, void* y, int
     const int vg = (v.p * elt >= 16) ? 16 / elt : v.p;
     a.st_vec = (hwx == hw && hw % vg == 0 && (uintptr_t)y % 16 == 0 && (uintptr_t)residual % 16 == 0) ? 1 : 0;
     a.st_grp = hwx % vg == 0 ? 1 : 0;
+    // 16-bit rows of Y that do not all start on an 8-byte boundary (7x7 images): nothing wider than one
+    // element can be stored, and the tensor-core kernel then lets consecutive lanes take consecutive pixels
+    if (v.mma && !a.y_f32 && !a.st_vec && ((size_t)hw * elt) % 8 != 0) a.st_grp = 2;
     const long long items = (long long)a.n_tiles * a.n_rg;
     if (items > 0x7fffffffll) return ALCS_ERR_SHAPE;
     // persistent thread blocks: as many as can be resident, each walks items with that stride
@@ -1335,6 +1338,7 @@ extern "C" ALCS_API int alcs_spconv1x1_noalloc(const alcs_packed* w, const void*
     const int vg = (v.p * elt >= 16) ? 16 / elt : v.p;
     a.st_vec = (hwx == hw && hw % vg == 0 && (uintptr_t)y % 16 == 0) ? 1 : 0;
     a.st_grp = hwx % vg == 0 ? 1 : 0;
+    if (v.mma && !a.y_f32 && !a.st_vec && ((size_t)hw * elt) % 8 != 0) a.st_grp = 2;
     const long long items = (long long)a.n_tiles * a.n_rg;
     if (items > 0x7fffffffll) return ALCS_ERR_SHAPE;
     const long long grid = std::min<long long>(items, (long long)di.sms * std::max(1, plan.occ));

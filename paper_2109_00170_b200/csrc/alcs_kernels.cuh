@@ -74,7 +74,8 @@ struct ConvArgs {
     int bulk;                 // 1: the producer uses bulk (TMA) copies; needs ld_bytes == 16
     int ros;                  // ints of rowoff per (row group, chunk): 4 per header
     int st_vec;               // 1 if vector stores are allowed
-    int st_grp;               // 1 if the pixels of one vector store of a lane always lie in one image
+    int st_grp;               // 1 if the pixels of one vector store of a lane always lie in one image; 2 (tensor-core
+                              // kernel, 16-bit output): store single elements, consecutive lanes on consecutive pixels
     // shared-memory layout (bytes): [mbarriers | stage 0 | stage 1 | ...]
     int off_rec, off_rowoff, stage_bytes;
 };

@@ -284,7 +284,7 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_mma_kernel(co
                                     const __half* src = rbase + yoff[gi] + (size_t)co * a.hwy;
                                     if constexpr (VG == 8) *reinterpret_cast<uint4*>(wp) = __ldg(reinterpret_cast<const uint4*>(src));
                                     else *reinterpret_cast<uint2*>(wp) = __ldg(reinterpret_cast<const uint2*>(src));
-                                } else if (!a.st_vec && a.st_grp) {
+                                } else if (!a.st_vec && a.st_grp == 1) {
                                     // the run lies in one image (padded rows are a multiple of VG long); its
                                     // pixels p >= hwy exist only as padding of the repacked X
                                     const int nreal = (have && yok[gi]) ? a.hwy - yp[gi] : 0;
@@ -332,6 +332,25 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_mma_kernel(co
                         stmatrix_x4_trans(st_addr + mp * 64, r[0], r[1], r[2], r[3]);
                     }
                     __syncwarp();
+                    if (a.st_grp == 2) {
+                        // element-wise stores: lane l of pass k writes pixel k*32 + l of the tile, so that a
+                        // warp's store covers consecutive addresses wherever the pixels lie in one image
+#pragma unroll 1
+                        for (int k = 0; k < P; ++k) {
+                            const int q = q0 + k * 32 + lane;
+                            const int nn = q / a.hw;
+                            const int pp = q - nn * a.hw;
+                            if (q >= a.q_total || pp >= a.hwy) continue;
+                            __half* dst = ybase + (size_t)nn * a.cout * a.hwy + pp;
+                            const __half* hp = reinterpret_cast<const __half*>(scratch) + k * 32 + lane;
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                const int co = rowid[s] * G + nb * 8 + j;
+                                if (nb * 8 + j < G && co < a.cout) dst[(size_t)co * a.hwy] = hp[j * (SCRB / 2)];
+                            }
+                        }
+                        continue;
+                    }
 #pragma unroll 2
                     for (int j = 0; j < 8; ++j) {
                         const int co = rowid[s] * G + nb * 8 + j;
@@ -344,7 +363,7 @@ __global__ void __launch_bounds__((NW + NPW) * 32, MINB) spconv1x1_mma_kernel(co
                                 __half* dst = ybase + yoff[gi] + (size_t)co * a.hwy;
                                 if constexpr (VG == 8) *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(rp);
                                 else *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(rp);
-                            } else if (a.st_grp) {
+                            } else if (a.st_grp == 1) {
                                 // the run lies in one image: one vector store where all its pixels are real
                                 // and the address allows it (two halves for a 16-byte run on an 8-byte
                                 // boundary), single elements otherwise

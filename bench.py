@@ -240,6 +240,8 @@ def measure_batch1(A, torch, dev, stream, steps, hbm_gbs, fp32_tf):
         flops += fl
         t_roof += max(fl / (fp32_tf * 1e12), by / (hbm_gbs * 1e9))
     stack = A.alcs_stack_create(layers, A.ALCS_STACK_GRAPH)
+    with torch.cuda.stream(stream):
+        A.alcs_stack_tune(stack, 0, stream)
     for _ in range(5):
         A.alcs_stack_run(stack, stream)
     torch.cuda.synchronize()
@@ -591,13 +593,22 @@ def main():
         stats.append(dict(name=s.name, nb=nb, sparsity=1 - nb / M.size, flops=fl, bytes=by, cfg=cfg))
         host.append((X, b))
         keep.append((W, M))
+    stack = None if args.cfg else A.alcs_stack_create(layers, A.ALCS_STACK_GRAPH if graph else 0)
+    stack_tune_us = None
+    if tuned_now and stack is not None:
+        # second tuning step, in context: the layers' best few configurations are tried inside the
+        # whole stack (dependent launches, the cache state the other layers leave behind)
+        with torch.cuda.stream(stream):
+            stack_tune_us = A.alcs_stack_tune(stack, 0, stream)
+        for i, st_ in enumerate(stats):
+            if st_["name"] in tuned_now:
+                st_["cfg"] = tuned_now[st_["name"]] = A.alcs_stack_layer_cfg(stack, i)
     if tuned_now and rank == 0 and not args.layers:
         try:
             os.makedirs(os.path.dirname(cache_path), exist_ok=True)
             json.dump({"source_hash": kernel_source_hash(), "layers": {**cache, **tuned_now}}, open(cache_path, "w"), indent=1)
         except OSError:
             pass
-    stack = None if args.cfg else A.alcs_stack_create(layers, A.ALCS_STACK_GRAPH if graph else 0)
 
     def run_stack():
         if stack is not None:
@@ -742,7 +753,8 @@ def main():
         "config": {"workload": wl, "layers": nl, "batch": specs[0].n, "g": specs[0].g,
                    "cache": "inputs larger than L2: one step touches %.0f MB of distinct X and Y" % (total_bytes / 1e6),
                    "cuda_graph": graph, "tuned": not args.no_tune,
-                   "launch_cfgs": "forced" if args.cfg else ("tuning cache" if cache else ("tuned in this run" if not args.no_tune else "model"))},
+                   "launch_cfgs": "forced" if args.cfg else ("tuning cache" if cache else ("tuned in this run" if not args.no_tune else "model")),
+                   "stack_tune_us": [round(v, 2) for v in stack_tune_us] if stack_tune_us else None},
         "roofline": roof,
         "stack_roofline": {"sum_t_roof_us": round(sum_roof, 1), "sum_layer_us": round(sum_us, 1),
                            "frac": round(sum_roof / sum_us, 4), "min_layer_frac": min(r["frac"] for r in rows),

@@ -504,6 +504,25 @@ ALCS_API int alcs_stack_create(const alcs_layer* layers, int n_layers, unsigned 
 ALCS_API int alcs_stack_run(alcs_stack* s, void* cuda_stream);
 ALCS_API int alcs_stack_destroy(alcs_stack* s);
 
+/*
+ * alcs_stack_tune: choose the layers' launch configurations IN CONTEXT.  alcs_spconv1x1_tune times a layer
+ * alone, with cold caches and nothing before it on the stream; inside a stack a layer starts while its
+ * predecessor drains (programmatic dependent launch), finds whatever the earlier layers left in L2, and, at
+ * batch 1, costs little more than its launch, so the configuration that wins alone is not always the one
+ * that wins there.  For every layer in turn this call tries the candidates (the best eight of the last
+ * alcs_spconv1x1_tune for the layer's shape if there was one, else the cost model's best eight and every
+ * shape of the small-problem kernel that applies), each time timing the WHOLE stack the way alcs_stack_run
+ * runs it (a graph stack is captured again), and keeps a candidate only if the stack gets faster by more
+ * than 0.4 %; `passes` sweeps over the layers (0 = 2), stopping early when a sweep changes nothing.  The
+ * chosen configurations are also remembered in the packed matrices for later calls with the same shape.
+ * us_before / us_after (may be NULL): microseconds per pass over the stack before and after.  The layers'
+ * outputs are overwritten many times with the same correct values.  Synchronises the stream; set-up time
+ * only.  alcs_stack_layer_cfg reports the configuration layer `layer` (0-based) of the stack uses now (all
+ * zero for an empty layer).
+ */
+ALCS_API int alcs_stack_tune(alcs_stack* s, int passes, void* cuda_stream, double* us_before, double* us_after);
+ALCS_API int alcs_stack_layer_cfg(const alcs_stack* s, int layer, alcs_launch_cfg* out);
+
 #ifdef __cplusplus
 }
 #endif

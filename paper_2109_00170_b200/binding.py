@@ -30,7 +30,7 @@ EXPORTS = ["alcs_strerror", "alcs_last_cuda_error", "alcs_version", "alcs_pack",
            "alcs_spconv1x1_plan", "alcs_spconv1x1_tune", "alcs_spconv1x1_set_cfg", "alcs_spconv1x1_host_workspace",
            "alcs_spconv1x1_host", "alcs_spconv1x1_noalloc", "alcs_spconv2d", "alcs_spconv2d_cfg", "alcs_spconv2d_plan", "alcs_layer_latency", "alcs_network_latency",
            "alcs_project_bisection", "alcs_probe_fma_peak", "alcs_probe_lds", "alcs_probe_segment_loop",
-           "alcs_stack_create", "alcs_stack_run", "alcs_stack_destroy"]
+           "alcs_stack_create", "alcs_stack_run", "alcs_stack_destroy", "alcs_stack_tune", "alcs_stack_layer_cfg"]
 
 
 class AlcsError(RuntimeError):
@@ -134,6 +134,8 @@ def lib():
     L.alcs_stack_create.argtypes = [C.POINTER(Layer), i, u, C.POINTER(vp)]
     L.alcs_stack_run.argtypes = [vp, vp]
     L.alcs_stack_destroy.argtypes = [vp]
+    L.alcs_stack_tune.argtypes = [vp, i, vp, C.POINTER(C.c_double), C.POINTER(C.c_double)]
+    L.alcs_stack_layer_cfg.argtypes = [vp, i, C.POINTER(LaunchCfg)]
     for name in EXPORTS:
         f = getattr(L, name)
         if f.restype is C.c_int and name not in ("alcs_version",):
@@ -494,6 +496,20 @@ def alcs_stack_create(layers: Sequence[dict], stack_flags: int = 0) -> Stack:
 
 def alcs_stack_run(s: Stack, stream=None):
     _check(lib().alcs_stack_run(s.handle, _stream(stream)), "alcs_stack_run")
+
+
+def alcs_stack_tune(s: Stack, passes: int = 0, stream=None):
+    """Choose the layers' launch configurations in the context of the whole stack; returns
+    (microseconds per pass before, after)."""
+    before, after = C.c_double(0.0), C.c_double(0.0)
+    _check(lib().alcs_stack_tune(s.handle, passes, _stream(stream), C.byref(before), C.byref(after)), "alcs_stack_tune")
+    return before.value, after.value
+
+
+def alcs_stack_layer_cfg(s: Stack, layer: int) -> dict:
+    c = LaunchCfg()
+    _check(lib().alcs_stack_layer_cfg(s.handle, layer, C.byref(c)), "alcs_stack_layer_cfg")
+    return c.as_dict()
 
 
 def alcs_stack_destroy(s: Stack):

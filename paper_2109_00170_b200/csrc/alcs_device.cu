@@ -602,6 +602,13 @@ int launch_gather_plan(const alcs_packed* w, const Plan& p, const void* x, void*
     a.tiles = (a.hw + 32 * p.gp - 1) / (32 * p.gp);
     a.relu = (flags & ALCS_RELU) ? 1 : 0;
     a.vec = (p.gp >= 4 && a.hw % 4 == 0 && (uintptr_t)x % 16 == 0) ? 1 : 0;
+    int longest = w->max_row_blocks;        // (no lock: a caller may hold w->mu, and every thread computes the same value)
+    if (longest < 0) {
+        longest = 0;
+        for (int r = 0; r < w->rows; ++r) longest = std::max(longest, w->row_ptr[r + 1] - w->row_ptr[r]);
+        w->max_row_blocks = longest;
+    }
+    a.stage_blocks = alcs::gather_stage_blocks(w->g, longest);
     ALCS_CUDA(alcs::launch_gather(w->g, p.gp, p.gks, a, st));
     return ALCS_OK;
 }
@@ -1021,12 +1028,15 @@ ALCS_API int alcs_spconv1x1_tune(alcs_packed* w, const void* x, void* y, int n, 
             const float ms = time_once((size_t)ranked[f].second, r);
             if (ms >= 0) samples[f].push_back(ms);
         }
+    std::vector<std::pair<float, int>> by_median;
     for (size_t f = 0; f < ranked.size(); ++f) {
         if (samples[f].size() < (size_t)rounds) continue;
         std::nth_element(samples[f].begin(), samples[f].begin() + rounds / 2, samples[f].end());
         const float med = samples[f][rounds / 2];
+        by_median.emplace_back(med, ranked[f].second);
         if (med < best_ms) { best_ms = med; best_i = ranked[f].second; }
     }
+    std::sort(by_median.begin(), by_median.end());
     cudaError_t e = cudaStreamSynchronize(st);
     cleanup();
     if (e != cudaSuccess) { alcs::set_cuda_error_text(cudaGetErrorString(e)); return ALCS_ERR_CUDA; }
@@ -1037,6 +1047,9 @@ ALCS_API int alcs_spconv1x1_tune(alcs_packed* w, const void* x, void* y, int n, 
         std::lock_guard<std::mutex> lk(w->mu);
         w->tuned[alcs::ShapeKey{n, h, wd, flags}] = c;
         w->plan_cache[alcs::ShapeKey{n, h, wd, flags}] = all[best_i];
+        std::vector<Plan>& fin = w->finalists[alcs::ShapeKey{n, h, wd, flags}];
+        fin.clear();
+        for (const auto& m : by_median) fin.push_back(all[m.second]);
     }
     {   // release the device copies of the schedules that did not win
         std::lock_guard<std::mutex> lk(w->mu);
@@ -1207,6 +1220,137 @@ ALCS_API int alcs_stack_run(alcs_stack* s, void* cuda_stream)
         }
     }
     ALCS_CUDA(cudaGraphLaunch(s->exec, st));
+    return ALCS_OK;
+}
+
+namespace {
+
+bool same_plan(const Plan& a, const Plan& b)
+{
+    return a.variant == b.variant && a.kc == b.kc && a.n_rg == b.n_rg && a.stages == b.stages && a.bulk == b.bulk &&
+           a.gather == b.gather && a.gp == b.gp && a.gks == b.gks;
+}
+
+// Run time of one pass over the whole stack in microseconds, as alcs_stack_run runs it (a graph stack
+// is captured again with the plans it holds now): the best of three batches of `reps` runs after two
+// untimed ones.  Negative if a launch failed.
+double time_stack(alcs_stack* s, cudaStream_t st, cudaEvent_t e0, cudaEvent_t e1, int reps)
+{
+    if (s->exec) { cudaGraphExecDestroy(s->exec); s->exec = nullptr; }
+    for (int i = 0; i < 2; ++i)
+        if (alcs_stack_run(s, st) != ALCS_OK) return -1.0;
+    double best = 1e30;
+    for (int b = 0; b < 3; ++b) {
+        cudaEventRecord(e0, st);
+        for (int i = 0; i < reps; ++i)
+            if (alcs_stack_run(s, st) != ALCS_OK) return -1.0;
+        cudaEventRecord(e1, st);
+        if (cudaEventSynchronize(e1) != cudaSuccess) return -1.0;
+        float ms = 0;
+        cudaEventElapsedTime(&ms, e0, e1);
+        best = std::min(best, (double)ms * 1e3 / reps);
+    }
+    return best;
+}
+
+// The plans worth trying for one layer of a stack: what the last alcs_spconv1x1_tune of its shape ranked
+// best, else the model's best few and every shape of the small-problem kernel that applies.
+int stack_candidates(const alcs_stack::Item& it, std::vector<Plan>& out)
+{
+    const alcs_layer& L = it.layer;
+    const bool extra = (L.stride > 1) || L.residual;
+    out.clear();
+    {
+        std::lock_guard<std::mutex> lk(L.w->mu);
+        auto f = L.w->finalists.find(alcs::ShapeKey{L.n, it.oh, it.ow, L.flags});
+        if (f != L.w->finalists.end())
+            for (const Plan& p : f->second)
+                if (!(extra && p.gather)) out.push_back(p);
+    }
+    if (!out.empty()) return ALCS_OK;
+    std::vector<Plan> all;
+    const int rc = enumerate_plans(L.w, it.q, it.oh * it.ow, all, !extra);
+    if (rc) return rc;
+    for (size_t i = 0; i < all.size(); ++i)
+        if (i < 8 || all[i].gather) out.push_back(all[i]);
+    return ALCS_OK;
+}
+
+}  // namespace
+
+ALCS_API int alcs_stack_tune(alcs_stack* s, int passes, void* cuda_stream, double* us_before, double* us_after)
+{
+    if (!s || passes < 0) return ALCS_ERR_INVALID_ARG;
+    if (passes == 0) passes = 2;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) {
+        if (e0) cudaEventDestroy(e0);
+        (void)cudaGetLastError();
+        alcs::set_cuda_error_text("cudaEventCreate failed");
+        return ALCS_ERR_CUDA;
+    }
+    struct Done { cudaEvent_t a, b; ~Done() { cudaEventDestroy(a); cudaEventDestroy(b); } } done{e0, e1};
+    double cur = time_stack(s, st, e0, e1, 3);
+    if (cur < 0) return ALCS_ERR_CUDA;
+    const int reps = (int)std::min(100.0, std::max(3.0, 3000.0 / std::max(cur, 1.0)));     // batches of about 3 ms
+    cur = time_stack(s, st, e0, e1, reps);
+    if (cur < 0) return ALCS_ERR_CUDA;
+    if (us_before) *us_before = cur;
+    for (int pass = 0; pass < passes; ++pass) {
+        bool changed = false;
+        for (auto& it : s->items) {
+            if (it.q == 0) continue;
+            const alcs_layer& L = it.layer;
+            int rc = check_device(L.w);
+            if (rc) return rc;
+            std::vector<Plan> cands;
+            rc = stack_candidates(it, cands);
+            if (rc) return rc;
+            Plan best = it.plan;
+            double best_t = cur;
+            for (const Plan& c : cands) {
+                if (same_plan(c, best) || same_plan(c, it.plan)) continue;
+                if (c.gather) {
+                    if (ensure_canonical_on_device(L.w, nullptr) != ALCS_OK) continue;
+                } else {
+                    const KernelVariant& v = g_variants[c.variant].v;
+                    Schedule* sc = get_schedule(L.w, c.kc, c.n_rg, true, flavour_of(v));
+                    if (!sc || (v.split && sc->max_x == 0) || upload_schedule(L.w, sc, nullptr) != ALCS_OK) continue;
+                }
+                const Plan keep = it.plan;
+                it.plan = c;
+                const double t = time_stack(s, st, e0, e1, reps);
+                it.plan = keep;
+                // a candidate must beat the incumbent by more than the timing noise
+                if (t > 0 && t < best_t * 0.996) { best_t = t; best = c; }
+            }
+            if (!same_plan(best, it.plan)) {
+                it.plan = best;
+                cur = best_t;
+                changed = true;
+                alcs_launch_cfg c;
+                plan_to_cfg(best, &c);
+                const bool extra = (L.stride > 1) || L.residual;
+                std::lock_guard<std::mutex> lk(L.w->mu);
+                L.w->tuned[alcs::ShapeKey{L.n, it.oh, it.ow, L.flags}] = c;
+                L.w->plan_cache[alcs::ShapeKey{L.n, it.oh, it.ow, L.flags | (extra ? kStagedOnly : 0u)}] = best;
+            }
+        }
+        if (!changed) break;
+    }
+    cur = time_stack(s, st, e0, e1, reps);      // (also leaves a graph stack captured with the chosen plans)
+    if (cur < 0) return ALCS_ERR_CUDA;
+    if (us_after) *us_after = cur;
+    return ALCS_OK;
+}
+
+ALCS_API int alcs_stack_layer_cfg(const alcs_stack* s, int layer, alcs_launch_cfg* out)
+{
+    if (!s || !out || layer < 0 || layer >= (int)s->items.size()) return ALCS_ERR_INVALID_ARG;
+    std::memset(out, 0, sizeof *out);
+    if (s->items[layer].q == 0) return ALCS_OK;
+    plan_to_cfg(s->items[layer].plan, out);
     return ALCS_OK;
 }
 

@@ -12,6 +12,7 @@
 // It walks the canonical storage format (row_ptr / col_idx / vals), not a launch schedule.
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cstdint>
 
 #include "alcs_gather.h"
@@ -46,7 +47,7 @@ __device__ __forceinline__ void load_weights(const float* __restrict__ p, float 
 template <int G, int P, bool VEC>
 __global__ void __launch_bounds__(512) gather_kernel(const GatherArgs a)
 {
-    extern __shared__ float red[];                       // [KS][G*P][32]
+    extern __shared__ __align__(16) float red[];         // [KS][G*P][32]
     const int lane = threadIdx.x & 31;
     const int ks = threadIdx.x >> 5;
     const int KS = blockDim.x >> 5;
@@ -74,7 +75,24 @@ __global__ void __launch_bounds__(512) gather_kernel(const GatherArgs a)
     asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
     const int k_first = __ldg(a.row_ptr + r);
     const int k1 = __ldg(a.row_ptr + r + 1);
-    {
+    // Rows that fit are copied into shared memory (the area the partial sums use later) before the wait, so
+    // that afterwards only the input vectors remain to be fetched: one memory round trip per batch of blocks
+    // instead of two dependent ones (column index, then the input it addresses).
+    const bool staged = a.stage_blocks > 0 && k1 - k_first <= a.stage_blocks;
+    int* scol = reinterpret_cast<int*>(red);                         // [stage_blocks]
+    float* sval = red + ((a.stage_blocks + 3) & ~3);                 // [stage_blocks][G], 16-byte aligned
+    if (staged) {
+        const int nbk = k1 - k_first;
+        for (int i = threadIdx.x; i < nbk; i += blockDim.x) scol[i] = __ldg(a.col_idx + k_first + i);
+        const float* vsrc = a.vals + (size_t)k_first * G;
+        if constexpr (G % 4 == 0) {
+            for (int i = threadIdx.x; i < nbk * (G / 4); i += blockDim.x)
+                reinterpret_cast<float4*>(sval)[i] = __ldg(reinterpret_cast<const float4*>(vsrc) + i);
+        } else {
+            for (int i = threadIdx.x; i < nbk * G; i += blockDim.x) sval[i] = __ldg(vsrc + i);
+        }
+        __syncthreads();
+    } else {
         const char* cb = reinterpret_cast<const char*>(a.col_idx + k_first);
         const char* vb = reinterpret_cast<const char*>(a.vals + (size_t)k_first * G);
         const long long cbytes = (long long)(k1 - k_first) * 4, vbytes = cbytes * G;
@@ -91,8 +109,19 @@ __global__ void __launch_bounds__(512) gather_kernel(const GatherArgs a)
         for (int u = 0; u < kUnroll; ++u) {
             const int kk = k + u * KS;
             const bool on = kk < k1;
-            const int col = on ? __ldg(a.col_idx + kk) : 0;
-            if (on) {
+            const int col = on ? (staged ? scol[kk - k_first] : __ldg(a.col_idx + kk)) : 0;
+            if (on && staged) {
+                if constexpr (G % 4 == 0) {
+#pragma unroll
+                    for (int i = 0; i < G / 4; ++i) {
+                        const float4 v = reinterpret_cast<const float4*>(sval)[(kk - k_first) * (G / 4) + i];
+                        w[u][4 * i] = v.x; w[u][4 * i + 1] = v.y; w[u][4 * i + 2] = v.z; w[u][4 * i + 3] = v.w;
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < G; ++j) w[u][j] = sval[(kk - k_first) * G + j];
+                }
+            } else if (on) {
                 load_weights<G>(a.vals + (size_t)kk * G, w[u]);
             } else {
 #pragma unroll
@@ -120,6 +149,7 @@ __global__ void __launch_bounds__(512) gather_kernel(const GatherArgs a)
     }
 
     // add the warps' partial sums in warp order, then bias, ReLU, store
+    if (staged) __syncthreads();        // (the staged row shares the area of the partial sums)
 #pragma unroll
     for (int j = 0; j < G; ++j)
 #pragma unroll
@@ -143,7 +173,8 @@ __global__ void __launch_bounds__(512) gather_kernel(const GatherArgs a)
 template <int G, int P>
 cudaError_t launch_gp(const GatherArgs& a, bool vec, unsigned grid, int ks, cudaStream_t st)
 {
-    const size_t smem = (size_t)ks * G * P * 32 * sizeof(float);
+    const size_t red_bytes = (size_t)ks * G * P * 32 * sizeof(float);
+    const size_t smem = std::max(red_bytes, (size_t)a.stage_blocks * 4 * (G + 1) + 16);
     // launched so that it may overlap the tail of the kernel before it on the stream (it waits for that
     // kernel before it touches x or y); a CUDA graph keeps the same programmatic edge
     cudaLaunchConfig_t lc = {};
@@ -185,6 +216,12 @@ bool gather_config_ok(int g, int p, int ks, bool vec)
     if (p == 2 && vec) return false;
     if (ks < 1 || ks > 16) return false;
     return (size_t)ks * g * p * 32 * sizeof(float) <= 48 * 1024;
+}
+
+int gather_stage_blocks(int g, int max_row_blocks)
+{
+    if (max_row_blocks <= 0) return 0;
+    return (size_t)max_row_blocks * 4 * (g + 1) + 16 <= 48 * 1024 ? max_row_blocks : 0;
 }
 
 cudaError_t launch_gather(int g, int p, int ks, const GatherArgs& a, cudaStream_t st)

@@ -119,13 +119,16 @@ struct alcs_packed {
     mutable int32_t* d_col_idx = nullptr;
     mutable void* d_vals = nullptr;
     mutable size_t xpad_bytes = 0;
+    mutable int max_row_blocks = -1;  // blocks of the longest block row (computed on first use)
     // by (kc, n_rg), built on demand; the tensor-core flavour of a schedule is stored under -kc
     mutable std::map<std::pair<int, int>, alcs::Schedule> sched;
     // schedules of the general k x k convolution, by {row groups, words per channel, words per parity
     // plane, plane pitch, stride, kh, kw, channels per chunk}: the column offsets baked into them depend
     // on the geometry
     mutable std::map<std::array<int, 8>, alcs::Schedule> sched2d;
-    std::map<alcs::ShapeKey, alcs_launch_cfg> tuned;   // filled by alcs_spconv1x1_tune
+    mutable std::map<alcs::ShapeKey, alcs_launch_cfg> tuned;   // filled by alcs_spconv1x1_tune, alcs_spconv1x1_set_cfg, alcs_stack_tune
+    // the best few plans of the last alcs_spconv1x1_tune per shape, best first: what alcs_stack_tune tries in context
+    mutable std::map<alcs::ShapeKey, std::vector<alcs::Plan>> finalists;
     mutable std::map<alcs::ShapeKey, alcs::Plan> plan_cache;   // resolved plans, by shape
     mutable std::mutex mu;                                      // guards plan_cache and sched
     size_t elt() const { return dt == ALCS_F32 ? 4 : 2; }

@@ -124,6 +124,57 @@ def test_stack_layers_with_stride_and_residual(alcs):
         alcs.alcs_stack_destroy(st)
 
 
+@pytest.mark.parametrize("graph", [False, True])
+def test_stack_tuned_in_context_stays_correct(alcs, graph):
+    """alcs_stack_tune swaps launch configurations (and, at batch 1, kernels) while timing the whole stack:
+    afterwards every layer must still match the oracle, the reported configurations must be the ones a
+    fresh stack resolves to, and the times must be positive."""
+    import torch
+    dev = torch.device("cuda:0")
+    specs = [(1, 64, 64, 14, 14, 4, 1, False), (1, 64, 96, 14, 14, 4, 1, True), (1, 96, 48, 14, 14, 4, 2, False), (1, 48, 40, 7, 7, 4, 1, False)]
+    layers, keep = [], []
+    stream = torch.cuda.Stream()
+    for i, (n, cin, cout, h, wd, g, s, with_res) in enumerate(specs):
+        W, M, X, b, R = _case(1200 + i, n, cin, cout, h, wd, g, 0.4, s)
+        if not with_res:
+            R = None
+        p = alcs.alcs_packed_upload(alcs.alcs_pack(W, M, g), 0)
+        oh, ow = -(-h // s), -(-wd // s)
+        xd = torch.from_numpy(X).to(dev)
+        yd = torch.full((n, cout, oh * ow), float("nan"), device=dev)
+        rd = None if R is None else torch.from_numpy(R).to(dev)
+        bd = torch.from_numpy(b).to(dev)
+        if i == 0:      # one layer with finalists of its own tuning run, the others from the cost model
+            with torch.cuda.stream(stream):
+                alcs.alcs_spconv1x1_tune(p, xd, yd, n, h, wd, bd, alcs.ALCS_RELU, stream)
+        layers.append(dict(w=p, x=xd, y=yd, n=n, h=h, wd=wd, bias=bd, flags=alcs.ALCS_RELU, residual=rd, stride=s))
+        keep.append((W, M, X, b, R, g, s, yd))
+    st = alcs.alcs_stack_create(layers, alcs.ALCS_STACK_GRAPH if graph else 0)
+    with torch.cuda.stream(stream):
+        before, after = alcs.alcs_stack_tune(st, 2, stream)
+    assert before > 0 and after > 0
+    cfgs = [alcs.alcs_stack_layer_cfg(st, i) for i in range(len(layers))]
+    assert all(c["pixels_per_lane"] > 0 for c in cfgs)
+    assert all(c["math_mode"] != 3 for c, sp in zip(cfgs, specs) if sp[6] > 1 or sp[7])   # (that kernel takes neither)
+    for k in keep:
+        k[7].fill_(float("nan"))
+    torch.cuda.synchronize()
+    alcs.alcs_stack_run(st, stream)
+    stream.synchronize()
+    for W, M, X, b, R, g, s, yd in keep:
+        Yref, A = oracle.conv1x1_ex(W, M, X, b, R, True, g, s, want_scale=True)
+        assert_parity(yd.cpu().numpy(), Yref, A, "f32")
+    alcs.alcs_stack_destroy(st)
+    st2 = alcs.alcs_stack_create(layers, 0)     # the packed matrices remember what the tuning chose
+    assert [alcs.alcs_stack_layer_cfg(st2, i) for i in range(len(layers))] == cfgs
+    alcs.alcs_stack_destroy(st2)
+    empty = alcs.alcs_stack_create([], 0)
+    with pytest.raises(alcs.AlcsError):
+        alcs.alcs_stack_layer_cfg(empty, 0)
+    assert alcs.alcs_stack_tune(empty, 1, stream)[1] >= 0
+    alcs.alcs_stack_destroy(empty)
+
+
 def test_argument_errors(alcs):
     import torch
     dev = torch.device("cuda:0")

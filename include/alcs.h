@@ -167,7 +167,12 @@ ALCS_API void alcs_packed_free(alcs_packed* p);
  *                     that are not a multiple of 16 bytes long are first repacked into a scratch tensor
  *                     with padded rows; 3 = per-lane cp.async of 8 bytes straight from X, without that
  *                     pass, for rows that are a multiple of 8 but not of 16 bytes long (16-bit elements,
- *                     14x14 images), stride 1 and X on an 8-byte boundary; elsewhere 3 acts like 1
+ *                     14x14 images), stride 1 and X on an 8-byte boundary; elsewhere 3 acts like 1;
+ *                     4 = X is first copied (one more kernel, into the same scratch) into a tile-major
+ *                     layout [pixel tile][channel][tile pixels], so that the channel rows of a chunk lie one
+ *                     after the other and a work item stages them with a few large bulk (TMA) copies: the
+ *                     staging then costs the kernel next to no instructions, at the price of one more pass
+ *                     over X where its rows would not have needed repacking.  Batches of more than 8 images
  *   producer_warps    warps of the thread block that only move data (1..4)
  *   math_mode         1 = fp32 FMA on the CUDA cores; 2 = tensor cores (fp16 weights and activations
  *                     only): 16 kept blocks of a block row times the 16 input rows they select is a
@@ -269,7 +274,7 @@ ALCS_API int alcs_spconv1x1_plan(const alcs_packed* w, int n, int h, int wd, uns
  * buffers (y is overwritten with the correct result each time), remember the fastest in w for
  * later alcs_spconv1x1 calls with the same (n, h, wd, flags), and write it to *best (may be
  * NULL).  Every launch is timed with cold caches (a buffer larger than L2 is rewritten before it):
- * each candidate three times, then the eight best fifteen times more in turn, and the lowest median
+ * each candidate three times, then the twelve best fifteen times more in turn, and the lowest median
  * wins.  Synchronises the stream; meant for set-up time, never for the timed path.
  */
 ALCS_API int alcs_spconv1x1_tune(alcs_packed* w, const void* x, void* y, int n, int h, int wd,
@@ -509,9 +514,9 @@ ALCS_API int alcs_stack_destroy(alcs_stack* s);
  * alone, with cold caches and nothing before it on the stream; inside a stack a layer starts while its
  * predecessor drains (programmatic dependent launch), finds whatever the earlier layers left in L2, and, at
  * batch 1, costs little more than its launch, so the configuration that wins alone is not always the one
- * that wins there.  For every layer in turn this call tries the candidates (the best eight of the last
- * alcs_spconv1x1_tune for the layer's shape if there was one, else the cost model's best eight and every
- * shape of the small-problem kernel that applies), each time timing the WHOLE stack the way alcs_stack_run
+ * that wins there.  For every layer in turn this call tries the candidates (the best twelve of the last
+ * alcs_spconv1x1_tune for the layer's shape if there was one, else the cost model's best eight; for batches
+ * of at most 8 images also every shape of the small-problem kernel that applies), each time timing the WHOLE stack the way alcs_stack_run
  * runs it (a graph stack is captured again), and keeps a candidate only if the stack gets faster by more
  * than 0.4 %; `passes` sweeps over the layers (0 = 2), stopping early when a sweep changes nothing.  The
  * chosen configurations are also remembered in the packed matrices for later calls with the same shape.

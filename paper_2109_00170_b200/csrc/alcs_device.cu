@@ -295,6 +295,9 @@ bool gather_plan(const alcs_packed* w, int n, int hw, int p, int ks, const Devic
 // the rows repacked?
 bool direct_rows_ok(int hw, int elt) { return ((size_t)hw * elt) % 16 == 8; }
 
+// How many of the best candidates the tuner times a second time and remembers for alcs_stack_tune.
+constexpr size_t kFinalists = 12;
+
 // Enumerate every valid launch configuration for this shape, cheapest (by the model) first.
 // Internal flag, only ever seen in plan-cache keys: the call has a residual operand or a stride, which
 // the small-problem kernel does not take, so only the staged kernels are listed.
@@ -372,6 +375,16 @@ int enumerate_plans(const alcs_packed* w, long long q, int hw, std::vector<Plan>
                         p3.bulk = 2;
                         p3.cost *= 1.1;
                         out.push_back(p3);
+                    }
+                    // A tile-major copy of X first (one more pass over X where its rows need no repacking
+                    // anyway), then a chunk is staged by a few large bulk copies: no copy instructions to
+                    // speak of, so one producer warp is enough.
+                    if (v.npw <= 2 && q > 8ll * hw) {
+                        Plan p4 = p;
+                        p4.bulk = 3;
+                        const double pass = 2.0 * (double)q * w->cin * elt / di.hbm_bps + 3e-6;
+                        p4.cost = p.cost * 0.9 + ((((size_t)hw * elt) % 16 == 0) ? pass : 0.0);
+                        out.push_back(p4);
                     }
                 }
             }
@@ -520,8 +533,83 @@ __global__ void repack_rows_kernel(const T* __restrict__ in, T* __restrict__ out
     }
 }
 
+// The same copy into a TILE-MAJOR layout: out[tile][channel][tile_px pixels (+ padding up to rowb elements)],
+// where pixel q = image * hwp + p of the padded pixel axis lies in tile q / tile_px.  A work item of the
+// convolution kernel then finds the channel rows of its tile one after the other and stages a whole chunk
+// of them with a few large bulk copies.  Pixels beyond the last image are written as zeros.
+template <typename T>
+__global__ void repack_tiles_kernel(const T* __restrict__ in, T* __restrict__ out, int n, int cin, int hw_in, int wd_in,
+                                    int ow, int stride, int hw_out, int hwp, int tile_px, int rowb, long long n_tiles)
+{
+    constexpr int EPV = 16 / (int)sizeof(T);
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const int vpr = tile_px / EPV;                   // 16-byte pieces per (tile, channel) row
+    const long long total = n_tiles * cin * vpr;
+    const long long q_total = (long long)n * hwp;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
+         i += (long long)gridDim.x * blockDim.x) {
+        const long long row = i / vpr;
+        const int piece = (int)(i - row * vpr);
+        const long long tile = row / cin;
+        const int c = (int)(row - tile * cin);
+        const long long q = tile * tile_px + (long long)piece * EPV;
+        alignas(16) T v[EPV];
+        if (q < q_total) {
+            const long long img = q / hwp;
+            const int p0 = (int)(q - img * hwp);      // (hwp is a multiple of EPV: the piece lies in one image)
+            const T* src = in + ((size_t)img * cin + c) * hw_in;
+#pragma unroll
+            for (int t = 0; t < EPV; ++t) {
+                const int p = p0 + t;
+                if (p >= hw_out) { v[t] = T(0); continue; }
+                if (stride == 1) {
+                    v[t] = __ldg(src + p);
+                } else {
+                    const int oy = p / ow, ox = p - oy * ow;
+                    v[t] = __ldg(src + (size_t)oy * stride * wd_in + (size_t)ox * stride);
+                }
+            }
+        } else {
+#pragma unroll
+            for (int t = 0; t < EPV; ++t) v[t] = T(0);
+        }
+        *reinterpret_cast<uint4*>(out + (size_t)row * rowb + (size_t)piece * EPV) = *reinterpret_cast<const uint4*>(v);
+    }
+}
+
 // pixels per image after padding the rows of X to a multiple of 16 bytes
 int padded_hw(int hw, int elt) { const int m = 16 / elt; return (hw + m - 1) / m * m; }
+
+// Bytes per channel row of a pixel tile in shared memory and in the tile-major copy of X.
+int tile_row_bytes(const KernelVariant& v, int elt) { return 32 * v.p * elt + (v.mma ? 16 : 0); }
+
+// Bytes of the tile-major copy of X for kernel variant v: n images of hw pixels (rows padded to 16 bytes).
+size_t tiled_bytes(const KernelVariant& v, int elt, int n, int cin, int hw)
+{
+    const long long q = (long long)n * padded_hw(hw, elt);
+    const long long tiles = (q + 32 * v.p - 1) / (32 * v.p);
+    return (size_t)tiles * cin * tile_row_bytes(v, elt);
+}
+
+int launch_repack_tiles(const KernelVariant& v, int elt, const void* x, void* out, int n, int cin, int h_in, int wd_in,
+                        int ow, int stride, int hw, int sms, cudaStream_t st)
+{
+    const int hwp = padded_hw(hw, elt);
+    const int T = 32 * v.p;
+    const long long tiles = ((long long)n * hwp + T - 1) / T;
+    const long long pieces = tiles * cin * (T * elt / 16);
+    const unsigned blocks = (unsigned)std::min<long long>((pieces + 255) / 256, (long long)sms * 8);
+    const int rowb = tile_row_bytes(v, elt) / elt;
+    if (elt == 4)
+        repack_tiles_kernel<float><<<blocks, 256, 0, st>>>(static_cast<const float*>(x), static_cast<float*>(out), n, cin,
+                                                          h_in * wd_in, wd_in, ow, stride, hw, hwp, T, rowb, tiles);
+    else
+        repack_tiles_kernel<unsigned short><<<blocks, 256, 0, st>>>(static_cast<const unsigned short*>(x),
+                                                                   static_cast<unsigned short*>(out), n, cin, h_in * wd_in,
+                                                                   wd_in, ow, stride, hw, hwp, T, rowb, tiles);
+    ALCS_CUDA(cudaGetLastError());
+    return ALCS_OK;
+}
 
 // Make sure the scratch of w can hold `bytes`.  Growing it frees the old block, which waits for
 // all earlier work on the device.
@@ -646,7 +734,20 @@ int launch_plan(const alcs_packed* w, const Plan& p, const void* x, void* y, int
     int hwx = hw;
     const void* xk = x;
     const bool direct = p.bulk == 2 && stride == 1 && direct_rows_ok(hw, elt) && (uintptr_t)x % 8 == 0;
-    if ((((size_t)hw * elt) % 16 != 0 && !direct) || stride != 1) {
+    bool tiled = false;
+    if (p.bulk == 3 && (long long)n * padded_hw(hw, elt) <= (1ll << 30)) {
+        // tile-major copy of X (also gathers the pixels a strided convolution reads)
+        const size_t need = tiled_bytes(v, elt, n, w->cin, hw);
+        if (scratch ? scratch_bytes >= need : ensure_xpad(w, need) == ALCS_OK) {
+            void* const xt = scratch ? scratch : w->d_xpad;
+            rc = launch_repack_tiles(v, elt, x, xt, n, w->cin, h_in, wd_in, wd, stride, hw, di.sms, st);
+            if (rc) return rc;
+            xk = xt;
+            hwx = padded_hw(hw, elt);
+            tiled = true;
+        }       // else: staged like copy mode 1
+    }
+    if (!tiled && ((((size_t)hw * elt) % 16 != 0 && !direct) || stride != 1)) {
         const int hwp = padded_hw(hw, elt);
         const size_t need = (size_t)n * w->cin * hwp * elt;
         if (scratch && scratch_bytes < need) return ALCS_ERR_STATE;
@@ -688,7 +789,7 @@ int launch_plan(const alcs_packed* w, const Plan& p, const void* x, void* y, int
     int ld = 16;
     while (ld > elt && (((size_t)hwx * elt) % ld || (uintptr_t)xk % ld)) ld >>= 1;
     a.ld_bytes = ld;
-    a.bulk = (ld == 16 && p.bulk == 1) ? 1 : 0;
+    a.bulk = tiled ? 2 : (ld == 16 && p.bulk == 1) ? 1 : 0;
     a.ros = sc->ros;
     const int vg = (v.p * elt >= 16) ? 16 / elt : v.p;
     a.st_vec = (hwx == hw && hw % vg == 0 && (uintptr_t)y % 16 == 0 && (uintptr_t)residual % 16 == 0) ? 1 : 0;
@@ -1018,7 +1119,7 @@ ALCS_API int alcs_spconv1x1_tune(alcs_packed* w, const void* x, void* y, int n, 
     // Second pass: the few best candidates differ by less than the noise of three launches, so they
     // are timed again, in turn, and the one with the lowest median wins.
     std::sort(ranked.begin(), ranked.end());
-    if (ranked.size() > 8) ranked.resize(8);
+    if (ranked.size() > kFinalists) ranked.resize(kFinalists);
     int best_i = -1;
     float best_ms = 1e30f;
     const int rounds = 15;
@@ -1156,6 +1257,10 @@ ALCS_API int alcs_stack_create(const alcs_layer* layers, int n_layers, unsigned 
             const long long hw = (long long)it.oh * it.ow;
             if (!rc && ((hw * elt) % 16 != 0 || stride > 1) && (long long)L.n * padded_hw((int)hw, elt) <= (1ll << 30))
                 scratch_need = std::max(scratch_need, (size_t)L.n * L.w->cin * padded_hw((int)hw, elt) * elt);
+            // room for the tile-major copy of X that copy mode 4 makes, for any tile width (alcs_stack_tune
+            // may switch a layer to it)
+            if (!rc && (long long)L.n * padded_hw((int)hw, elt) <= (1ll << 30) && it.q > 8 * hw)
+                scratch_need = std::max(scratch_need, ((size_t)L.n * padded_hw((int)hw, elt) + 512) * L.w->cin * (elt + 1));
         }
         if (rc) { delete s; return rc; }
         s->items.push_back(it);
@@ -1267,12 +1372,18 @@ int stack_candidates(const alcs_stack::Item& it, std::vector<Plan>& out)
             for (const Plan& p : f->second)
                 if (!(extra && p.gather)) out.push_back(p);
     }
-    if (!out.empty()) return ALCS_OK;
+    const bool had = !out.empty();
+    const bool small = !extra && it.oh * it.ow > 0 && it.q / ((long long)it.oh * it.ow) <= 8;
+    if (had && !small) return ALCS_OK;
     std::vector<Plan> all;
     const int rc = enumerate_plans(L.w, it.q, it.oh * it.ow, all, !extra);
     if (rc) return rc;
-    for (size_t i = 0; i < all.size(); ++i)
-        if (i < 8 || all[i].gather) out.push_back(all[i]);
+    for (size_t i = 0; i < all.size(); ++i) {
+        if (!((!had && i < 8) || all[i].gather)) continue;
+        bool dup = false;
+        for (const Plan& p : out) dup |= same_plan(p, all[i]);
+        if (!dup) out.push_back(all[i]);
+    }
     return ALCS_OK;
 }
 
@@ -1434,7 +1545,19 @@ extern "C" ALCS_API int alcs_spconv1x1_noalloc(const alcs_packed* w, const void*
     int hwx = hw;
     const void* xk = x;
     const bool direct = plan.bulk == 2 && direct_rows_ok(hw, elt) && (uintptr_t)x % 8 == 0;
-    if (((size_t)hw * elt) % 16 != 0 && !direct) {
+    bool tiled = false;
+    if (plan.bulk == 3 && (long long)n * padded_hw(hw, elt) <= (1ll << 30) &&
+        tiled_bytes(v, elt, n, w->cin, hw) <= ALCS_NOALLOC_SCRATCH_BYTES) {
+        void* scratch = nullptr;
+        rc = noalloc_scratch_address(w->device, &scratch);
+        if (rc) return rc;
+        rc = launch_repack_tiles(v, elt, x, scratch, n, w->cin, h, wd, wd, 1, hw, di.sms, st);
+        if (rc) return rc;
+        xk = scratch;
+        hwx = padded_hw(hw, elt);
+        tiled = true;
+    }
+    if (!tiled && ((size_t)hw * elt) % 16 != 0 && !direct) {
         // rows that cannot be staged with 16-byte copies: repack into the fixed array
         const int hwp = padded_hw(hw, elt);
         const unsigned long long need = (unsigned long long)n * w->cin * hwp * elt;
@@ -1477,7 +1600,7 @@ extern "C" ALCS_API int alcs_spconv1x1_noalloc(const alcs_packed* w, const void*
     int ld = 16;
     while (ld > elt && (((size_t)hwx * elt) % ld || (uintptr_t)xk % ld)) ld >>= 1;
     a.ld_bytes = ld;
-    a.bulk = (ld == 16 && plan.bulk == 1) ? 1 : 0;
+    a.bulk = tiled ? 2 : (ld == 16 && plan.bulk == 1) ? 1 : 0;
     a.ros = sc->ros;
     const int vg = (v.p * elt >= 16) ? 16 / elt : v.p;
     a.st_vec = (hwx == hw && hw % vg == 0 && (uintptr_t)y % 16 == 0) ? 1 : 0;

@@ -71,7 +71,9 @@ struct ConvArgs {
     int relu;
     int y_f32;                // only meaningful for XT = __half
     int ld_bytes;             // bytes per X staging copy: 16, 8, 4 or 2
-    int bulk;                 // 1: the producer uses bulk (TMA) copies; needs ld_bytes == 16
+    int bulk;                 // 1: the producer uses bulk (TMA) copies; needs ld_bytes == 16.  2: the same, and x is a
+                              // tile-major copy of the input: [pixel tile][channel][32*P pixels (+ row padding)], so
+                              // that the channel rows of a chunk are one contiguous run
     int ros;                  // ints of rowoff per (row group, chunk): 4 per header
     int st_vec;               // 1 if vector stores are allowed
     int st_grp;               // 1 if the pixels of one vector store of a lane always lie in one image; 2 (tensor-core
@@ -624,7 +626,9 @@ __device__ __forceinline__ void produce_bulk(const ConvArgs& a, unsigned char* s
                 const int nrows = min(a.kc, a.cin - cbase);
                 const int r0 = __shfl_sync(0xffffffffu, sl_lo, k & 31);
                 const int rbytes = (__shfl_sync(0xffffffffu, sl_hi, k & 31) - r0) * 16;
-                if (lane == 0 && pw == 0) mbar_arrive_expect_tx(bar, (uint32_t)(nrows * vt * SZ + rbytes + a.ros * 4));
+                const bool tiled = a.bulk == 2;
+                if (lane == 0 && pw == 0)
+                    mbar_arrive_expect_tx(bar, (uint32_t)(nrows * (tiled ? ROWB : vt * SZ) + rbytes + a.ros * 4));
                 __syncwarp();
                 if (lane == 0 && pw == 0 && rbytes > 0) bulk_copy_g2s(st + a.off_rec, a.rec + (size_t)r0 * 16, (uint32_t)rbytes, bar);
                 if (lane == 1 && pw == 0)
@@ -632,8 +636,16 @@ __device__ __forceinline__ void produce_bulk(const ConvArgs& a, unsigned char* s
                 // X (or its repacked copy) is the predecessor kernel's output: wait for it once,
                 // after the first weight copies are already in flight
                 if (!dep_ok) { grid_dep_wait(); dep_ok = true; }
+                if (tiled) {
+                    // the chunk's channel rows of this tile lie one after the other: copies of eight rows each
+                    const unsigned char* src = static_cast<const unsigned char*>(a.x) + ((size_t)tile * a.cin + cbase) * ROWB;
+                    const uint32_t total = (uint32_t)nrows * ROWB;
+                    constexpr uint32_t PIECE = 8 * ROWB;
+                    for (uint32_t o = (uint32_t)(lane + 32 * pw) * PIECE; o < total; o += 32u * npw * PIECE)
+                        bulk_copy_g2s(st + o, src + o, min(PIECE, total - o), bar);
+                }
                 // X: channel rows lane, lane+32, ...; each row is one copy per image it touches
-                for (int c = lane + 32 * pw; c < nrows; c += 32 * npw) {
+                for (int c = lane + 32 * pw; c < nrows && !tiled; c += 32 * npw) {
                     const unsigned char* src = xbase + (size_t)(cbase + c) * ch_bytes;
                     uint32_t dst = st + c * ROWB;
                     int left = vt, p = p0;

@@ -505,6 +505,21 @@ def bench_conv2d(args):
     print(json.dumps(out))
 
 
+def kernels_per_layer(spec, cfg):
+    """Kernel launches one layer costs: the convolution kernel, plus the pass that repacks X when its rows
+    are not 16-byte multiples (unless they are staged as they are, copy_mode 3) or that makes the
+    tile-major copy (copy_mode 4).  The small-problem kernel (math_mode 3) never repacks."""
+    if cfg.get("math_mode") == 3:
+        return 1
+    row_bytes = spec.hw * (4 if spec.dtype == "f32" else 2)
+    cm = cfg.get("copy_mode")
+    if cm == 4:
+        return 2
+    if row_bytes % 16 == 0 or (cm == 3 and row_bytes % 16 == 8):
+        return 1
+    return 2
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -646,6 +661,11 @@ def main():
 
     # ---- region B: the same steps with an event between layers (per-layer durations) --------
     nl = len(layers)
+    # (one untimed pass through the per-layer entry point first: a packed matrix allocates its own repacking
+    # scratch on its first such call, the stack above used the stack's)
+    for L in layers:
+        A.alcs_spconv1x1(L["w"], L["x"], L["y"], L["n"], L["h"], L["wd"], L["bias"], L["flags"], stream, L["cfg"])
+    torch.cuda.synchronize()
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(nl + 1)] for _ in range(args.steps)]
     for k in range(args.steps):
         evs[k][0].record(stream)
@@ -657,6 +677,8 @@ def main():
     clocks = sampler.stop(tw0, tw1) if rank == 0 else None
     per_layer_ms = [statistics.mean(evs[k][i].elapsed_time(evs[k][i + 1]) for k in range(args.steps)) for i in range(nl)]
     per_layer_min = [min(evs[k][i].elapsed_time(evs[k][i + 1]) for k in range(args.steps)) for i in range(nl)]
+    per_layer_med = [statistics.median(evs[k][i].elapsed_time(evs[k][i + 1]) for k in range(args.steps)) for i in range(nl)]
+    per_layer_max = [max(evs[k][i].elapsed_time(evs[k][i + 1]) for k in range(args.steps)) for i in range(nl)]
 
     ms_total = max_over_ranks(ms_total, world, dev)
     ms_step = ms_total / args.steps
@@ -708,14 +730,14 @@ def main():
 
     # ---- per-layer roofline ------------------------------------------------------------------
     rows = []
-    for st, ms, mn in zip(stats, per_layer_ms, per_layer_min):
+    for st, ms, mn, md, mx in zip(stats, per_layer_ms, per_layer_min, per_layer_med, per_layer_max):
         t_hbm = st["bytes"] / (hbm_gbs * 1e9)
         t_alu = st["flops"] / (fp32_tf * 1e12)
         t_roof = max(t_hbm, t_alu)
         rows.append(dict(layer=st["name"], sparsity=round(st["sparsity"], 4), kept_blocks=st["nb"],
                          nz_mflop=round(st["flops"] / 1e6, 1), mbytes=round(st["bytes"] / 1e6, 2),
                          t_roof_us=round(t_roof * 1e6, 2), bound="hbm" if t_hbm >= t_alu else "alu",
-                         us=round(ms * 1e3, 2), us_min=round(mn * 1e3, 2),
+                         us=round(ms * 1e3, 2), us_min=round(mn * 1e3, 2), us_median=round(md * 1e3, 2), us_max=round(mx * 1e3, 2),
                          nz_gflops=round(st["flops"] / (ms * 1e-3) / 1e9, 1),
                          frac=round(t_roof / (ms * 1e-3), 4), cfg=st["cfg"]))
     dom = max(range(nl), key=lambda i: per_layer_ms[i])
@@ -760,7 +782,8 @@ def main():
                            "frac": round(sum_roof / sum_us, 4), "min_layer_frac": min(r["frac"] for r in rows),
                            "step_frac": round(sum_roof / (ms_step * 1e3), 4),
                            "us_per_layer": round(ms_step * 1e3 / nl, 2)},
-        "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": nl * args.steps, "clocks": clocks,
+        "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": sum(kernels_per_layer(sp, st["cfg"]) for sp, st in zip(specs, stats)) * args.steps,
+        "clocks": clocks,
         "batch1": batch1, "layers": rows,
     }
     print(json.dumps(out))
